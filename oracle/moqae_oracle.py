@@ -1,0 +1,551 @@
+"""CPU oracle for the MoQAE inference hot path.  TEST INFRASTRUCTURE ONLY.
+
+This module is the slow, plain reference that the CUDA library is checked
+against.  It is written from the paper's definitions (Section 3.1 overview,
+Section 3.2 Eq. 1 and Eq. 2, Section 3.4 routing freezing / routing sharing,
+and the Limitations section's "dequantise, then attend in high precision") and
+from the storage format fixed in this repository.  It shares no code with the
+CUDA path and must never be imported by the product package: only the tests,
+the smoke check and the benchmark's CPU-baseline leg may call it.
+
+Arithmetic: the router and attention are evaluated in float64 from the exact
+values of the 16-bit inputs.  The quantiser follows a fixed sequence of
+single IEEE binary32 operations (stated in `quantize_groups`) so that integer
+codes and packed words have exactly one correct value.
+
+Parity pins (see tests, all CPU-only):
+  * attention   - pinned (textbook softmax attention, library SDPA, invariants)
+  * quantiser   - pinned (error bound, brute force over fp16 pairs, lossless
+                  integer case, constant groups)
+  * packing     - pinned (closed-form sizes, independent bit-position check,
+                  round trip)
+  * router      - pinned (hand-built score matrices with every tie pattern,
+                  brute force, library GEMV in linear mode); the paper prints
+                  no worked example, so beyond these definitional pins the
+                  router and quantiser are "parity unpinned by the paper".
+
+Input convention: 16-bit tensors arrive as numpy uint16 bit patterns plus a
+dtype flag (0 = IEEE fp16, 1 = bfloat16), because numpy has no bfloat16.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+EXPERT_BITS = (2, 4, 8, 16)      # expert index -> bit width (ascending)
+N_EXPERTS = 4
+HEAD_DIM = 128
+GROUP = 32                        # quantisation group length
+TILE_TOKENS = 32                  # tokens per storage tile (= one key group)
+META_BYTES = 1024                 # per quantised tile
+DT_FP16 = 0
+DT_BF16 = 1
+
+
+# ----------------------------------------------------------------------------
+# exact conversions
+# ----------------------------------------------------------------------------
+def to_f32(u16: np.ndarray, dtype: int) -> np.ndarray:
+    """Exact value of fp16 / bf16 bit patterns as float32."""
+    u16 = np.ascontiguousarray(u16, dtype=np.uint16)
+    if dtype == DT_FP16:
+        return u16.view(np.float16).astype(np.float32)
+    if dtype == DT_BF16:
+        return (u16.astype(np.uint32) << np.uint32(16)).view(np.float32)
+    raise ValueError("dtype must be 0 (fp16) or 1 (bf16)")
+
+
+def to_f64(u16: np.ndarray, dtype: int) -> np.ndarray:
+    return to_f32(u16, dtype).astype(np.float64)
+
+
+def fp16_round_down(x32: np.ndarray) -> np.ndarray:
+    """Largest fp16 value <= x (x float32)."""
+    x32 = np.asarray(x32, dtype=np.float32)
+    with np.errstate(over="ignore"):
+        h = x32.astype(np.float16)                      # round to nearest even
+    too_big = h.astype(np.float32) > x32
+    return np.where(too_big, np.nextafter(h, np.float16(-np.inf)), h).astype(np.float16)
+
+
+def fp16_round_up(x32: np.ndarray) -> np.ndarray:
+    """Smallest fp16 value >= x (x float32)."""
+    x32 = np.asarray(x32, dtype=np.float32)
+    with np.errstate(over="ignore"):
+        h = x32.astype(np.float16)
+    too_small = h.astype(np.float32) < x32
+    return np.where(too_small, np.nextafter(h, np.float16(np.inf)), h).astype(np.float16)
+
+
+# ----------------------------------------------------------------------------
+# Router: Eq. 1, Eq. 2, routing freezing, routing sharing
+# ----------------------------------------------------------------------------
+def router_logits(x64: np.ndarray, W1: np.ndarray, W2=None, W3=None, bias=None) -> np.ndarray:
+    """Eq. 1 per token, float64.
+
+    x64 [n, D]; W1, W2 [D, M]; W3 [M, M]; bias [M] (all float64).
+    Gated form (W2 and W3 given):  P = f((x W1) * (x W2)) W3 + bias with
+    f = SiLU applied AFTER the element-wise product, as Eq. 1 is written.
+    Linear form (W2 = W3 = None):  P = x W1 + bias.
+    No softmax: argmax over probabilities equals argmax over logits.
+    """
+    u = x64 @ W1
+    if W2 is None:
+        if W3 is not None:
+            raise ValueError("W3 without W2")
+        P = u
+    else:
+        a = u * (x64 @ W2)
+        h = a / (1.0 + np.exp(-a))          # SiLU(a) = a * sigmoid(a)
+        P = h @ W3
+    if bias is not None:
+        P = P + np.asarray(bias, dtype=np.float64)
+    return P
+
+
+def token_experts(P: np.ndarray) -> np.ndarray:
+    """Per-token top-1 (Section 3.2): first index of the row maximum."""
+    return np.argmax(P, axis=1).astype(np.int64)    # numpy argmax = first occurrence
+
+
+def chunk_vote(e: np.ndarray, n_experts: int = N_EXPERTS):
+    """Eq. 2 for one chunk: histogram of token choices, winner = first maximum."""
+    votes = np.zeros(n_experts, dtype=np.int32)
+    for k in e:
+        votes[int(k)] += 1
+    return votes, int(np.argmax(votes))
+
+
+def route(hidden_u16: np.ndarray, dtype: int, chunk: int, W1_u16, W2_u16=None, W3=None,
+          bias=None, rf_first_chunk: bool = True):
+    """Bit-width map of one routing-sharing group.
+
+    hidden_u16 [B, T, D_in]; W1_u16/W2_u16 [D_in, M] in the same 16-bit dtype;
+    W3 [M, M] and bias [M] float32.
+    Returns dict(map uint8 [B, C], votes int32 [B, C, M], token_expert [B, C*N],
+    margin float64 [B, C*N] (top-1 minus top-2 logit), pmax float64 [B, C*N]).
+    C = T // chunk; the T mod chunk trailing tokens are never routed (they stay
+    in the 16-bit tail, Section 3.2).  With routing freezing the first chunk
+    is fixed to the 16-bit expert without consulting the router (Section 3.4);
+    its votes row is all zero.
+    """
+    B, T, D = hidden_u16.shape
+    C = T // chunk
+    W1 = to_f64(W1_u16, dtype)
+    W2 = None if W2_u16 is None else to_f64(W2_u16, dtype)
+    W3_ = None if W3 is None else np.asarray(W3, dtype=np.float32).astype(np.float64)
+    b_ = None if bias is None else np.asarray(bias, dtype=np.float32).astype(np.float64)
+    M = W1.shape[1]
+    bmap = np.zeros((B, C), dtype=np.uint8)
+    votes = np.zeros((B, C, M), dtype=np.int32)
+    tok = np.full((B, C * chunk), -1, dtype=np.int64)
+    margin = np.full((B, C * chunk), np.inf)
+    pmax = np.zeros((B, C * chunk))
+    for b in range(B):
+        for c in range(C):
+            if c == 0 and rf_first_chunk:
+                bmap[b, c] = M - 1          # the 16-bit expert is the last one
+                continue
+            x = to_f64(hidden_u16[b, c * chunk:(c + 1) * chunk], dtype)
+            P = router_logits(x, W1, W2, W3_, b_)
+            e = token_experts(P)
+            v, r = chunk_vote(e, M)
+            bmap[b, c] = r
+            votes[b, c] = v
+            tok[b, c * chunk:(c + 1) * chunk] = e
+            srt = np.sort(P, axis=1)
+            margin[b, c * chunk:(c + 1) * chunk] = srt[:, -1] - srt[:, -2]
+            pmax[b, c * chunk:(c + 1) * chunk] = np.max(np.abs(P), axis=1)
+    return dict(map=bmap, votes=votes, token_expert=tok, margin=margin, pmax=pmax)
+
+
+def reachable_winners(votes_row: np.ndarray, fragile_tokens_experts, fragile_alt):
+    """Winners a chunk can reach when each fragile token may flip to its runner-up.
+
+    votes_row [M]; fragile_tokens_experts / fragile_alt: lists of the current and
+    the runner-up expert of each fragile token.  Exhaustive for few tokens,
+    otherwise a conservative superset (any expert whose best-case count can reach
+    the best-case-for-others maximum).
+    """
+    M = len(votes_row)
+    nf = len(fragile_tokens_experts)
+    winners = set()
+    if nf <= 12:
+        for mask in range(1 << nf):
+            v = votes_row.astype(np.int64).copy()
+            for i in range(nf):
+                if mask >> i & 1:
+                    v[fragile_tokens_experts[i]] -= 1
+                    v[fragile_alt[i]] += 1
+            winners.add(int(np.argmax(v)))
+        return winners
+    gain = np.zeros(M, dtype=np.int64)
+    loss = np.zeros(M, dtype=np.int64)
+    for cur, alt in zip(fragile_tokens_experts, fragile_alt):
+        loss[cur] += 1
+        gain[alt] += 1
+    for k in range(M):
+        best_k = votes_row[k] + gain[k]
+        others = [votes_row[j] - loss[j] for j in range(M) if j != k]
+        if best_k >= max(others):
+            winners.add(k)
+    return winners
+
+
+def layer_group(layer: int, rs_group: int) -> int:
+    """Routing sharing (Section 3.4): blocks are partitioned into runs of
+    rs_group consecutive blocks; every block of a run uses the map of the run's
+    first block.  A short last run is allowed."""
+    return layer // rs_group
+
+
+def n_groups(n_layers: int, rs_group: int) -> int:
+    return (n_layers + rs_group - 1) // rs_group
+
+
+def assign_slots(bmap: np.ndarray, n_experts: int = N_EXPERTS):
+    """Chunk index table: slot of chunk c = number of earlier chunks of the same
+    sequence with the same width.  bmap [B, C] -> slot int32 [B, C], count [B, M]."""
+    B, C = bmap.shape
+    slot = np.zeros((B, C), dtype=np.int32)
+    count = np.zeros((B, n_experts), dtype=np.int32)
+    for b in range(B):
+        for c in range(C):
+            w = int(bmap[b, c])
+            slot[b, c] = count[b, w]
+            count[b, w] += 1
+    return slot, count
+
+
+# ----------------------------------------------------------------------------
+# Quantiser (group-wise asymmetric min-max, group 32)
+# ----------------------------------------------------------------------------
+def quantize_groups(x32: np.ndarray, bits: int):
+    """Quantise along the LAST axis, which must have length 32 (one group).
+
+    Canonical sequence, every step one IEEE binary32 operation (round to
+    nearest even) unless a direction is stated:
+        mn, mx   exact minimum / maximum of the group
+        z  = largest fp16 <= mn                      (stored zero)
+        r  = mx - float(z)
+        s  = smallest fp16 >= r / (2^bits - 1)       (stored scale)
+        if s == 0: every code is 0
+        inv = 1 / float(s)
+        code = min(2^bits - 1, max(0, rint((x - float(z)) * inv)))
+    rint rounds halves to even.  Returns (scale fp16, zero fp16, codes uint8).
+    Dequantised value (defined, not computed here): code * s + z.
+    """
+    x32 = np.asarray(x32, dtype=np.float32)
+    assert x32.shape[-1] == GROUP
+    qmax = np.float32((1 << bits) - 1)
+    mn = x32.min(axis=-1)
+    mx = x32.max(axis=-1)
+    z = fp16_round_down(mn)
+    zf = z.astype(np.float32)
+    r = (mx - zf).astype(np.float32)
+    s = fp16_round_up((r / qmax).astype(np.float32))
+    sf = s.astype(np.float32)
+    with np.errstate(divide="ignore", invalid="ignore", over="ignore"):
+        inv = (np.float32(1.0) / sf).astype(np.float32)
+        d = (x32 - zf[..., None]).astype(np.float32)
+        t = (d * inv[..., None]).astype(np.float32)
+        c = np.rint(t)
+    c = np.minimum(qmax, np.maximum(np.float32(0), c))
+    c = np.where((sf == 0)[..., None], np.float32(0), c)
+    return s, z, c.astype(np.uint8)
+
+
+def quantize_tile(K32: np.ndarray, V32: np.ndarray, bits: int):
+    """One tile: K32, V32 float32 [32 tokens, 128 channels].
+
+    Keys: one group per channel over the tile's 32 tokens (per-channel inside
+    the chunk).  Values: one group per token over 32 consecutive channels.
+    Returns dict with k_scale/k_zero fp16 [128], k_codes uint8 [32,128],
+    v_scale/v_zero fp16 [4, 32] ([channel group, token]), v_codes uint8 [32,128].
+    """
+    assert K32.shape == (TILE_TOKENS, HEAD_DIM) and V32.shape == (TILE_TOKENS, HEAD_DIM)
+    ks, kz, kc = quantize_groups(K32.T, bits)                   # [128, 32] groups over tokens
+    vg = V32.reshape(TILE_TOKENS, HEAD_DIM // GROUP, GROUP)     # [32, 4, 32]
+    vs, vz, vc = quantize_groups(vg, bits)                      # vs [32, 4]
+    return dict(k_scale=ks, k_zero=kz, k_codes=np.ascontiguousarray(kc.T),
+                v_scale=np.ascontiguousarray(vs.T), v_zero=np.ascontiguousarray(vz.T),
+                v_codes=vc.reshape(TILE_TOKENS, HEAD_DIM))
+
+
+def dequantize_tile(t: dict):
+    """float64 K̂, V̂ [32, 128] of a quantised tile: code * scale + zero."""
+    Kh = t["k_codes"].astype(np.float64) * t["k_scale"].astype(np.float64)[None, :] \
+        + t["k_zero"].astype(np.float64)[None, :]
+    vs = np.repeat(t["v_scale"].astype(np.float64).T, GROUP, axis=1)   # [32 tok, 128]
+    vz = np.repeat(t["v_zero"].astype(np.float64).T, GROUP, axis=1)
+    Vh = t["v_codes"].astype(np.float64) * vs + vz
+    return Kh, Vh
+
+
+# ----------------------------------------------------------------------------
+# Storage format
+# ----------------------------------------------------------------------------
+def tile_bytes(bits: int) -> int:
+    """Bytes of one 32-token tile of one kv head (K and V together)."""
+    return 16384 if bits == 16 else META_BYTES + 2 * TILE_TOKENS * 16 * bits
+
+
+def slot_bytes(bits: int, chunk: int) -> int:
+    return (chunk // TILE_TOKENS) * tile_bytes(bits)
+
+
+def v_channel_of_position(p: int) -> int:
+    """Value rows store channels interleaved by channel group: position
+    p = 16*u + 4*cg + k holds channel 32*cg + 4*u + k."""
+    u, cg, k = p >> 4, (p >> 2) & 3, p & 3
+    return 32 * cg + 4 * u + k
+
+
+def code_location(p: int, t: int, bits: int):
+    """(byte offset inside the payload row, bit offset inside the little-endian
+    32-bit word) of position p of token row t, bits in {2, 4, 8}.
+
+    A word holds n = 32/bits consecutive positions; position i of a word sits at
+    bit  bits*(i >> 1) + 16*(i & 1)  (even positions fill the low half-word, odd
+    positions the high half-word).  Words are grouped in 16-byte units; rows of
+    128 bytes or more store unit U at  U xor (t mod 8).
+    """
+    n = 32 // bits
+    j, i = divmod(p, n)
+    bit = bits * (i >> 1) + 16 * (i & 1)
+    unit, w_in_unit = j >> 2, j & 3
+    if 16 * bits >= 128:
+        unit ^= (t & 7)
+    return unit * 16 + w_in_unit * 4, bit
+
+
+def raw_location(c: int, t: int) -> int:
+    """Byte offset of channel c in a 256-byte raw (16-bit) row of token row t:
+    16-byte unit U = c // 8 stored at (U & 8) | ((U xor t) & 7)."""
+    U = c >> 3
+    Up = (U & 8) | ((U ^ t) & 7)
+    return Up * 16 + (c & 7) * 2
+
+
+_TABLES = {}
+
+
+def _tables(bits: int):
+    """Index tables built from `code_location`, cached (pure bookkeeping)."""
+    if bits in _TABLES:
+        return _TABLES[bits]
+    row_words = 4 * bits
+    word = np.zeros((TILE_TOKENS, HEAD_DIM), dtype=np.int64)
+    shift = np.zeros((TILE_TOKENS, HEAD_DIM), dtype=np.uint32)
+    for t in range(TILE_TOKENS):
+        for p in range(HEAD_DIM):
+            byte, bit = code_location(p, t, bits)
+            word[t, p] = t * row_words + byte // 4
+            shift[t, p] = bit
+    vperm = np.array([v_channel_of_position(p) for p in range(HEAD_DIM)], dtype=np.int64)
+    _TABLES[bits] = (word, shift, vperm)
+    return _TABLES[bits]
+
+
+def _raw_table():
+    if "raw" not in _TABLES:
+        off = np.zeros((TILE_TOKENS, HEAD_DIM), dtype=np.int64)
+        for t in range(TILE_TOKENS):
+            for c in range(HEAD_DIM):
+                off[t, c] = (t * 256 + raw_location(c, t)) // 2
+        _TABLES["raw"] = off
+    return _TABLES["raw"]
+
+
+def _pack_payload(codes_by_position: np.ndarray, bits: int) -> np.ndarray:
+    word, shift, _ = _tables(bits)
+    out = np.zeros(TILE_TOKENS * 4 * bits, dtype=np.uint32)
+    np.bitwise_or.at(out, word.ravel(),
+                     (codes_by_position.astype(np.uint32) << shift).ravel())
+    return out.view(np.uint8)
+
+
+def _unpack_payload(payload_u8: np.ndarray, bits: int) -> np.ndarray:
+    word, shift, _ = _tables(bits)
+    w = np.ascontiguousarray(payload_u8).view(np.uint32)
+    return ((w[word] >> shift) & np.uint32((1 << bits) - 1)).astype(np.uint8)
+
+
+def pack_tile(t: dict, bits: int) -> np.ndarray:
+    """Quantised tile -> bytes.  Layout: K scale fp16[128] | K zero fp16[128] |
+    V scale fp16[4][32] | V zero fp16[4][32] | K payload (32 rows) | V payload."""
+    _, _, vperm = _tables(bits)
+    out = np.zeros(tile_bytes(bits), dtype=np.uint8)
+    out[0:256] = t["k_scale"].astype(np.float16).view(np.uint8)
+    out[256:512] = t["k_zero"].astype(np.float16).view(np.uint8)
+    out[512:768] = np.ascontiguousarray(t["v_scale"], dtype=np.float16).view(np.uint8).ravel()
+    out[768:1024] = np.ascontiguousarray(t["v_zero"], dtype=np.float16).view(np.uint8).ravel()
+    pb = TILE_TOKENS * 16 * bits
+    out[1024:1024 + pb] = _pack_payload(t["k_codes"], bits)
+    out[1024 + pb:1024 + 2 * pb] = _pack_payload(t["v_codes"][:, vperm], bits)
+    return out
+
+
+def unpack_tile(buf: np.ndarray, bits: int) -> dict:
+    _, _, vperm = _tables(bits)
+    buf = np.ascontiguousarray(buf, dtype=np.uint8)
+    pb = TILE_TOKENS * 16 * bits
+    vcp = _unpack_payload(buf[1024 + pb:1024 + 2 * pb], bits)
+    vc = np.zeros_like(vcp)
+    vc[:, vperm] = vcp
+    return dict(k_scale=buf[0:256].view(np.float16).copy(),
+                k_zero=buf[256:512].view(np.float16).copy(),
+                v_scale=buf[512:768].view(np.float16).reshape(4, 32).copy(),
+                v_zero=buf[768:1024].view(np.float16).reshape(4, 32).copy(),
+                k_codes=_unpack_payload(buf[1024:1024 + pb], bits), v_codes=vc)
+
+
+def pack_raw_tile(K_u16: np.ndarray, V_u16: np.ndarray) -> np.ndarray:
+    """16-bit tile: K rows then V rows, input bit patterns, swizzled units."""
+    off = _raw_table()
+    out = np.zeros(16384 // 2, dtype=np.uint16)
+    out[off.ravel()] = K_u16.ravel()
+    out[4096 + off.ravel()] = V_u16.ravel()
+    return out.view(np.uint8)
+
+
+def unpack_raw_tile(buf: np.ndarray):
+    off = _raw_table()
+    w = np.ascontiguousarray(buf, dtype=np.uint8).view(np.uint16)
+    return w[off], w[4096 + off]
+
+
+# ----------------------------------------------------------------------------
+# Cache construction (prefill): quantise + pack into per-width pools
+# ----------------------------------------------------------------------------
+def quantize_kv(K_u16: np.ndarray, V_u16: np.ndarray, dtype: int, chunk: int,
+                bmap: np.ndarray, capacity=None):
+    """K_u16, V_u16 [B, T, H_kv, 128]; bmap uint8 [B, C] (expert index per chunk).
+
+    Returns dict(pools=[4 x uint8 [B, H_kv, capacity_w, slot_bytes_w]],
+    slot [B, C], count [B, 4], tail_k/tail_v uint16 [B, H_kv, r, 128], tail_len r).
+    Chunk c of sequence b goes to pool[w] slot slot[b, c] for every kv head;
+    trailing T mod chunk tokens are kept as raw 16-bit rows (Section 3.2).
+    """
+    B, T, H, d = K_u16.shape
+    assert d == HEAD_DIM and chunk % TILE_TOKENS == 0
+    C = T // chunk
+    assert bmap.shape == (B, C)
+    slot, count = assign_slots(bmap)
+    if capacity is None:
+        capacity = [max(1, int(count[:, w].max())) for w in range(N_EXPERTS)]
+    pools = [np.zeros((B, H, capacity[w], slot_bytes(EXPERT_BITS[w], chunk)), dtype=np.uint8)
+             for w in range(N_EXPERTS)]
+    tpc = chunk // TILE_TOKENS
+    for b in range(B):
+        for c in range(C):
+            w = int(bmap[b, c])
+            bits = EXPERT_BITS[w]
+            tb = tile_bytes(bits)
+            for h in range(H):
+                for j in range(tpc):
+                    t0 = c * chunk + j * TILE_TOKENS
+                    Kt = K_u16[b, t0:t0 + TILE_TOKENS, h]
+                    Vt = V_u16[b, t0:t0 + TILE_TOKENS, h]
+                    if bits == 16:
+                        blob = pack_raw_tile(Kt, Vt)
+                    else:
+                        blob = pack_tile(quantize_tile(to_f32(Kt, dtype), to_f32(Vt, dtype), bits), bits)
+                    pools[w][b, h, slot[b, c], j * tb:(j + 1) * tb] = blob
+    r = T - C * chunk
+    tail_k = np.ascontiguousarray(np.transpose(K_u16[:, C * chunk:], (0, 2, 1, 3)))
+    tail_v = np.ascontiguousarray(np.transpose(V_u16[:, C * chunk:], (0, 2, 1, 3)))
+    return dict(pools=pools, slot=slot, count=count, capacity=list(capacity),
+                tail_k=tail_k, tail_v=tail_v, tail_len=r)
+
+
+def uniform_quantize_reference(X_u16: np.ndarray, dtype: int, bits: int, per_channel: bool, chunk: int):
+    """Stand-alone uniform quantiser over a whole [T, 128] tensor, chunk by chunk,
+    used to pin "all chunks routed to one width == uniform quantisation".
+    Returns the dequantised float64 tensor for the T//chunk*chunk leading tokens."""
+    X = to_f32(X_u16, dtype)
+    T = (X.shape[0] // chunk) * chunk
+    out = np.zeros((T, HEAD_DIM))
+    for t0 in range(0, T, GROUP):
+        blk = X[t0:t0 + GROUP]
+        if per_channel:
+            s, z, c = quantize_groups(blk.T, bits)
+            out[t0:t0 + GROUP] = (c.astype(np.float64) * s.astype(np.float64)[:, None]
+                                  + z.astype(np.float64)[:, None]).T
+        else:
+            g = blk.reshape(GROUP, HEAD_DIM // GROUP, GROUP)
+            s, z, c = quantize_groups(g, bits)
+            out[t0:t0 + GROUP] = (c.astype(np.float64) * s.astype(np.float64)[..., None]
+                                  + z.astype(np.float64)[..., None]).reshape(GROUP, HEAD_DIM)
+    return out
+
+
+# ----------------------------------------------------------------------------
+# Decode attention over the mixed-precision cache
+# ----------------------------------------------------------------------------
+def cache_kv_rows(cache: dict, dtype: int, chunk: int, b: int, h: int):
+    """All cached rows of (sequence b, kv head h) as float64 K̂, V̂ [n, 128],
+    pool by pool then the tail (softmax attention does not depend on key order)."""
+    Ks, Vs = [], []
+    tpc = chunk // TILE_TOKENS
+    for w in range(N_EXPERTS):
+        bits = EXPERT_BITS[w]
+        tb = tile_bytes(bits)
+        for s in range(int(cache["count"][b, w])):
+            blob = cache["pools"][w][b, h, s]
+            for j in range(tpc):
+                tile = blob[j * tb:(j + 1) * tb]
+                if bits == 16:
+                    Ku, Vu = unpack_raw_tile(tile)
+                    Ks.append(to_f64(Ku, dtype))
+                    Vs.append(to_f64(Vu, dtype))
+                else:
+                    Kh, Vh = dequantize_tile(unpack_tile(tile, bits))
+                    Ks.append(Kh)
+                    Vs.append(Vh)
+    if cache["tail_len"] > 0:
+        Ks.append(to_f64(cache["tail_k"][b, h, :cache["tail_len"]], dtype))
+        Vs.append(to_f64(cache["tail_v"][b, h, :cache["tail_len"]], dtype))
+    if not Ks:
+        return np.zeros((0, HEAD_DIM)), np.zeros((0, HEAD_DIM))
+    return np.concatenate(Ks, axis=0), np.concatenate(Vs, axis=0)
+
+
+def softmax_attention(q64: np.ndarray, K64: np.ndarray, V64: np.ndarray, scale: float) -> np.ndarray:
+    """out = softmax(scale * K q) V for one query (no mask: a decode query sees
+    every cached token).  An empty cache gives zeros."""
+    if K64.shape[0] == 0:
+        return np.zeros(V64.shape[1])
+    s = (K64 @ q64) * scale
+    p = np.exp(s - s.max())
+    return (p @ V64) / p.sum()
+
+
+def decode_attn(q_u16: np.ndarray, dtype: int, cache: dict, chunk: int, scale=None) -> np.ndarray:
+    """q_u16 [B, H_q, 128] -> float64 out [B, H_q, 128].  Query head h reads kv
+    head h // (H_q / H_kv).  Keys are dequantised, then scores, softmax and the
+    weighted sum are taken in float64 (Limitations section: dequantise before
+    the product with the query)."""
+    B, Hq, d = q_u16.shape
+    Hkv = cache["pools"][0].shape[1]
+    G = Hq // Hkv
+    if scale is None:
+        scale = 1.0 / np.sqrt(d)
+    q = to_f64(q_u16, dtype)
+    out = np.zeros((B, Hq, d))
+    for b in range(B):
+        for h in range(Hkv):
+            K64, V64 = cache_kv_rows(cache, dtype, chunk, b, h)
+            for g in range(G):
+                out[b, h * G + g] = softmax_attention(q[b, h * G + g], K64, V64, scale)
+    return out
+
+
+def cache_bytes(count: np.ndarray, chunk: int, n_kv_heads: int, tail_len: int) -> int:
+    """Closed form of the bytes a cache holds: sum_w count_w * slot_bytes_w per head,
+    plus 512 bytes per tail token per head."""
+    total = 0
+    for b in range(count.shape[0]):
+        for w in range(N_EXPERTS):
+            total += int(count[b, w]) * slot_bytes(EXPERT_BITS[w], chunk) * n_kv_heads
+        total += tail_len * n_kv_heads * 2 * HEAD_DIM * 2
+    return total
