@@ -1,0 +1,206 @@
+/*
+ * moqae.h - C ABI of the B200 (sm_100a) MoQAE inference hot path.
+ *
+ * The library implements, as CUDA kernels, the three inference-time steps of MoQAE
+ * (Section 3.1 of the paper: input chunks -> per-block quantisation strategy -> quantised
+ * KV -> attention):
+ *   moqae_route        chunk-wise router, Section 3.2 Eq. 1 and Eq. 2, with routing freezing
+ *                      and routing sharing of Section 3.4
+ *   moqae_quantize_kv  quantise + bit-pack each chunk at its routed width into per-width pools
+ *   moqae_decode_attn  decode attention over the mixed-precision cache, dequantising inside
+ *                      the kernel (Limitations section: keys are dequantised before the
+ *                      product with the query)
+ *
+ * General rules
+ *   - Every function returns an int: MOQAE_OK (0) or a negative MOQAE_ERR_* code.  Argument
+ *     errors are found on the host before anything is launched.
+ *   - Unless a parameter says "host", every pointer is a DEVICE pointer owned by the caller.
+ *     The library allocates no device memory and keeps no per-call state; work is enqueued on
+ *     the caller's stream (a cudaStream_t passed as void*) and the call returns without
+ *     synchronising.  Calls on the same cache must be ordered by the caller (same stream or
+ *     events).
+ *   - Device pointers must be 16-byte aligned.
+ *   - No C++ types or exceptions cross this boundary.
+ *
+ * Fixed by this build: head_dim = 128, quantisation group = 32, experts = 4 with bit widths
+ * {2, 4, 8, 16} at expert indices {0, 1, 2, 3}, chunk a multiple of 32, 16 <= d_in and
+ * d_in a multiple of 32, n_q_heads / n_kv_heads in {1, .., 8}.
+ *
+ * Storage format of the cache (what moqae_quantize_kv writes and moqae_decode_attn reads)
+ *   tile   = 32 consecutive tokens of one chunk and one kv head.
+ *   quantised tile, b in {2, 4, 8} bits, 1024 + 1024*b bytes:
+ *       [   0,  256)  key scale   fp16[128]      (one per channel, over the tile's 32 tokens)
+ *       [ 256,  512)  key zero    fp16[128]
+ *       [ 512,  768)  value scale fp16[4][32]    ([channel group of 32][token])
+ *       [ 768, 1024)  value zero  fp16[4][32]
+ *       [1024, 1024+512b)         key payload,   32 token rows of 16*b bytes
+ *       [1024+512b, 1024+1024b)   value payload, 32 token rows of 16*b bytes
+ *     A payload row holds 128 positions of b bits.  Key rows: position p = channel p.  Value
+ *     rows: position p = 16*u + 4*cg + k holds channel 32*cg + 4*u + k.  A little-endian 32-bit
+ *     word holds n = 32/b consecutive positions; position i of a word sits at bit
+ *     b*(i>>1) + 16*(i&1).  Words form 16-byte units; rows of >= 128 bytes (b = 8) store unit
+ *     U of token row t at U xor (t mod 8).
+ *     Dequantised value = code * scale + zero.
+ *   16-bit tile, 16384 bytes: 32 key rows then 32 value rows of 256 bytes in the input dtype;
+ *     16-byte unit U of row t is stored at (U & 8) | ((U xor t) & 7).
+ *   slot   = the chunk/32 tiles of one chunk and one kv head, in token order.
+ *   pool[w] = [n_layers][batch][n_kv_heads][capacity[w]] slots of width w.
+ *   map/slot/count/votes tables are per routing-sharing group: [n_groups][batch][max_chunks]
+ *     (count: [n_groups][batch][4], votes: [n_groups][batch][max_chunks][4]),
+ *     n_groups = ceil(n_layers / rs_group), max_chunks = max_tokens / chunk.
+ *   tail_k / tail_v = [n_layers][batch][n_kv_heads][tail_capacity][128] rows in the input
+ *     dtype (tokens that do not fill a chunk stay 16-bit, Section 3.2); tail_len =
+ *     int32 [n_layers][batch].
+ */
+#ifndef MOQAE_H
+#define MOQAE_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define MOQAE_OK 0
+#define MOQAE_ERR_INVALID_ARG (-1)
+#define MOQAE_ERR_UNSUPPORTED (-2)
+#define MOQAE_ERR_MISALIGNED (-3)
+#define MOQAE_ERR_POOL_FULL (-4)
+#define MOQAE_ERR_WORKSPACE_TOO_SMALL (-5)
+#define MOQAE_ERR_CUDA (-6)
+#define MOQAE_ERR_TIMEOUT (-7)
+
+#define MOQAE_DTYPE_FP16 0
+#define MOQAE_DTYPE_BF16 1
+
+#define MOQAE_N_EXPERTS 4
+#define MOQAE_N_CACHE_BUFFERS 12
+
+/* Problem description shared by every call (plain data, passed by pointer, host memory). */
+typedef struct moqae_config {
+  int32_t n_layers;
+  int32_t n_q_heads;
+  int32_t n_kv_heads;
+  int32_t head_dim;        /* 128 */
+  int32_t chunk;           /* tokens per chunk, multiple of 32 */
+  int32_t group;           /* 32 */
+  int32_t dtype;           /* MOQAE_DTYPE_* of hidden states, K, V, q, W1, W2 */
+  int32_t n_experts;       /* 4 */
+  int32_t expert_bits[4];  /* {2, 4, 8, 16} */
+  int32_t rs_group;        /* routing sharing: consecutive layers per group (>= 1) */
+  int32_t rf_first_chunk;  /* routing freezing: 1 = chunk 0 is fixed to the 16-bit expert */
+  int32_t d_in;            /* router input width */
+  int32_t max_tokens;      /* largest context the tables are sized for */
+  int32_t tail_capacity;   /* rows per (layer, batch, kv head) in the 16-bit tail */
+  int32_t batch;
+} moqae_config;
+
+/* View of a cache: device pointers supplied by the caller (see moqae_cache_bytes for sizes). */
+typedef struct moqae_cache {
+  void* pool[4];
+  int64_t capacity[4];     /* slots per (layer, batch, kv head) in pool[w] */
+  uint8_t* map;            /* expert index per chunk */
+  int32_t* slot;           /* slot of each chunk inside its width's pool */
+  int32_t* count;          /* chunks per width */
+  int32_t* votes;          /* Eq. 2 histograms */
+  void* tail_k;
+  void* tail_v;
+  int32_t* tail_len;
+  int32_t* status;         /* int32[4]: sticky device-side error code and two detail words */
+} moqae_cache;
+
+/* Library version, major*10000 + minor*100 + patch. */
+int moqae_version(void);
+
+/* Last CUDA runtime error code seen by a call that returned MOQAE_ERR_CUDA (0 if none). */
+int moqae_last_cuda_error(void);
+
+/* Static string for an error code (host pointer, never NULL). */
+const char* moqae_error_string(int code);
+
+/*
+ * Sizes in bytes of the twelve cache buffers for `cfg` and per-width capacities (host
+ * arrays): out_bytes[0..3] pools, [4] map, [5] slot, [6] count, [7] votes, [8] tail_k,
+ * [9] tail_v, [10] tail_len, [11] status.  Pure host arithmetic.
+ */
+int moqae_cache_bytes(const moqae_config* cfg, const int64_t capacity[4],
+                      int64_t out_bytes[MOQAE_N_CACHE_BUFFERS]);
+
+/*
+ * Fill `out` from twelve device pointers in the order of moqae_cache_bytes; checks
+ * alignment.  Allocates nothing.  The caller must have zeroed count, tail_len and status.
+ */
+int moqae_cache_bind(const moqae_config* cfg, const int64_t capacity[4],
+                     void* const buffers[MOQAE_N_CACHE_BUFFERS], moqae_cache* out);
+
+/*
+ * Router of one routing-sharing group (Section 3.2, Eq. 1 and Eq. 2; Section 3.4).
+ *   hidden  [batch][T][d_in] input-dtype rows of the group's FIRST layer.
+ *   W1, W2  [d_in][4] input dtype; W3 [4][4] float32 row-major; bias [4] float32.
+ *           W2 = W3 = NULL selects the linear router P = C W1 + bias; all non-NULL selects
+ *           Eq. 1, P = SiLU((C W1) * (C W2)) W3 + bias.  bias may be NULL (zero).
+ *   Each token takes its arg-max expert, each chunk the expert most tokens chose (ties: the
+ *   lower index, i.e. the narrower width).  With cfg->rf_first_chunk chunk 0 is not routed and
+ *   is the 16-bit expert.  The T mod chunk trailing tokens are not routed.
+ *   Writes map, slot, count and votes of group `layer_group`; if votes_out is not NULL it
+ *   also receives the group's [batch][T/chunk][4] int32 histograms (compact).
+ *   Products are exact, sums are float32 in an unspecified order.
+ */
+int moqae_route(const moqae_config* cfg, const void* hidden, int32_t T, const void* W1,
+                const void* W2, const float* W3, const float* bias, int32_t layer_group,
+                const moqae_cache* cache, int32_t* votes_out, void* stream);
+
+/*
+ * Quantise and pack the keys and values of one layer (prefill).
+ *   K, V [batch][T][n_kv_heads][128] input dtype.
+ *   forced_map: NULL = use the map routed for the layer's group; otherwise uint8
+ *   [batch][T/chunk] expert indices that REPLACE the group's map (slot and count are
+ *   recomputed) before quantising.
+ *   Chunk c of sequence b goes to pool[map] slot `slot[b][c]` of every kv head; trailing
+ *   T mod chunk tokens are copied to the tail and tail_len[layer][b] is set.
+ *   A chunk whose slot index is >= capacity is skipped and status[0] becomes
+ *   MOQAE_ERR_POOL_FULL (read it with moqae_poll_status).
+ *   Quantiser: group-wise asymmetric min-max, group 32 (keys per channel over the tile's
+ *   tokens, values per token over 32 channels); zero = largest fp16 <= min,
+ *   scale = smallest fp16 >= (max - zero)/(2^b - 1), code = clamp(rint((x - zero) * (1/scale)))
+ *   with every operation a single binary32 operation; inputs must be finite with
+ *   |x| < 32752.
+ */
+int moqae_quantize_kv(const moqae_config* cfg, const void* K, const void* V, int32_t T,
+                      int32_t layer, const uint8_t* forced_map, const moqae_cache* cache,
+                      void* stream);
+
+/*
+ * Append one decoded token per sequence to the 16-bit tail of `layer` (tokens that do not
+ * fill a chunk stay 16-bit, Section 3.2).  k_new, v_new [batch][n_kv_heads][128].  A full
+ * tail sets status[0] = MOQAE_ERR_POOL_FULL and drops the token.
+ */
+int moqae_append_kv(const moqae_config* cfg, const void* k_new, const void* v_new,
+                    int32_t layer, const moqae_cache* cache, void* stream);
+
+/* Bytes of scratch moqae_decode_attn needs for `cfg` on the current device (host out). */
+int moqae_decode_attn_workspace(const moqae_config* cfg, int64_t* out_bytes);
+
+/*
+ * One decode step of attention for one layer: for every query head h,
+ *   out[b][h] = softmax(scale * K̂ q[b][h]) V̂   over all cached tokens of kv head
+ *   h / (n_q_heads / n_kv_heads), K̂ and V̂ being the dequantised cache rows plus the tail.
+ *   q [batch][n_q_heads][128] input dtype; out [batch][n_q_heads][128] float32;
+ *   scale <= 0 selects 1/sqrt(128).  An empty cache gives zeros.
+ *   workspace: at least moqae_decode_attn_workspace bytes, 16-byte aligned; contents are
+ *   scratch (split partials), overwritten by every call.
+ */
+int moqae_decode_attn(const moqae_config* cfg, const void* q, int32_t layer,
+                      const moqae_cache* cache, float* out, float scale, void* workspace,
+                      int64_t workspace_bytes, void* stream);
+
+/*
+ * Synchronous read of the cache's device status word: *out_status (host) receives MOQAE_OK
+ * or the first device-side error recorded since the buffer was zeroed.  Waits for `stream`.
+ */
+int moqae_poll_status(const moqae_cache* cache, void* stream, int32_t* out_status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOQAE_H */

@@ -1,0 +1,81 @@
+// Shared declarations of the MoQAE CUDA library (sm_100a).
+#pragma once
+
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "moqae.h"
+
+namespace moqae {
+
+constexpr int kHeadDim = 128;
+constexpr int kGroup = 32;
+constexpr int kTileTokens = 32;
+constexpr int kMetaBytes = 1024;
+constexpr int kRawTileBytes = 16384;
+constexpr int kMaxQueryGroup = 8;
+constexpr int kMaxSplits = 64;
+
+__host__ __device__ constexpr int bits_of_expert(int w) { return 2 << w; }   // 2,4,8,16
+__host__ __device__ constexpr int tile_bytes_of_expert(int w) {
+  return w == 3 ? kRawTileBytes : kMetaBytes + 1024 * (2 << w);
+}
+// Cost of one tile in KiB (3, 5, 9, 16): the unit in which decode work is balanced.
+__host__ __device__ constexpr int tile_cost_of_expert(int w) { return tile_bytes_of_expert(w) >> 10; }
+
+// Everything a kernel needs to find its way around a cache (passed by value).
+struct CacheView {
+  uint8_t* pool[4];
+  long long capacity[4];
+  uint8_t* map;
+  int32_t* slot;
+  int32_t* count;
+  int32_t* votes;
+  uint16_t* tail_k;
+  uint16_t* tail_v;
+  int32_t* tail_len;
+  int32_t* status;
+};
+
+struct Dims {
+  int n_layers, n_q_heads, n_kv_heads, chunk, dtype, rs_group, rf_first_chunk, d_in;
+  int max_chunks, tail_capacity, batch;
+};
+
+__device__ __forceinline__ void set_status(int32_t* status, int code, int d0, int d1) {
+  if (atomicCAS(status, 0, code) == 0) {
+    status[1] = d0;
+    status[2] = d1;
+  }
+}
+
+__device__ __forceinline__ float load16_as_float(uint16_t u, int dtype) {
+  return dtype == MOQAE_DTYPE_FP16 ? __half2float(__ushort_as_half(u))
+                                   : __uint_as_float(static_cast<uint32_t>(u) << 16);
+}
+
+// Address of slot `slot` of (layer, b, h) in pool w.
+__device__ __forceinline__ uint8_t* slot_ptr(const CacheView& cv, const Dims& dm, int w, int layer,
+                                             int b, int h, long long slot) {
+  const long long slot_bytes = static_cast<long long>(dm.chunk / kTileTokens) * tile_bytes_of_expert(w);
+  const long long idx = ((static_cast<long long>(layer) * dm.batch + b) * dm.n_kv_heads + h) *
+                            cv.capacity[w] + slot;
+  return cv.pool[w] + idx * slot_bytes;
+}
+
+// Launchers implemented in the .cu files (host side, return cudaError_t).
+cudaError_t launch_route(const Dims& dm, const CacheView& cv, const void* hidden, int T, const void* W1,
+                         const void* W2, const float* W3, const float* bias, int group,
+                         int32_t* votes_out, cudaStream_t st);
+cudaError_t launch_finalize_map(const Dims& dm, const CacheView& cv, int group, int n_chunks,
+                                const uint8_t* forced_map, cudaStream_t st);
+cudaError_t launch_quantize(const Dims& dm, const CacheView& cv, const void* K, const void* V, int T,
+                            int layer, cudaStream_t st);
+cudaError_t launch_append(const Dims& dm, const CacheView& cv, const void* k_new, const void* v_new,
+                          int layer, cudaStream_t st);
+int decode_num_splits(const Dims& dm);
+cudaError_t launch_decode(const Dims& dm, const CacheView& cv, const void* q, int layer, float* out,
+                          float scale, float* workspace, int n_splits, cudaStream_t st);
+
+}  // namespace moqae

@@ -1,0 +1,112 @@
+"""GPU parity: moqae_decode_attn against the oracle on the same packed cache."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import moqae_oracle as O
+from paper_2506_07533_b200 import binding as mq
+from paper_2506_07533_b200 import synth
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+
+def decode_case(B, T, Hq, Hkv, chunk, dtype, bmap, seed, from_oracle_cache, q_scale=1.0):
+    K, V = H.make_kv(B, T, Hkv, dtype, seed)
+    q = synth.normal((B, Hq, 128), dtype, seed + 1, "cpu", std=q_scale)
+    ocache = O.quantize_kv(synth.to_u16(K), synth.to_u16(V), dtype, chunk, bmap)
+    ref = O.decode_attn(synth.to_u16(q), dtype, ocache, chunk)
+    cfg = mq.make_config(n_layers=2, n_q_heads=Hq, n_kv_heads=Hkv, chunk=chunk, dtype=dtype, d_in=64,
+                         max_tokens=max(T, chunk), batch=B)
+    cap = [max(1, int(ocache["count"][:, w].max())) if bmap.size else 1 for w in range(4)]
+    cache = mq.moqae_cache_bind(cfg, cap, zero_pools=True)
+    layer = 1
+    if from_oracle_cache:
+        H.upload_oracle_cache(cache, ocache, layer)
+    else:
+        fm = torch.from_numpy(bmap).cuda() if bmap.size else None
+        mq.moqae_quantize_kv(cfg, K.cuda(), V.cuda(), T, layer, cache, forced_map=fm)
+    ws = torch.empty(mq.moqae_decode_attn_workspace(cfg), dtype=torch.uint8, device="cuda")
+    out = torch.full((B, Hq, 128), float("nan"), dtype=torch.float32, device="cuda")
+    mq.moqae_decode_attn(cfg, q.cuda(), layer, cache, out, ws)
+    torch.cuda.synchronize()
+    ok, e_abs, e_rel = H.attn_tolerance_ok(out.cpu().numpy(), ref)
+    assert ok, (e_abs, e_rel)
+    return e_abs, e_rel
+
+
+@pytest.mark.parametrize("dtype", [0, 1])
+@pytest.mark.parametrize("from_oracle_cache", [True, False])
+def test_mixed_cache_mha(dtype, from_oracle_cache):
+    B, T, chunk = 2, 32 * 9 + 11, 32
+    rs = np.random.RandomState(3 + dtype)
+    bmap = rs.randint(0, 4, size=(B, T // chunk)).astype(np.uint8)
+    decode_case(B, T, 4, 4, chunk, dtype, bmap, 40 + dtype, from_oracle_cache)
+
+
+@pytest.mark.parametrize("G", [1, 2, 4, 8])
+def test_query_groups(G):
+    B, T, chunk, Hkv = 2, 128 * 6 + 5, 128, 2
+    rs = np.random.RandomState(G)
+    bmap = rs.randint(0, 4, size=(B, T // chunk)).astype(np.uint8)
+    decode_case(B, T, Hkv * G, Hkv, chunk, 1, bmap, 50 + G, True)
+
+
+@pytest.mark.parametrize("w", [0, 1, 2, 3])
+def test_uniform_width_config1_shape(w):
+    # config 1: batch 1, 8 heads, context 4096, chunk 128, fp16
+    bmap = np.full((1, 32), w, np.uint8)
+    decode_case(1, 4096, 8, 8, 128, 0, bmap, 60 + w, False)
+
+
+def test_config1_mixed_with_frozen_first_chunk():
+    bmap = synth.multinomial_map(1, 32, [0.25, 0.25, 0.25, 0.25], seed=9)
+    assert bmap[0, 0] == 3
+    decode_case(1, 4096, 8, 8, 128, 0, bmap, 70, False)
+
+
+def test_edge_cases():
+    decode_case(1, 7, 2, 2, 32, 0, np.zeros((1, 0), np.uint8), 80, False)         # tail only
+    decode_case(2, 32, 2, 1, 32, 1, np.array([[0], [3]], np.uint8), 81, False)    # one chunk, no tail
+    decode_case(1, 33, 1, 1, 32, 0, np.array([[1]], np.uint8), 82, True)          # one chunk + 1 tail token
+    decode_case(1, 512 * 2 + 500, 4, 1, 512, 1, np.array([[2, 0]], np.uint8), 83, False)   # long tail, big chunk
+    decode_case(1, 256, 2, 2, 64, 0, np.array([[0, 0, 0, 0]], np.uint8), 84, False, q_scale=4.0)  # peaky softmax
+
+
+def test_empty_cache_gives_zeros():
+    cfg = mq.make_config(n_layers=1, n_q_heads=2, n_kv_heads=2, chunk=32, dtype=0, d_in=64,
+                         max_tokens=32, batch=1)
+    cache = mq.moqae_cache_bind(cfg, [1, 1, 1, 1])
+    ws = torch.empty(mq.moqae_decode_attn_workspace(cfg), dtype=torch.uint8, device="cuda")
+    out = torch.full((1, 2, 128), float("nan"), dtype=torch.float32, device="cuda")
+    q = synth.normal((1, 2, 128), 0, 1, "cuda")
+    mq.moqae_decode_attn(cfg, q, 0, cache, out, ws)
+    torch.cuda.synchronize()
+    assert (out == 0).all()
+
+
+def test_append_then_decode_matches_oracle_with_longer_tail():
+    # decode loop: new tokens are appended to the 16-bit tail, routing is not re-run
+    B, T, Hq, Hkv, chunk, dtype = 2, 64 * 3, 4, 2, 64, 1
+    bmap = np.array([[3, 0, 1], [3, 2, 0]], np.uint8)
+    K, V = H.make_kv(B, T + 5, Hkv, dtype, 90)
+    cfg = mq.make_config(n_layers=1, n_q_heads=Hq, n_kv_heads=Hkv, chunk=chunk, dtype=dtype, d_in=64,
+                         max_tokens=T + chunk, batch=B)
+    cache = mq.moqae_cache_bind(cfg, [2, 2, 2, 2], zero_pools=True)
+    Kc, Vc = K.cuda(), V.cuda()
+    mq.moqae_quantize_kv(cfg, Kc[:, :T].contiguous(), Vc[:, :T].contiguous(), T, 0, cache,
+                         forced_map=torch.from_numpy(bmap).cuda())
+    ws = torch.empty(mq.moqae_decode_attn_workspace(cfg), dtype=torch.uint8, device="cuda")
+    out = torch.empty((B, Hq, 128), dtype=torch.float32, device="cuda")
+    for step in range(5):
+        mq.moqae_append_kv(cfg, Kc[:, T + step].contiguous(), Vc[:, T + step].contiguous(), 0, cache)
+        q = synth.normal((B, Hq, 128), dtype, 200 + step, "cpu")
+        mq.moqae_decode_attn(cfg, q.cuda(), 0, cache, out, ws)
+        torch.cuda.synchronize()
+        n = T + step + 1
+        ocache = O.quantize_kv(synth.to_u16(K[:, :n]), synth.to_u16(V[:, :n]), dtype, chunk, bmap)
+        assert ocache["tail_len"] == step + 1
+        ref = O.decode_attn(synth.to_u16(q), dtype, ocache, chunk)
+        ok, e_abs, e_rel = H.attn_tolerance_ok(out.cpu().numpy(), ref)
+        assert ok, (step, e_abs, e_rel)
+    assert mq.moqae_poll_status(cache) == 0
