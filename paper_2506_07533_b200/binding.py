@@ -145,7 +145,11 @@ class Cache:
         return self.cfg.max_tokens // self.cfg.chunk
 
     def table(self, idx, dtype, shape):
-        return self.buffers[idx].view(dtype).view(*shape)
+        n = 1
+        for d in shape:
+            n *= d
+        nbytes = n * torch.empty(0, dtype=dtype).element_size()
+        return self.buffers[idx][:nbytes].view(dtype).view(*shape)
 
     @property
     def map(self):
@@ -171,11 +175,13 @@ class Cache:
         """uint8 view [n_layers, batch, n_kv_heads, capacity_w, slot_bytes_w]."""
         tb = 16384 if w == 3 else 1024 + 1024 * EXPERT_BITS[w]
         sb = (self.cfg.chunk // 32) * tb
-        return self.buffers[w].view(self.cfg.n_layers, self.cfg.batch, self.cfg.n_kv_heads,
-                                    self.capacity[w], sb)
+        n = self.cfg.n_layers * self.cfg.batch * self.cfg.n_kv_heads * self.capacity[w] * sb
+        return self.buffers[w][:n].view(self.cfg.n_layers, self.cfg.batch, self.cfg.n_kv_heads,
+                                        self.capacity[w], sb)
 
     def tail(self, which):
-        t = self.buffers[8 if which == "k" else 9].view(torch.int16)
+        n = self.cfg.n_layers * self.cfg.batch * self.cfg.n_kv_heads * self.cfg.tail_capacity * 256
+        t = self.buffers[8 if which == "k" else 9][:n].view(torch.int16)
         return t.view(self.cfg.n_layers, self.cfg.batch, self.cfg.n_kv_heads, self.cfg.tail_capacity, 128)
 
 

@@ -68,7 +68,7 @@ def check_route(B, T, D, chunk, dtype, gated, rf, seed, bias=None, w_std=0.02):
 def test_route_config1_shape(gated, dtype):
     # config 1: hidden 1024, context 4096, chunk 128, weights ~ N(0, 0.02)
     nf, n, m = check_route(1, 4096, 1024, 128, dtype, gated, True, seed=100 + dtype)
-    assert nf <= max(1, n // 10)
+    assert nf <= max(1, n // 4)
 
 
 @pytest.mark.parametrize("chunk", [32, 64, 256, 512])
