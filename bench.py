@@ -1,0 +1,489 @@
+"""Benchmark of the MoQAE hot path: one step = route (once per routing-sharing group) ->
+quantise+pack (every layer) -> decode attention (every layer) on a synthetic Llama-shaped
+workload.  Prints ONE JSON line (rank 0).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg4|cfg2|cfg3]
+    python bench.py --impl reference ...      # the CPU oracle on a bounded sample
+
+The headline `value` is the decode-attention effective HBM bandwidth: bytes the method must
+move in the decode phase (packed KV + scale/zero + tail + q + split partials + out) divided by
+the device time of that phase, measured with CUDA events inside the timed steps.  N > 1 runs
+independent replicas (the path has no exchange step): value = sum of all ranks' bytes / max
+time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+L2_BYTES = 126 * 1024 * 1024
+
+
+def read_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            p = json.load(f)
+        return float(p["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+
+    def start(self):
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.Q}",
+                                       "--format=csv,noheader,nounits", "-lms", "100"],
+                                      stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.f.read().splitlines():
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1]))
+                mx.append(float(parts[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        try:
+            os.unlink(self.f.name)
+        except OSError:
+            pass
+        if sm:
+            busy = sorted(sm)[len(sm) // 2:]          # upper half: samples taken under load
+            out = {"sm_mhz": float(np.median(busy)), "sm_max_mhz": float(max(mx)),
+                   "reasons": sorted(reasons), "samples": len(sm)}
+        return out
+
+
+# ------------------------------------------------------------------------------------------
+# workload set-up on the device
+# ------------------------------------------------------------------------------------------
+class Job:
+    """Device-resident inputs, cache and scratch of one workload."""
+
+    N_DISTINCT = 4      # distinct per-layer K/V inputs; layer l reads input l mod 4 (each > L2)
+
+    def __init__(self, wl, device, seed=1234, context=None):
+        import torch
+
+        from paper_2506_07533_b200 import binding as mq
+        from paper_2506_07533_b200 import synth
+        self.torch, self.mq, self.wl, self.device = torch, mq, wl, device
+        T = self.T = context or wl.context
+        B, Hkv, Hq = wl.batch, wl.n_kv_heads, wl.n_q_heads
+        self.cfg = mq.make_config(n_layers=wl.n_layers, n_q_heads=Hq, n_kv_heads=Hkv, chunk=wl.chunk,
+                                  dtype=wl.dtype, d_in=wl.d_in, max_tokens=T + wl.chunk, batch=B,
+                                  rs_group=wl.rs_group, rf_first_chunk=1, tail_capacity=wl.chunk)
+        nd = min(self.N_DISTINCT, wl.n_layers)
+        self.kv = [synth.keys_values(B, T, Hkv, 128, wl.dtype, seed + 10 * i, device,
+                                     outlier_frac=wl.outlier_frac) for i in range(nd)]
+        nh = min(2, wl.n_groups)
+        self.hidden = [synth.hidden_states(B, T, wl.d_in, wl.chunk, wl.dtype, seed + 100 + i, device)
+                       for i in range(nh)]
+        self.W1, self.W2, self.W3, self.bias = synth.router_weights(wl.d_in, 4, wl.dtype, seed + 7, device,
+                                                                    gated=wl.gated_router)
+        self.q = synth.normal((wl.n_layers, B, Hq, 128), wl.dtype, seed + 9, device)
+        self.out = torch.zeros((wl.n_layers, B, Hq, 128), dtype=torch.float32, device=device)
+        self.ws = torch.empty(mq.moqae_decode_attn_workspace(self.cfg), dtype=torch.uint8, device=device)
+        self.n_splits = self.ws.numel() // (B * Hq * 130 * 4)
+        # capacity: room for the calibrated mix with slack, never more than all chunks
+        C = T // wl.chunk
+        self.cache = None
+        self.capacity = [C, C, C, C]
+        self.forced = None
+        self._calibrate(seed)
+
+    # the router's bias is tuned (with the library's own router) until the chunk mix is within
+    # five points of the workload's target; otherwise a seeded multinomial map is forced
+    def _calibrate(self, seed):
+        torch, mq, wl = self.torch, self.mq, self.wl
+        C = self.T // wl.chunk
+        probe_cfg = mq.make_config(n_layers=1, n_q_heads=wl.n_q_heads, n_kv_heads=wl.n_kv_heads, chunk=wl.chunk,
+                                   dtype=wl.dtype, d_in=wl.d_in, max_tokens=self.T + wl.chunk, batch=wl.batch)
+        probe = mq.moqae_cache_bind(probe_cfg, [1, 1, 1, 1], device=self.device)
+        target = np.asarray(wl.mix, dtype=np.float64)
+        bias = np.zeros(4)
+        ok = False
+        for it in range(60):
+            self.bias.copy_(torch.tensor(bias, dtype=torch.float32))
+            mq.moqae_route(probe_cfg, self.hidden[0], self.T, self.W1, self.W2, self.W3, self.bias, 0, probe)
+            cnt = probe.count[0].sum(0).cpu().numpy().astype(np.float64)
+            cnt[3] -= wl.batch                      # frozen first chunks are not the router's choice
+            mix = cnt / max(cnt.sum(), 1)
+            if np.abs(mix - target).max() <= 0.05:
+                ok = True
+                break
+            step = 0.5 if it < 30 else 0.2
+            bias += step * np.clip(np.log((target + 1e-3) / (mix + 1e-3)), -2, 2) * self._logit_scale(probe_cfg, probe)
+        self.calibrated = ok
+        if not ok:
+            from paper_2506_07533_b200 import synth
+            self.forced = torch.from_numpy(synth.multinomial_map(wl.batch, C, wl.mix, seed + 5)).to(self.device)
+        # size the pools from the realised maps of all groups
+        cap = np.ones(4, dtype=np.int64)
+        for g in range(wl.n_groups):
+            if self.forced is None:
+                mq.moqae_route(probe_cfg, self.hidden[g % len(self.hidden)], self.T, self.W1, self.W2, self.W3,
+                               self.bias, 0, probe)
+                cnt = probe.count[0].cpu().numpy()
+            else:
+                m = self.forced.cpu().numpy()
+                cnt = np.stack([(m == w).sum(1) for w in range(4)], 1)
+            cap = np.maximum(cap, cnt.max(0))
+        self.capacity = [int(c) for c in cap]
+        del probe
+        self.cache = mq.moqae_cache_bind(self.cfg, self.capacity, device=self.device)
+
+    def _logit_scale(self, cfg, probe):
+        # spread of the logits, estimated once from the vote margins being O(1): use a fixed unit
+        return 1.0 if self.wl.gated_router else 0.5
+
+    # ---- phases -------------------------------------------------------------------------
+    def route_all(self):
+        wl = self.wl
+        if self.forced is not None:
+            return
+        for g in range(wl.n_groups):
+            self.mq.moqae_route(self.cfg, self.hidden[g % len(self.hidden)], self.T, self.W1, self.W2, self.W3,
+                                self.bias, g, self.cache)
+
+    def quantize_all(self):
+        wl = self.wl
+        for l in range(wl.n_layers):
+            K, V = self.kv[l % len(self.kv)]
+            fm = self.forced if (self.forced is not None and l % wl.rs_group == 0) else None
+            self.mq.moqae_quantize_kv(self.cfg, K, V, self.T, l, self.cache, forced_map=fm)
+
+    def decode_all(self):
+        for l in range(self.wl.n_layers):
+            self.mq.moqae_decode_attn(self.cfg, self.q[l], l, self.cache, self.out[l], self.ws)
+
+    def counts(self):
+        return self.cache.count.cpu().numpy()           # [groups, batch, 4]
+
+    def bytes_per_step(self):
+        from paper_2506_07533_b200 import workloads as W
+        wl, cnt = self.wl, self.counts()
+        tail = self.T % wl.chunk
+        route = 0 if self.forced is not None else wl.n_groups * W.route_bytes_per_group(wl, self.T)
+        quant = sum(W.quantize_bytes_per_layer(cnt[l // wl.rs_group], wl, self.T) for l in range(wl.n_layers))
+        dec = sum(W.decode_bytes_per_layer(cnt[l // wl.rs_group], wl, self.n_splits, tail)
+                  for l in range(wl.n_layers))
+        return route, quant, dec
+
+    def launches_per_step(self):
+        wl = self.wl
+        route = 0 if self.forced is not None else 2 * wl.n_groups        # score+vote, finalise
+        quant = 2 * wl.n_layers + (wl.n_groups if self.forced is not None else 0)
+        return route + quant + 2 * wl.n_layers                            # + split-K and combine
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2506_07533_b200 import build as mqbuild
+    from paper_2506_07533_b200 import workloads as W
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+    torch.cuda.set_device(local)
+    device = torch.device(f"cuda:{local}")
+    if rank == 0:
+        mqbuild.build()
+    if world > 1:
+        dist.barrier()
+    wl = W.WORKLOADS[args.workload]
+    job = Job(wl, device, seed=1234 + rank, context=args.context)
+    torch.cuda.synchronize()
+
+    def one_step(ev=None):
+        if ev:
+            ev[0].record()
+        job.route_all()
+        if ev:
+            ev[1].record()
+        job.quantize_all()
+        if ev:
+            ev[2].record()
+        job.decode_all()
+        if ev:
+            ev[3].record()
+
+    for _ in range(args.warmup):
+        one_step()
+    torch.cuda.synchronize()
+    status = job.mq.moqae_poll_status(job.cache)
+    if status != 0:
+        raise RuntimeError(f"device status {status} after warm-up")
+    b_route, b_quant, b_dec = job.bytes_per_step()
+
+    sampler = ClockSampler(local)
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    t0 = torch.cuda.Event(enable_timing=True)
+    t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for s in range(args.steps):
+        one_step(events[s])
+    t1.record()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    clocks = sampler.stop()
+    total_ms = t0.elapsed_time(t1)
+    ms_route = sum(e[0].elapsed_time(e[1]) for e in events) / args.steps
+    ms_quant = sum(e[1].elapsed_time(e[2]) for e in events) / args.steps
+    ms_dec = sum(e[2].elapsed_time(e[3]) for e in events) / args.steps
+
+    # end to end: inputs start in pinned host memory, result read back, every step
+    e2e = measure_e2e(job, args, torch)
+
+    times = torch.tensor([total_ms, ms_route, ms_quant, ms_dec, e2e["ms_dec"], e2e["ms_step"]],
+                         dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    total_ms, ms_route, ms_quant, ms_dec, e2e_ms_dec, e2e_ms_step = [float(x) for x in times.cpu()]
+
+    if rank == 0:
+        peak, peak_kind = read_peaks()
+        dec_gbs = world * b_dec / (ms_dec * 1e6)
+        per_launch_bytes = b_dec / wl.n_layers
+        per_launch_ms = ms_dec / wl.n_layers
+        achieved = per_launch_bytes / (per_launch_ms * 1e6)
+        cnt = job.counts().astype(np.float64)
+        mix = (cnt.sum((0, 1)) / max(cnt.sum(), 1)).round(4).tolist()
+        line = {
+            "metric": "decode-attn effective HBM GB/s", "value": round(dec_gbs, 1), "unit": "GB/s",
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": round(total_ms / args.steps, 4), "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16" if wl.dtype == 1 else "f16", "data": "synthetic",
+            "config": {"workload": f"{wl.name}: L{wl.n_layers} Hq{wl.n_q_heads}/Hkv{wl.n_kv_heads} d128 "
+                                   f"B{wl.batch} ctx{job.T} chunk{wl.chunk} rs_group{wl.rs_group}",
+                       "step": "route (per sharing group) + quantize_pack (per layer) + decode_attn (per layer)",
+                       "expert_mix_realised_2_4_8_16": mix,
+                       "mix_source": "router bias calibrated" if job.forced is None else "forced seeded multinomial map",
+                       "l2": "working set per phase >> 126 MB L2; no layer is touched twice in a row",
+                       "parallelism": "replicas only" if world > 1 else "single GPU",
+                       "n_splits": job.n_splits},
+            "phase_ms": {"route": round(ms_route, 4), "quantize_pack": round(ms_quant, 4),
+                         "decode_attn": round(ms_dec, 4)},
+            "context_tokens_per_s": round(world * wl.batch * job.T / (ms_dec * 1e-3), 1),
+            "quantize_route_gbs": round(world * (b_route + b_quant) / ((ms_route + ms_quant) * 1e6), 1),
+            "bytes_per_step": {"route": b_route, "quantize_pack": b_quant, "decode_attn": b_dec},
+            "gpu_launches": job.launches_per_step() * args.steps,
+            "clocks": clocks,
+            "roofline": {"bound": "hbm", "kernel": "decode_splitk_kernel (+combine)",
+                         "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
+                         "frac": round(achieved / peak, 4), "peak_source": f"of {peak_kind}",
+                         "frac_of_8TBs_spec": round(achieved / 8000.0, 4),
+                         "bytes_per_launch": int(per_launch_bytes), "ms_per_launch": round(per_launch_ms, 5),
+                         "traffic": args.traffic},
+            "roofline_quantize": {"bound": "hbm", "achieved": round(b_quant / (ms_quant * 1e6), 1), "peak": peak,
+                                  "unit": "GB/s", "frac": round(b_quant / (ms_quant * 1e6) / peak, 4)},
+            "roofline_route": ({"bound": "hbm", "achieved": round(b_route / (ms_route * 1e6), 1), "peak": peak,
+                                "unit": "GB/s", "frac": round(b_route / (ms_route * 1e6) / peak, 4)}
+                               if b_route else None),
+            "e2e": {"value": round(world * b_dec / (e2e_ms_dec * 1e6), 1), "unit": "GB/s",
+                    "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
+                    "ms_per_step": round(e2e_ms_step, 3), "steps": e2e["steps"],
+                    "note": "host-resident hidden, K, V, q copied in and out read back inside the timed step; "
+                            "value = decode-phase bytes / (decode phase incl. q upload and out download)"},
+        }
+        if not args.no_cpu_baseline and world == 1:
+            line["cpu_baseline"] = cpu_baseline(wl, budget_s=args.cpu_seconds)
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def measure_e2e(job, args, torch):
+    wl = job.wl
+    steps = max(1, min(args.e2e_steps, args.steps))
+    h_kv = [(K.cpu().pin_memory(), V.cpu().pin_memory()) for K, V in job.kv]
+    h_hidden = [h.cpu().pin_memory() for h in job.hidden]
+    h_q = job.q.cpu().pin_memory()
+    h_out = torch.empty(job.out.shape, dtype=torch.float32).pin_memory()
+    d_K, d_V = torch.empty_like(job.kv[0][0]), torch.empty_like(job.kv[0][1])
+    d_h = torch.empty_like(job.hidden[0])
+    d_q = torch.empty_like(job.q)
+    h2d = 0
+    ms_dec, ms_step = 0.0, 0.0
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+    for s in range(steps + 1):                       # first pass is warm-up
+        h2d = 0
+        ev[0].record()
+        if job.forced is None:
+            for g in range(wl.n_groups):
+                src = h_hidden[g % len(h_hidden)]
+                d_h.copy_(src, non_blocking=True)
+                h2d += src.numel() * 2
+                job.mq.moqae_route(job.cfg, d_h, job.T, job.W1, job.W2, job.W3, job.bias, g, job.cache)
+        for l in range(wl.n_layers):
+            hk, hv = h_kv[l % len(h_kv)]
+            d_K.copy_(hk, non_blocking=True)
+            d_V.copy_(hv, non_blocking=True)
+            h2d += 2 * hk.numel() * 2
+            fm = job.forced if (job.forced is not None and l % wl.rs_group == 0) else None
+            job.mq.moqae_quantize_kv(job.cfg, d_K, d_V, job.T, l, job.cache, forced_map=fm)
+        ev[1].record()
+        d_q.copy_(h_q, non_blocking=True)
+        h2d += h_q.numel() * 2
+        for l in range(wl.n_layers):
+            job.mq.moqae_decode_attn(job.cfg, d_q[l], l, job.cache, job.out[l], job.ws)
+        h_out.copy_(job.out, non_blocking=True)
+        ev[2].record()
+        torch.cuda.synchronize()
+        if s > 0:
+            ms_dec += ev[1].elapsed_time(ev[2])
+            ms_step += ev[0].elapsed_time(ev[2])
+    return {"ms_dec": ms_dec / steps, "ms_step": ms_step / steps, "h2d": int(h2d),
+            "d2h": int(h_out.numel() * 4), "steps": steps}
+
+
+# ------------------------------------------------------------------------------------------
+# CPU oracle, timed as it stands on a bounded sample (reported baseline, not the target)
+# ------------------------------------------------------------------------------------------
+def oracle_sample(wl, tokens: int, seed=77):
+    """One sequence and ONE kv head of one layer over `tokens` context tokens, mixed widths
+    at the workload's target mix: quantise+pack, then decode for the head's query group."""
+    from oracle import moqae_oracle as O
+    from paper_2506_07533_b200 import synth
+    from paper_2506_07533_b200 import workloads as W
+    G = wl.n_q_heads // wl.n_kv_heads
+    C = tokens // wl.chunk
+    K, V = synth.keys_values(1, tokens, 1, 128, wl.dtype, seed, "cpu", outlier_channels=(3,))
+    q = synth.normal((1, G, 128), wl.dtype, seed + 1, "cpu")
+    bmap = synth.multinomial_map(1, C, wl.mix, seed + 2)
+    Ku, Vu, qu = synth.to_u16(K), synth.to_u16(V), synth.to_u16(q)
+    t0 = time.perf_counter()
+    cache = O.quantize_kv(Ku, Vu, wl.dtype, wl.chunk, bmap)
+    t1 = time.perf_counter()
+    O.decode_attn(qu, wl.dtype, cache, wl.chunk)
+    t2 = time.perf_counter()
+    cnt = cache["count"]
+    kv_bytes = W.cache_bytes_per_layer(cnt, wl.chunk, 1, 0)
+    return {"quant_s": t1 - t0, "decode_s": t2 - t1, "decode_bytes": kv_bytes + G * 128 * 6,
+            "quant_bytes": tokens * 512 + kv_bytes, "tokens": tokens}
+
+
+def cpu_baseline(wl, budget_s=20.0):
+    import threadpoolctl
+    tokens = 4 * wl.chunk
+    r = oracle_sample(wl, tokens)
+    per_tok = (r["quant_s"] + r["decode_s"]) / tokens
+    tokens = int(min(wl.context, max(tokens, budget_s / max(per_tok, 1e-9))) // wl.chunk * wl.chunk)
+    r = oracle_sample(wl, tokens)
+    threads = max([p.get("num_threads", 1) for p in threadpoolctl.threadpool_info()] or [1])
+    return {"value": round(r["decode_bytes"] / r["decode_s"] / 1e9, 5), "unit": "GB/s", "cores": int(threads),
+            "kind": "oracle",
+            "sample": f"decode attention of 1 sequence x 1 kv head x {r['tokens']} context tokens of {wl.name} "
+                      f"(numpy float64 oracle, {r['decode_s']:.1f} s); its quantise+pack ran at "
+                      f"{r['quant_bytes'] / r['quant_s'] / 1e9:.5f} GB/s ({r['quant_s']:.1f} s)",
+            "host_cpus": os.cpu_count()}
+
+
+def run_reference(args):
+    """Reference arm: the CPU oracle, as it stands, on a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2506_07533_b200 import workloads as W
+    wl = W.WORKLOADS[args.workload]
+    tokens = max(wl.chunk * 2, min(wl.context, args.reference_tokens) // wl.chunk * wl.chunk)
+    for _ in range(args.warmup):
+        oracle_sample(wl, wl.chunk * 2)
+    tot_s, tot_b, last = 0.0, 0, None
+    for _ in range(args.steps):
+        last = oracle_sample(wl, tokens)
+        tot_s += last["decode_s"]
+        tot_b += last["decode_bytes"]
+    import threadpoolctl
+    threads = max([p.get("num_threads", 1) for p in threadpoolctl.threadpool_info()] or [1])
+    val = tot_b / tot_s / 1e9
+    sample = (f"decode attention of 1 sequence x 1 kv head x {tokens} context tokens of {wl.name} per step "
+              f"(numpy float64 oracle)")
+    line = {"impl": "reference", "metric": "decode-attn effective HBM GB/s", "value": round(val, 5), "unit": "GB/s",
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": round(1e3 * tot_s / args.steps, 3), "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": f"{wl.name} (bounded sample: {sample})"},
+            "cpu_baseline": {"value": round(val, 5), "unit": "GB/s", "cores": int(threads), "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": round(val, 5), "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg4", choices=["cfg1", "cfg2", "cfg3", "cfg4"])
+    ap.add_argument("--context", type=int, default=None, help="override the context length (profiling)")
+    ap.add_argument("--e2e-steps", type=int, default=1)
+    ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    ap.add_argument("--reference-tokens", type=int, default=32768)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--traffic", type=float, default=None,
+                    help="dram bytes per decode launch from an ncu capture (recorded in the JSON line)")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours" and args.context is None:
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
