@@ -7,6 +7,8 @@
 // size in KiB (3, 5, 9, 16), so every CTA streams about the same number of bytes.
 // Each CTA writes, per query head of the group, a partial (max, sum, 128 weighted values);
 // decode_combine_kernel merges the partials with the log-sum-exp rule.
+#include <cstdlib>
+
 #include "common.cuh"
 
 namespace moqae {
@@ -20,7 +22,11 @@ struct SplitRange {
 };
 
 // Tiles of width w whose cost-axis start lies in [lo_cost, hi_cost).
-__device__ __forceinline__ SplitRange split_range(const int32_t* cnt, int tiles_per_chunk, int split, int n_splits) {
+__device__ __forceinline__ SplitRange split_range(const int32_t* cnt_in, const long long* capacity,
+                                                  int tiles_per_chunk, int split, int n_splits) {
+  int cnt[4];   // never walk past a pool's end, whatever the table says
+#pragma unroll
+  for (int w = 0; w < 4; ++w) cnt[w] = static_cast<int>(min(static_cast<long long>(max(cnt_in[w], 0)), capacity[w]));
   long long base[5];
   base[0] = 0;
 #pragma unroll
@@ -193,7 +199,7 @@ decode_splitk_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int 
   const int group = layer / dm.rs_group;
   const int32_t* cnt = cv.count + (static_cast<long long>(group) * dm.batch + b) * 4;
   const int tpc = dm.chunk / kTileTokens;
-  const SplitRange rg = split_range(cnt, tpc, split, n_splits);
+  const SplitRange rg = split_range(cnt, cv.capacity, tpc, split, n_splits);
 
   WarpState st;
 #pragma unroll
@@ -290,8 +296,10 @@ int decode_num_splits(const Dims& dm) {
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev);
     sms = v > 0 ? v : 148;
   }
+  // one full wave: every CTA gets the same number of bytes, so a partial second wave would
+  // cost a whole extra pass
   const int pairs = dm.batch * dm.n_kv_heads;
-  int s = (sms * 4 + pairs - 1) / pairs;
+  int s = (sms * decode_mma_ctas_per_sm()) / pairs;
   if (s < 1) s = 1;
   if (s > kMaxSplits) s = kMaxSplits;
   return s;
@@ -302,6 +310,16 @@ cudaError_t launch_decode(const Dims& dm, const CacheView& cv, const void* q, in
   const long long rows = static_cast<long long>(dm.batch) * dm.n_q_heads * n_splits;
   float* ws_o = workspace;
   float* ws_ml = workspace + rows * kHeadDim;
+  static const bool scalar = [] {
+    const char* e = getenv("MOQAE_DECODE_KERNEL");      // "scalar": plain-FMA kernel, for debugging
+    return e && e[0] == 's';
+  }();
+  if (!scalar) {
+    cudaError_t e = launch_decode_mma(dm, cv, q, layer, scale, ws_o, ws_ml, n_splits, st);
+    if (e != cudaSuccess) return e;
+    decode_combine_kernel<<<dm.batch * dm.n_q_heads, kHeadDim, 0, st>>>(ws_o, ws_ml, out, n_splits);
+    return cudaGetLastError();
+  }
   switch (dm.n_q_heads / dm.n_kv_heads) {
     case 1: return launch_decode_g<1>(dm, cv, q, layer, out, scale, ws_o, ws_ml, n_splits, st);
     case 2: return launch_decode_g<2>(dm, cv, q, layer, out, scale, ws_o, ws_ml, n_splits, st);

@@ -1,0 +1,680 @@
+// Split-K decode attention, tensor-core version (the production path).
+//
+// Each warp is an independent stream processor: it owns a private ring of shared-memory
+// stages that one elected lane fills with 1-D bulk copies (cp.async.bulk + mbarrier
+// complete_tx), and it consumes whole tiles from that ring.  Per 32-token tile:
+//
+//   scores   S[t][q] = sum_c code[t][c] * (q[c] s_k[c]) + sum_c q[c] z_k[c]
+//            The codes are never converted: a masked word IS a pair of fp16 subnormals
+//            (code * 4^j * 2^-24), the power of two and the key scale are folded into the
+//            query fragment once per tile, and the product runs on mma.sync m16n8k16
+//            (A = 16 tokens x 16 channels of codes, B = folded queries of the GQA group
+//            padded to 8 columns, fp32 accumulate).  The zero-point term is a second MMA
+//            chain with exact fp16 operands (A = z_k, B = q).
+//   softmax  online, base 2, in registers; the 64x offset keeps p*s_v in fp16 range.
+//   output   out[c][q] = sum_t code[t][c] * (p[t][q] s_v[t][cg]) + sum_t p[t][q] z_v[t][cg]
+//            again with untouched codes as the A operand (A = V^T, 16 channels x 16 tokens),
+//            P transposed in registers with movmatrix, and one extra MMA for the zero term.
+//
+// 16-bit tiles and the 16-bit tail run the same MMAs on the raw values.
+// Every wait on an mbarrier is bounded; on expiry the warp records MOQAE_ERR_TIMEOUT in
+// the cache's status word and stops consuming.
+#include <cuda_bf16.h>
+
+#include "common.cuh"
+
+namespace moqae {
+
+namespace {
+
+constexpr int kWarps = 6;
+constexpr int kThreads = kWarps * 32;
+constexpr int kRingBytes = 18432;             // per warp: 6 x 3 KiB = 3 x 5 KiB(+) = 2 x 9 KiB = 2 x 8 KiB(+)
+constexpr int kQBytes = 8 * kHeadDim * 2;     // one 8-query fragment source, 16-bit
+constexpr long long kWaitLimit = 1ll << 20;   // try_wait attempts before giving up
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, int count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
+               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+  for (long long i = 0; i < kWaitLimit; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  return false;
+}
+
+template <bool BF16>
+__device__ __forceinline__ void mma16816(float d[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1) {
+  if (BF16) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+  } else {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+  }
+}
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x) {
+  uint32_t r;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;\n" : "=r"(r) : "r"(x));
+  return r;
+}
+__device__ __forceinline__ float ex2f(float x) {
+  float r;
+  asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(r) : "f"(x));
+  return r;
+}
+__device__ __forceinline__ uint32_t hmul2_u32(uint32_t a, uint32_t b) {
+  uint32_t r;
+  asm("mul.rn.f16x2 %0, %1, %2;\n" : "=r"(r) : "r"(a), "r"(b));
+  return r;
+}
+// a*b - c in one rounding: with c = round(a*b) this is the exact rounding error of the product
+__device__ __forceinline__ uint32_t hfma2_sub_u32(uint32_t a, uint32_t b, uint32_t c) {
+  uint32_t r;
+  asm("{\n.reg .b32 n;\nneg.f16x2 n, %3;\nfma.rn.f16x2 %0, %1, %2, n;\n}\n" : "=r"(r) : "r"(a), "r"(b), "r"(c));
+  return r;
+}
+__device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
+  const __half2 h = __floats2half2_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&h);
+}
+__device__ __forceinline__ uint32_t pack_bf162(float lo, float hi) {
+  const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&h);
+}
+
+// ---- code extraction: masked words are pairs of fp16 subnormals ------------------------
+template <int BITS> struct Fmt;
+template <> struct Fmt<2> { static constexpr int regs = 8, direct = 5, shift = 10; static constexpr uint32_t mask = 0x00030003u; };
+template <> struct Fmt<4> { static constexpr int regs = 4, direct = 2, shift = 8;  static constexpr uint32_t mask = 0x000F000Fu; };
+template <> struct Fmt<8> { static constexpr int regs = 2, direct = 1, shift = 8;  static constexpr uint32_t mask = 0x00FF00FFu; };
+
+// bit position (inside a half-word) of the code that register m of a word carries
+template <int BITS> __host__ __device__ constexpr int bitpos(int m) {
+  return m < Fmt<BITS>::direct ? BITS * m : BITS * (m - Fmt<BITS>::direct);
+}
+template <int BITS> __device__ __forceinline__ uint32_t ext(uint32_t w, uint32_t wsh, int m) {
+  return m < Fmt<BITS>::direct ? (w & (Fmt<BITS>::mask << (BITS * m)))
+                               : (wsh & (Fmt<BITS>::mask << (BITS * (m - Fmt<BITS>::direct))));
+}
+// fp16 constant 2^e as a half2 bit pattern (e in the normal range)
+__host__ __device__ constexpr uint32_t half2_pow2(int e) {
+  return (static_cast<uint32_t>(e + 15) << 10) | (static_cast<uint32_t>(e + 15) << 26);
+}
+
+struct State {
+  float acc[8][4];   // M-tile mt = 2*cg + hf: rows g / g+8 = channels 32cg+4g+2hf / +1; cols = queries 2t4, 2t4+1
+  float oz[4];       // rows 0..3 (lanes g < 4): zero-point term per channel group; row 4 (g == 4): the
+                     // running sums l, taken over the SAME rounded weights the values are multiplied by
+  float m[2];        // running maxima (base-2 exponent units) of queries 2t4, 2t4+1
+};
+
+__device__ __forceinline__ void rescale(State& st, float c0, float c1) {
+#pragma unroll
+  for (int mt = 0; mt < 8; ++mt) {
+    st.acc[mt][0] *= c0; st.acc[mt][1] *= c1; st.acc[mt][2] *= c0; st.acc[mt][3] *= c1;
+  }
+  st.oz[0] *= c0; st.oz[1] *= c1; st.oz[2] *= c0; st.oz[3] *= c1;
+}
+
+// Online-softmax update for NV score vectors x[v][4] (d-fragment order: row g q0, row g q1,
+// row g+8 q0, row g+8 q1; already in base-2 units; -inf = masked).  Returns p~ = 64 * p.
+template <int NV>
+__device__ __forceinline__ void softmax_update(State& st, float x[NV][4]) {
+  float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+  for (int v = 0; v < NV; ++v) {
+    mx0 = fmaxf(mx0, fmaxf(x[v][0], x[v][2]));
+    mx1 = fmaxf(mx1, fmaxf(x[v][1], x[v][3]));
+  }
+#pragma unroll
+  for (int o = 4; o <= 16; o <<= 1) {
+    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, o));
+    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, o));
+  }
+  const float n0 = fmaxf(st.m[0], mx0), n1 = fmaxf(st.m[1], mx1);
+  const bool changed = (n0 != st.m[0]) || (n1 != st.m[1]);
+  if (__any_sync(0xffffffffu, changed)) {
+    const float c0 = (st.m[0] == -INFINITY) ? 0.0f : ex2f(st.m[0] - n0);
+    const float c1 = (st.m[1] == -INFINITY) ? 0.0f : ex2f(st.m[1] - n1);
+    rescale(st, c0, c1);
+    st.m[0] = n0; st.m[1] = n1;
+  }
+  const float o0 = 6.0f - st.m[0], o1 = 6.0f - st.m[1];
+#pragma unroll
+  for (int v = 0; v < NV; ++v) {
+    x[v][0] = ex2f(x[v][0] + o0); x[v][1] = ex2f(x[v][1] + o1);
+    x[v][2] = ex2f(x[v][2] + o0); x[v][3] = ex2f(x[v][3] + o1);
+  }
+}
+
+// ---- one quantised tile (32 tokens) from shared memory ---------------------------------
+// qc[r], r = 0..15: fp16 pair q[32*t4 + 2r], q[.. + 1] of query g (zero for g >= G), times the
+// power of two that undoes the bit position of the codes register r multiplies.  qsm: the
+// same pairs unscaled, in shared memory.
+template <int BITS>
+__device__ __forceinline__ void process_qtile(const uint8_t* __restrict__ tile, State& st,
+                                              const uint32_t (&qc)[16], const uint16_t* __restrict__ qsm,
+                                              float c_score, float c_bias, int lane) {
+  using F = Fmt<BITS>;
+  const int g = lane >> 2, t4 = lane & 3;
+  constexpr int kRowBytes = 16 * BITS;
+  const uint8_t* kpay = tile + kMetaBytes;
+  const uint8_t* vpay = kpay + kTileTokens * kRowBytes;
+
+  // fold the key scales into the query fragment: q*s = hi + lo exactly (two fp16 each)
+  uint32_t qf[16], ql[16];
+  {
+    const uint4* sp = reinterpret_cast<const uint4*>(tile + 64 * t4);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const uint4 s4 = sp[i];
+      const uint32_t sv[4] = {s4.x, s4.y, s4.z, s4.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int r = 4 * i + j;
+        qf[r] = hmul2_u32(qc[r], sv[j]);
+        ql[r] = hfma2_sub_u32(qc[r], sv[j], qf[r]);
+      }
+    }
+  }
+  // zero-point term of the scores: bias[q] = sum_c z_k[c] q[c], exact products (row 0 only)
+  float bz[4] = {0.f, 0.f, 0.f, 0.f}, bz2[4] = {0.f, 0.f, 0.f, 0.f};
+  {
+    const uint4* zp = reinterpret_cast<const uint4*>(tile + 256 + 64 * t4);
+    const uint4* qp = reinterpret_cast<const uint4*>(qsm + g * kHeadDim + 32 * t4);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      uint4 z4 = make_uint4(0u, 0u, 0u, 0u);
+      if (g == 0) z4 = zp[i];
+      const uint4 q4 = qp[i];
+      mma16816<false>(bz, z4.x, 0u, z4.y, 0u, q4.x, q4.y);
+      mma16816<false>(bz2, z4.z, 0u, z4.w, 0u, q4.z, q4.w);
+    }
+  }
+  const float bias0 = __shfl_sync(0xffffffffu, bz[0] + bz2[0], t4) * c_bias;
+  const float bias1 = __shfl_sync(0xffffffffu, bz[1] + bz2[1], t4) * c_bias;
+
+  // scores of the two 16-token blocks
+  float x[2][4];
+#pragma unroll
+  for (int blk = 0; blk < 2; ++blk) {
+    uint32_t a[2][16];
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+      const int row = 16 * blk + g + 8 * hh;
+      const uint8_t* rp = kpay + row * kRowBytes;
+      uint32_t w[BITS];           // 2, 4 or 8 words per thread and row
+      if (BITS == 2) {
+        const uint2 v = *reinterpret_cast<const uint2*>(rp + 8 * t4);
+        w[0] = v.x; w[1] = v.y;
+      } else if (BITS == 4) {
+        const uint4 v = *reinterpret_cast<const uint4*>(rp + 16 * t4);
+        w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
+      } else {
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+          const uint4 v = *reinterpret_cast<const uint4*>(rp + (((2 * t4 + j) ^ (row & 7)) << 4));
+          w[4 * j] = v.x; w[4 * j + 1] = v.y; w[4 * j + 2] = v.z; w[4 * j + 3] = v.w;
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < BITS; ++j) {
+        const uint32_t wsh = w[j] >> F::shift;
+#pragma unroll
+        for (int m = 0; m < F::regs; ++m) a[hh][j * F::regs + m] = ext<BITS>(w[j], wsh, m);
+      }
+    }
+    float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int ks = 0; ks < 8; ks += 2) {
+      mma16816<false>(s0, a[0][2 * ks], a[1][2 * ks], a[0][2 * ks + 1], a[1][2 * ks + 1], qf[2 * ks], qf[2 * ks + 1]);
+      mma16816<false>(s1, a[0][2 * ks + 2], a[1][2 * ks + 2], a[0][2 * ks + 3], a[1][2 * ks + 3], qf[2 * ks + 2], qf[2 * ks + 3]);
+      mma16816<false>(s0, a[0][2 * ks], a[1][2 * ks], a[0][2 * ks + 1], a[1][2 * ks + 1], ql[2 * ks], ql[2 * ks + 1]);
+      mma16816<false>(s1, a[0][2 * ks + 2], a[1][2 * ks + 2], a[0][2 * ks + 3], a[1][2 * ks + 3], ql[2 * ks + 2], ql[2 * ks + 3]);
+    }
+    x[blk][0] = fmaf(s0[0] + s1[0], c_score, bias0);
+    x[blk][1] = fmaf(s0[1] + s1[1], c_score, bias1);
+    x[blk][2] = fmaf(s0[2] + s1[2], c_score, bias0);
+    x[blk][3] = fmaf(s0[3] + s1[3], c_score, bias1);
+  }
+  softmax_update<2>(st, x);
+
+  const __half* vs = reinterpret_cast<const __half*>(tile + 512);
+  const __half* vz = reinterpret_cast<const __half*>(tile + 768);
+#pragma unroll
+  for (int blk = 0; blk < 2; ++blk) {
+    const uint32_t p0 = movmatrix_trans(pack_half2(x[blk][0], x[blk][1]));   // tokens 2t4, 2t4+1 of query g
+    const uint32_t p1 = movmatrix_trans(pack_half2(x[blk][2], x[blk][3]));   // tokens 2t4+8, 2t4+9
+    const int tk = 16 * blk + 2 * t4;
+    {  // zero-point term: rows = channel groups (lanes g < 4)
+      uint32_t z0 = (g == 4) ? 0x3C003C00u : 0u, z1 = z0;      // row 4: ones -> sum of the weights
+      if (g < 4) {
+        z0 = *reinterpret_cast<const uint32_t*>(vz + g * 32 + tk);
+        z1 = *reinterpret_cast<const uint32_t*>(vz + g * 32 + tk + 8);
+      }
+      mma16816<false>(st.oz, z0, 0u, z1, 0u, p0, p1);
+    }
+    uint32_t pb[4][2];
+#pragma unroll
+    for (int cg = 0; cg < 4; ++cg) {
+      pb[cg][0] = hmul2_u32(p0, *reinterpret_cast<const uint32_t*>(vs + cg * 32 + tk));
+      pb[cg][1] = hmul2_u32(p1, *reinterpret_cast<const uint32_t*>(vs + cg * 32 + tk + 8));
+    }
+    // value codes of token rows tk, tk+1, tk+8, tk+9: this lane's 16 positions 16g..16g+15
+    constexpr int NWV = BITS / 2;
+    uint32_t wv[4][NWV];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int row = tk + (i & 1) + 8 * (i >> 1);
+      const uint8_t* rp = vpay + row * kRowBytes;
+      if (BITS == 2) {
+        wv[i][0] = *reinterpret_cast<const uint32_t*>(rp + 4 * g);
+      } else if (BITS == 4) {
+        const uint2 v = *reinterpret_cast<const uint2*>(rp + 8 * g);
+        wv[i][0] = v.x; wv[i][NWV - 1] = v.y;
+      } else {
+        const uint4 v = *reinterpret_cast<const uint4*>(rp + ((g ^ (row & 7)) << 4));
+        wv[i][0] = v.x; wv[i][1 % NWV] = v.y; wv[i][2 % NWV] = v.z; wv[i][3 % NWV] = v.w;
+      }
+    }
+#pragma unroll
+    for (int jv = 0; jv < NWV; ++jv) {
+      const uint32_t lo01 = __byte_perm(wv[0][jv], wv[1][jv], 0x5410), hi01 = __byte_perm(wv[0][jv], wv[1][jv], 0x7632);
+      const uint32_t lo23 = __byte_perm(wv[2][jv], wv[3][jv], 0x5410), hi23 = __byte_perm(wv[2][jv], wv[3][jv], 0x7632);
+      const uint32_t lo01s = lo01 >> F::shift, hi01s = hi01 >> F::shift, lo23s = lo23 >> F::shift, hi23s = hi23 >> F::shift;
+#pragma unroll
+      for (int m = 0; m < F::regs; ++m) {
+        // register m of word jv holds positions jv*n + 2m (low halves) and + 2m + 1 (high halves)
+        constexpr int n = 32 / BITS;
+        const int i16 = jv * n + 2 * m;
+        const int cg = i16 >> 2, hf = (i16 & 3) >> 1;
+        mma16816<false>(st.acc[2 * cg + hf], ext<BITS>(lo01, lo01s, m), ext<BITS>(hi01, hi01s, m),
+                        ext<BITS>(lo23, lo23s, m), ext<BITS>(hi23, hi23s, m), pb[cg][0], pb[cg][1]);
+      }
+    }
+  }
+}
+
+// power of two that M-tile mt's accumulator carries inside a quantised phase (code unit / 2^-24)
+template <int BITS> __host__ __device__ constexpr int v_bitpos_of_mtile(int mt) {
+  // i16 = 4*cg + 2*hf with mt = 2*cg + hf;  word jv = i16 / n, register m = (i16 % n) / 2
+  return bitpos<BITS>(((2 * mt) % (32 / BITS)) / 2);
+}
+template <int BITS>
+__device__ __forceinline__ void phase_scale(State& st, bool enter) {
+#pragma unroll
+  for (int mt = 0; mt < 8; ++mt) {
+    const int e = v_bitpos_of_mtile<BITS>(mt) - 24;          // accumulator = true * 2^e
+    const float f = enter ? exp2f(static_cast<float>(e)) : exp2f(static_cast<float>(-e));
+#pragma unroll
+    for (int i = 0; i < 4; ++i) st.acc[mt][i] *= f;
+  }
+}
+
+// ---- 16 raw rows (pool tile half or tail block) from shared memory ---------------------
+// ks/vs: 16 rows x 256 B, 16-byte units swizzled by (row & 7).  qr[r]: q pairs of the raw
+// channel set (units 2t4, 2t4+1, 8+2t4, 9+2t4) in the INPUT dtype.
+template <bool BF16>
+__device__ __forceinline__ void process_raw16(const uint8_t* __restrict__ ks, const uint8_t* __restrict__ vs,
+                                              int n_valid, State& st, const uint32_t (&qr)[16], float c_score, int lane) {
+  const int g = lane >> 2, t4 = lane & 3;
+  float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+  for (int jj = 0; jj < 4; ++jj) {
+    const int U = (jj & 2) * 4 + 2 * t4 + (jj & 1);
+    const int up = (U & 8) | ((U ^ g) & 7);                  // (g + 8) & 7 == g & 7
+    const uint4 lo = *reinterpret_cast<const uint4*>(ks + g * 256 + up * 16);
+    const uint4 hi = *reinterpret_cast<const uint4*>(ks + (g + 8) * 256 + up * 16);
+    mma16816<BF16>(s0, lo.x, hi.x, lo.y, hi.y, qr[4 * jj], qr[4 * jj + 1]);
+    mma16816<BF16>(s1, lo.z, hi.z, lo.w, hi.w, qr[4 * jj + 2], qr[4 * jj + 3]);
+  }
+  float x[1][4];
+  x[0][0] = (g < n_valid) ? (s0[0] + s1[0]) * c_score : -INFINITY;
+  x[0][1] = (g < n_valid) ? (s0[1] + s1[1]) * c_score : -INFINITY;
+  x[0][2] = (g + 8 < n_valid) ? (s0[2] + s1[2]) * c_score : -INFINITY;
+  x[0][3] = (g + 8 < n_valid) ? (s0[3] + s1[3]) * c_score : -INFINITY;
+  softmax_update<1>(st, x);
+  uint32_t p0, p1, q0 = 0u, q1 = 0u;
+  if (BF16) {   // p~ = hi + lo, both bf16, so the weights keep ~16 bits
+    const uint32_t h01 = pack_bf162(x[0][0], x[0][1]), h23 = pack_bf162(x[0][2], x[0][3]);
+    const float r0 = x[0][0] - __uint_as_float(h01 << 16), r1 = x[0][1] - __uint_as_float(h01 & 0xffff0000u);
+    const float r2 = x[0][2] - __uint_as_float(h23 << 16), r3 = x[0][3] - __uint_as_float(h23 & 0xffff0000u);
+    p0 = movmatrix_trans(h01); p1 = movmatrix_trans(h23);
+    q0 = movmatrix_trans(pack_bf162(r0, r1)); q1 = movmatrix_trans(pack_bf162(r2, r3));
+  } else {
+    p0 = movmatrix_trans(pack_half2(x[0][0], x[0][1]));
+    p1 = movmatrix_trans(pack_half2(x[0][2], x[0][3]));
+  }
+  {  // running sums: a row of ones in oz row 4
+    const uint32_t ones = (g == 4) ? (BF16 ? 0x3F803F80u : 0x3C003C00u) : 0u;
+    mma16816<BF16>(st.oz, ones, 0u, ones, 0u, p0, p1);
+    if (BF16) mma16816<BF16>(st.oz, ones, 0u, ones, 0u, q0, q1);
+  }
+#pragma unroll
+  for (int cg = 0; cg < 4; ++cg) {
+    // channels 32cg + 4g .. +3 of token rows 2t4, 2t4+1, 2t4+8, 2t4+9
+    const int U = 4 * cg + (g >> 1);
+    uint2 w[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int row = 2 * t4 + (i & 1) + 8 * (i >> 1);
+      const int up = (U & 8) | ((U ^ row) & 7);
+      w[i] = *reinterpret_cast<const uint2*>(vs + row * 256 + up * 16 + (g & 1) * 8);
+    }
+#pragma unroll
+    for (int hf = 0; hf < 2; ++hf) {
+      const uint32_t w0 = hf ? w[0].y : w[0].x, w1 = hf ? w[1].y : w[1].x;
+      const uint32_t w2 = hf ? w[2].y : w[2].x, w3 = hf ? w[3].y : w[3].x;
+      const uint32_t a0 = __byte_perm(w0, w1, 0x5410), a1 = __byte_perm(w0, w1, 0x7632);
+      const uint32_t a2 = __byte_perm(w2, w3, 0x5410), a3 = __byte_perm(w2, w3, 0x7632);
+      mma16816<BF16>(st.acc[2 * cg + hf], a0, a1, a2, a3, p0, p1);
+      if (BF16) mma16816<BF16>(st.acc[2 * cg + hf], a0, a1, a2, a3, q0, q1);
+    }
+  }
+}
+
+struct SplitRange { int lo[4], hi[4]; };
+
+__device__ __forceinline__ SplitRange split_range(const int32_t* cnt_in, const long long* capacity,
+                                                  int tiles_per_chunk, int split, int n_splits) {
+  int cnt[4];   // never walk past a pool's end, whatever the table says
+#pragma unroll
+  for (int w = 0; w < 4; ++w) cnt[w] = static_cast<int>(min(static_cast<long long>(max(cnt_in[w], 0)), capacity[w]));
+  long long base[5];
+  base[0] = 0;
+#pragma unroll
+  for (int w = 0; w < 4; ++w)
+    base[w + 1] = base[w] + static_cast<long long>(cnt[w]) * tiles_per_chunk * tile_cost_of_expert(w);
+  const long long total = base[4];
+  const long long lo_c = total * split / n_splits, hi_c = total * (split + 1) / n_splits;
+  SplitRange r;
+#pragma unroll
+  for (int w = 0; w < 4; ++w) {
+    const long long cost = tile_cost_of_expert(w);
+    const long long n = static_cast<long long>(cnt[w]) * tiles_per_chunk;
+    long long a = lo_c - base[w], b = hi_c - base[w];
+    a = a <= 0 ? 0 : (a + cost - 1) / cost;
+    b = b <= 0 ? 0 : (b + cost - 1) / cost;
+    r.lo[w] = static_cast<int>(a < n ? a : n);
+    r.hi[w] = static_cast<int>(b < n ? b : n);
+  }
+  return r;
+}
+
+// per-warp pipeline bookkeeping
+struct Pipe {
+  uint32_t ring;        // shared address of this warp's ring
+  uint32_t bars;        // shared address of its 6 mbarriers
+  uint32_t parity;      // bit s = parity to wait for on stage s
+  bool ok;
+};
+
+// Stream `n_units` units of `unit_bytes` (each made of `pieces` bulk copies) through the ring.
+// UNIT_BYTES / STAGES are compile-time; src(u, piece) gives each piece's global address.
+template <int STAGES, int STAGE_BYTES, int PIECES, typename SrcFn, typename ConsumeFn>
+__device__ __forceinline__ void stream_units(Pipe& pp, int n_units, int lane, SrcFn src, ConsumeFn consume,
+                                             const uint8_t* ring_generic) {
+  if (n_units <= 0 || !pp.ok) return;
+  constexpr uint32_t piece_bytes = STAGE_BYTES / PIECES;
+  if (lane == 0) {
+    const int pre = n_units < STAGES ? n_units : STAGES;
+    for (int u = 0; u < pre; ++u) {
+      const uint32_t bar = pp.bars + 8 * u;
+      mbar_expect_tx(bar, STAGE_BYTES);
+#pragma unroll
+      for (int p = 0; p < PIECES; ++p) bulk_load(pp.ring + u * STAGE_BYTES + p * piece_bytes, src(u, p), piece_bytes, bar);
+    }
+  }
+  for (int u = 0; u < n_units; ++u) {
+    const int s = u % STAGES;
+    const uint32_t bar = pp.bars + 8 * s;
+    if (!mbar_wait_bounded(bar, (pp.parity >> s) & 1u)) { pp.ok = false; return; }
+    pp.parity ^= (1u << s);
+    consume(ring_generic + s * STAGE_BYTES, u);
+    __syncwarp();
+    if (lane == 0 && u + STAGES < n_units) {
+      mbar_expect_tx(bar, STAGE_BYTES);
+#pragma unroll
+      for (int p = 0; p < PIECES; ++p)
+        bulk_load(pp.ring + s * STAGE_BYTES + p * piece_bytes, src(u + STAGES, p), piece_bytes, bar);
+    }
+  }
+}
+
+__device__ __forceinline__ void load_qraw(uint32_t (&qraw)[16], const uint16_t* qsrc, int g, int t4) {
+  const uint4* p = reinterpret_cast<const uint4*>(qsrc + g * kHeadDim + 32 * t4);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const uint4 v = p[i];
+    qraw[4 * i] = v.x; qraw[4 * i + 1] = v.y; qraw[4 * i + 2] = v.z; qraw[4 * i + 3] = v.w;
+  }
+}
+__device__ __forceinline__ void load_qraw_rawset(uint32_t (&qr)[16], const uint16_t* qsrc, int g, int t4) {
+#pragma unroll
+  for (int jj = 0; jj < 4; ++jj) {
+    const int U = (jj & 2) * 4 + 2 * t4 + (jj & 1);
+    const uint4 v = *reinterpret_cast<const uint4*>(qsrc + g * kHeadDim + 8 * U);
+    qr[4 * jj] = v.x; qr[4 * jj + 1] = v.y; qr[4 * jj + 2] = v.z; qr[4 * jj + 3] = v.w;
+  }
+}
+
+template <bool BF16>
+__global__ void __launch_bounds__(kThreads, 2)
+decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int layer, float scale,
+                  float* __restrict__ ws_o, float* __restrict__ ws_ml, int n_splits) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  uint8_t* rings = smem;                                              // kWarps * kRingBytes
+  uint16_t* q_in = reinterpret_cast<uint16_t*>(smem + kWarps * kRingBytes);        // [8][128] input dtype
+  uint16_t* q_h = q_in + 8 * kHeadDim;                                             // [8][128] fp16
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kWarps * kRingBytes + 2 * kQBytes);
+
+  const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int g = lane >> 2, t4 = lane & 3;
+  const int G = dm.n_q_heads / dm.n_kv_heads;
+
+  for (int i = threadIdx.x; i < 8 * kHeadDim; i += kThreads) {
+    const int qi = i / kHeadDim, c = i % kHeadDim;
+    uint16_t raw = 0;
+    if (qi < G) raw = q[(static_cast<long long>(b) * dm.n_q_heads + h * G + qi) * kHeadDim + c];
+    q_in[i] = raw;
+    q_h[i] = BF16 ? __half_as_ushort(__float2half_rn(__uint_as_float(static_cast<uint32_t>(raw) << 16))) : raw;
+  }
+  Pipe pp;
+  pp.ring = smem_u32(rings + warp * kRingBytes);
+  pp.bars = smem_u32(bars + warp * 6);
+  pp.parity = 0u;
+  pp.ok = true;
+  if (lane == 0) {
+    for (int s = 0; s < 6; ++s) mbar_init(pp.bars + 8 * s, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+  }
+  __syncthreads();
+
+  const int group = layer / dm.rs_group;
+  const int32_t* cnt = cv.count + (static_cast<long long>(group) * dm.batch + b) * 4;
+  const int tpc = dm.chunk / kTileTokens;
+  const SplitRange rg = split_range(cnt, cv.capacity, tpc, split, n_splits);
+
+  State st;
+#pragma unroll
+  for (int mt = 0; mt < 8; ++mt)
+#pragma unroll
+    for (int i = 0; i < 4; ++i) st.acc[mt][i] = 0.0f;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) st.oz[i] = 0.0f;
+  st.m[0] = st.m[1] = -INFINITY;
+
+  const float log2e = 1.4426950408889634f;
+  const float c_bias = scale * log2e;
+  const float c_qscore = c_bias * 1048576.0f;      // scores of quantised tiles carry 2^-20
+  const uint8_t* my_ring = rings + warp * kRingBytes;
+
+  uint32_t qraw[16];
+  load_qraw(qraw, q_h, g, t4);
+  uint32_t qc[16];
+
+  // ---- quantised phases
+  {
+    const int first = rg.lo[0] + warp;
+    const int n = first < rg.hi[0] ? (rg.hi[0] - first + kWarps - 1) / kWarps : 0;
+    if (n > 0) {
+      const uint8_t* stream = slot_ptr(cv, dm, 0, layer, b, h, 0);
+      phase_scale<2>(st, true);
+#pragma unroll
+      for (int r = 0; r < 16; ++r) qc[r] = hmul2_u32(qraw[r], half2_pow2(4 - bitpos<2>(r % Fmt<2>::regs)));
+      stream_units<6, 3072, 1>(pp, n, lane,
+          [&](int u, int) { return stream + static_cast<long long>(first + u * kWarps) * 3072; },
+          [&](const uint8_t* tile, int) { process_qtile<2>(tile, st, qc, q_h, c_qscore, c_bias, lane); }, my_ring);
+      phase_scale<2>(st, false);
+    }
+  }
+  {
+    const int first = rg.lo[1] + warp;
+    const int n = first < rg.hi[1] ? (rg.hi[1] - first + kWarps - 1) / kWarps : 0;
+    if (n > 0) {
+      const uint8_t* stream = slot_ptr(cv, dm, 1, layer, b, h, 0);
+      phase_scale<4>(st, true);
+#pragma unroll
+      for (int r = 0; r < 16; ++r) qc[r] = hmul2_u32(qraw[r], half2_pow2(4 - bitpos<4>(r % Fmt<4>::regs)));
+      stream_units<3, 5120, 1>(pp, n, lane,
+          [&](int u, int) { return stream + static_cast<long long>(first + u * kWarps) * 5120; },
+          [&](const uint8_t* tile, int) { process_qtile<4>(tile, st, qc, q_h, c_qscore, c_bias, lane); }, my_ring);
+      phase_scale<4>(st, false);
+    }
+  }
+  {
+    const int first = rg.lo[2] + warp;
+    const int n = first < rg.hi[2] ? (rg.hi[2] - first + kWarps - 1) / kWarps : 0;
+    if (n > 0) {
+      const uint8_t* stream = slot_ptr(cv, dm, 2, layer, b, h, 0);
+      phase_scale<8>(st, true);
+#pragma unroll
+      for (int r = 0; r < 16; ++r) qc[r] = hmul2_u32(qraw[r], half2_pow2(4 - bitpos<8>(r % Fmt<8>::regs)));
+      stream_units<2, 9216, 1>(pp, n, lane,
+          [&](int u, int) { return stream + static_cast<long long>(first + u * kWarps) * 9216; },
+          [&](const uint8_t* tile, int) { process_qtile<8>(tile, st, qc, q_h, c_qscore, c_bias, lane); }, my_ring);
+      phase_scale<8>(st, false);
+    }
+  }
+  // ---- 16-bit tiles: units of 16 tokens (4 KiB of key rows + 4 KiB of value rows)
+  uint32_t qr[16];
+  load_qraw_rawset(qr, q_in, g, t4);
+  {
+    const int first = rg.lo[3] + warp;
+    const int n = first < rg.hi[3] ? (rg.hi[3] - first + kWarps - 1) / kWarps : 0;
+    if (n > 0) {
+      const uint8_t* stream = slot_ptr(cv, dm, 3, layer, b, h, 0);
+      stream_units<2, 8192, 2>(pp, 2 * n, lane,
+          [&](int u, int piece) {
+            return stream + static_cast<long long>(first + (u >> 1) * kWarps) * kRawTileBytes + piece * 8192 + (u & 1) * 4096;
+          },
+          [&](const uint8_t* stg, int) { process_raw16<BF16>(stg, stg + 4096, 16, st, qr, c_bias, lane); }, my_ring);
+    }
+  }
+  // ---- 16-bit tail (last split, warp 0): rows are staged by hand, swizzled, zero padded
+  if (split == n_splits - 1 && warp == 0 && pp.ok) {
+    const int len = cv.tail_len[layer * dm.batch + b];
+    const long long tbase = ((static_cast<long long>(layer) * dm.batch + b) * dm.n_kv_heads + h) * dm.tail_capacity * kHeadDim;
+    uint8_t* stg = rings;    // warp 0's ring; all its bulk copies have completed
+    for (int t0 = 0; t0 < len; t0 += 16) {
+      const int nv = min(16, len - t0);
+      __syncwarp();
+      for (int i = lane; i < 16 * 16; i += 32) {          // 16 rows x 16 units
+        const int row = i >> 4, U = i & 15;
+        const int up = (U & 8) | ((U ^ row) & 7);
+        uint4 kv = make_uint4(0u, 0u, 0u, 0u), vv = kv;
+        if (row < nv) {
+          kv = *reinterpret_cast<const uint4*>(cv.tail_k + tbase + static_cast<long long>(t0 + row) * kHeadDim + 8 * U);
+          vv = *reinterpret_cast<const uint4*>(cv.tail_v + tbase + static_cast<long long>(t0 + row) * kHeadDim + 8 * U);
+        }
+        *reinterpret_cast<uint4*>(stg + row * 256 + up * 16) = kv;
+        *reinterpret_cast<uint4*>(stg + 4096 + row * 256 + up * 16) = vv;
+      }
+      __syncwarp();
+      process_raw16<BF16>(stg, stg + 4096, nv, st, qr, c_bias, lane);
+    }
+  }
+  if (!pp.ok && lane == 0) set_status(cv.status, MOQAE_ERR_TIMEOUT, blockIdx.x, warp);
+
+  // ---- merge: lanes -> warp -> CTA -> split partial
+  __syncthreads();                       // every warp is done with its ring
+  float* red_o = reinterpret_cast<float*>(smem);                 // [kWarps][8 q][128 c]
+  float* red_ml = red_o + kWarps * 8 * kHeadDim;                 // [kWarps][8 q][2]
+#pragma unroll
+  for (int mt = 0; mt < 8; ++mt) {
+    const int cg = mt >> 1;
+    const float z0 = __shfl_sync(0xffffffffu, st.oz[0], cg * 4 + t4);
+    const float z1 = __shfl_sync(0xffffffffu, st.oz[1], cg * 4 + t4);
+    const int ch = 32 * cg + 4 * g + 2 * (mt & 1);
+    float* o0 = red_o + (warp * 8 + 2 * t4) * kHeadDim;
+    float* o1 = o0 + kHeadDim;
+    o0[ch] = st.acc[mt][0] + z0; o1[ch] = st.acc[mt][1] + z1;
+    o0[ch + 1] = st.acc[mt][2] + z0; o1[ch + 1] = st.acc[mt][3] + z1;
+  }
+  if (g == 4) {                          // this lane's oz row holds the sums
+    red_ml[(warp * 8 + 2 * t4) * 2] = st.m[0]; red_ml[(warp * 8 + 2 * t4) * 2 + 1] = st.oz[0];
+    red_ml[(warp * 8 + 2 * t4 + 1) * 2] = st.m[1]; red_ml[(warp * 8 + 2 * t4 + 1) * 2 + 1] = st.oz[1];
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < G * kHeadDim; i += kThreads) {
+    const int qi = i / kHeadDim, c = i % kHeadDim;
+    float m = -INFINITY;
+#pragma unroll
+    for (int wv = 0; wv < kWarps; ++wv) m = fmaxf(m, red_ml[(wv * 8 + qi) * 2]);
+    float l = 0.0f, o = 0.0f;
+#pragma unroll
+    for (int wv = 0; wv < kWarps; ++wv) {
+      const float mw = red_ml[(wv * 8 + qi) * 2];
+      const float f = (mw == -INFINITY) ? 0.0f : ex2f(mw - m);
+      l += red_ml[(wv * 8 + qi) * 2 + 1] * f;
+      o += red_o[(wv * 8 + qi) * kHeadDim + c] * f;
+    }
+    const long long row = (static_cast<long long>(b) * dm.n_q_heads + h * G + qi) * n_splits + split;
+    ws_o[row * kHeadDim + c] = o;
+    // the combine kernel works with natural-log maxima
+    if (c == 0) { ws_ml[row * 2] = m * 0.6931471805599453f; ws_ml[row * 2 + 1] = l; }
+  }
+}
+
+}  // namespace
+
+int decode_mma_ctas_per_sm() { return 2; }
+
+cudaError_t launch_decode_mma(const Dims& dm, const CacheView& cv, const void* q, int layer, float scale,
+                              float* ws_o, float* ws_ml, int n_splits, cudaStream_t st) {
+  const size_t smem = static_cast<size_t>(kWarps) * kRingBytes + 2 * kQBytes + kWarps * 6 * 8;
+  dim3 grid(n_splits, dm.n_kv_heads, dm.batch);
+  cudaError_t e;
+  if (dm.dtype == MOQAE_DTYPE_BF16) {
+    e = cudaFuncSetAttribute(decode_mma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (e != cudaSuccess) return e;
+    decode_mma_kernel<true><<<grid, kThreads, smem, st>>>(dm, cv, static_cast<const uint16_t*>(q), layer, scale, ws_o, ws_ml, n_splits);
+  } else {
+    e = cudaFuncSetAttribute(decode_mma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (e != cudaSuccess) return e;
+    decode_mma_kernel<false><<<grid, kThreads, smem, st>>>(dm, cv, static_cast<const uint16_t*>(q), layer, scale, ws_o, ws_ml, n_splits);
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace moqae
