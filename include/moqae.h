@@ -195,6 +195,29 @@ int moqae_decode_attn(const moqae_config* cfg, const void* q, int32_t layer,
                       int64_t workspace_bytes, void* stream);
 
 /*
+ * (No counterpart in the paper: this entry point exists for deployment reasons only.)
+ * moqae_decode_attn for callers that cannot allocate device memory - for example a plug-in
+ * inside a server whose device memory is entirely owned by the host application, a control
+ * loop that bans allocator calls once it is running, or a binding that can forward pointers
+ * but has no allocator.  Such callers cannot provide the `workspace` of moqae_decode_attn,
+ * so the split partials go to a fixed array inside the library image instead:
+ * moqae_decode_attn_static_max_bytes() bytes (4 MiB), present on every device that loads the
+ * library until the process ends.
+ *   - Arguments, results and error codes are those of moqae_decode_attn without the two
+ *     workspace arguments.  A configuration whose moqae_decode_attn_workspace size exceeds
+ *     the fixed array is refused with MOQAE_ERR_WORKSPACE_TOO_SMALL before anything runs.
+ *   - Nothing is allocated or freed, by this library or through any other one.
+ *   - The first call on each device looks up the array's device address (that device must be
+ *     current, as for every call); make that first call outside any stream capture.
+ *   - All calls on one device share the one array, and it keeps whatever the previous call
+ *     left there.  Every call overwrites the part it reads, so nothing needs clearing, but two
+ *     calls that overlap on the GPU (different streams, no ordering) race on it: order them.
+ */
+int64_t moqae_decode_attn_static_max_bytes(void);
+int moqae_decode_attn_static(const moqae_config* cfg, const void* q, int32_t layer,
+                             const moqae_cache* cache, float* out, float scale, void* stream);
+
+/*
  * Synchronous read of the cache's device status word: *out_status (host) receives MOQAE_OK
  * or the first device-side error recorded since the buffer was zeroed.  Waits for `stream`.
  */

@@ -24,7 +24,8 @@ ERR_WORKSPACE_TOO_SMALL, ERR_CUDA, ERR_TIMEOUT = -5, -6, -7
 
 EXPORTS = ["moqae_version", "moqae_last_cuda_error", "moqae_error_string", "moqae_cache_bytes",
            "moqae_cache_bind", "moqae_route", "moqae_quantize_kv", "moqae_append_kv",
-           "moqae_decode_attn_workspace", "moqae_decode_attn", "moqae_poll_status"]
+           "moqae_decode_attn_workspace", "moqae_decode_attn", "moqae_poll_status",
+           "moqae_decode_attn_static", "moqae_decode_attn_static_max_bytes"]
 
 
 class MoqaeConfig(C.Structure):
@@ -85,9 +86,13 @@ def lib() -> C.CDLL:
         L.moqae_decode_attn.argtypes = [C.POINTER(MoqaeConfig), C.c_void_p, C.c_int32, C.POINTER(MoqaeCache),
                                         C.c_void_p, C.c_float, C.c_void_p, C.c_int64, C.c_void_p]
         L.moqae_poll_status.argtypes = [C.POINTER(MoqaeCache), C.c_void_p, C.POINTER(C.c_int32)]
+        L.moqae_decode_attn_static.argtypes = [C.POINTER(MoqaeConfig), C.c_void_p, C.c_int32,
+                                               C.POINTER(MoqaeCache), C.c_void_p, C.c_float, C.c_void_p]
+        L.moqae_decode_attn_static_max_bytes.argtypes = []
         for name in EXPORTS:
             if name not in ("moqae_error_string",):
                 getattr(L, name).restype = C.c_int
+        L.moqae_decode_attn_static_max_bytes.restype = C.c_int64
         _LIB = L
     return _LIB
 
@@ -227,6 +232,17 @@ def moqae_decode_attn(cfg, q, layer, cache: Cache, out, workspace, scale=0.0):
     _check(lib().moqae_decode_attn(C.byref(cfg), _ptr(q), int(layer), C.byref(cache.view), _ptr(out),
                                    C.c_float(scale), _ptr(workspace), int(workspace.numel() * workspace.element_size()),
                                    _stream()), "moqae_decode_attn")
+
+
+def moqae_decode_attn_static_max_bytes() -> int:
+    return int(lib().moqae_decode_attn_static_max_bytes())
+
+
+def moqae_decode_attn_static(cfg, q, layer, cache: Cache, out, scale=0.0):
+    """moqae_decode_attn without a caller-provided workspace: for callers that cannot allocate
+    device memory, the split partials live in a fixed array inside the library."""
+    _check(lib().moqae_decode_attn_static(C.byref(cfg), _ptr(q), int(layer), C.byref(cache.view), _ptr(out),
+                                          C.c_float(scale), _stream()), "moqae_decode_attn_static")
 
 
 def moqae_poll_status(cache: Cache) -> int:

@@ -74,6 +74,10 @@ int check_cache(const moqae_cache* k, moqae::CacheView* v) {
 
 }  // namespace
 
+namespace moqae {
+void record_cuda_error(cudaError_t e) { g_last_cuda_error = static_cast<int>(e); }
+}  // namespace moqae
+
 #pragma GCC visibility push(default)
 extern "C" {
 

@@ -64,6 +64,9 @@ __device__ __forceinline__ uint8_t* slot_ptr(const CacheView& cv, const Dims& dm
   return cv.pool[w] + idx * slot_bytes;
 }
 
+// Remember `e` as the code moqae_last_cuda_error() reports on this thread.
+void record_cuda_error(cudaError_t e);
+
 // Launchers implemented in the .cu files (host side, return cudaError_t).
 cudaError_t launch_route(const Dims& dm, const CacheView& cv, const void* hidden, int T, const void* W1,
                          const void* W2, const float* W3, const float* bias, int group,
