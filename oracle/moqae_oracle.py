@@ -222,16 +222,19 @@ def assign_slots(bmap: np.ndarray, n_experts: int = N_EXPERTS):
 def quantize_groups(x32: np.ndarray, bits: int):
     """Quantise along the LAST axis, which must have length 32 (one group).
 
-    Canonical sequence, every step one IEEE binary32 operation (round to
-    nearest even) unless a direction is stated:
+    Canonical sequence; "binary32" steps are single IEEE operations rounded to
+    nearest even unless a direction is stated:
         mn, mx   exact minimum / maximum of the group
-        z  = largest fp16 <= mn                      (stored zero)
-        r  = mx - float(z)
-        s  = smallest fp16 >= r / (2^bits - 1)       (stored scale)
+        z  = largest fp16 <= mn, with -0 stored as +0        (stored zero)
+        r  = mx - float(z)                                    (binary32)
+        s  = smallest fp16 >= r / (2^bits - 1)                (binary32 division; stored scale)
         if s == 0: every code is 0
-        inv = 1 / float(s)
-        code = min(2^bits - 1, max(0, rint((x - float(z)) * inv)))
-    rint rounds halves to even.  Returns (scale fp16, zero fp16, codes uint8).
+        inv = 1 / float(s)                                    (binary32)
+        d   = x - float(z)                                    (binary32)
+        code = min(2^bits - 1, max(0, rint(d * inv)))
+    where d * inv is the EXACT product of the two binary32 numbers (it has at most
+    48 significant bits, so float64 holds it exactly) and rint rounds it to the
+    nearest integer, halves to even.  Returns (scale fp16, zero fp16, codes uint8).
     Dequantised value (defined, not computed here): code * s + z.
     """
     x32 = np.asarray(x32, dtype=np.float32)
@@ -240,6 +243,7 @@ def quantize_groups(x32: np.ndarray, bits: int):
     mn = x32.min(axis=-1)
     mx = x32.max(axis=-1)
     z = fp16_round_down(mn)
+    z = np.where(z == 0, np.float16(0.0), z).astype(np.float16)     # -0 -> +0
     zf = z.astype(np.float32)
     r = (mx - zf).astype(np.float32)
     s = fp16_round_up((r / qmax).astype(np.float32))
@@ -247,10 +251,10 @@ def quantize_groups(x32: np.ndarray, bits: int):
     with np.errstate(divide="ignore", invalid="ignore", over="ignore"):
         inv = (np.float32(1.0) / sf).astype(np.float32)
         d = (x32 - zf[..., None]).astype(np.float32)
-        t = (d * inv[..., None]).astype(np.float32)
+        t = d.astype(np.float64) * inv[..., None].astype(np.float64)   # exact
         c = np.rint(t)
-    c = np.minimum(qmax, np.maximum(np.float32(0), c))
-    c = np.where((sf == 0)[..., None], np.float32(0), c)
+    c = np.minimum(np.float64(qmax), np.maximum(0.0, c))
+    c = np.where((sf == 0)[..., None], 0.0, c)
     return s, z, c.astype(np.uint8)
 
 
@@ -284,6 +288,16 @@ def dequantize_tile(t: dict):
 # ----------------------------------------------------------------------------
 # Storage format
 # ----------------------------------------------------------------------------
+# A quantised tile (32 tokens x 128 channels of one kv head, b = 2, 4 or 8 bits)
+# is 1024 + 1024*b bytes:
+#   [   0,  256)  key scale    fp16 x 128
+#   [ 256,  512)  key zero     fp16 x 128
+#   [ 512,  768)  value scale  fp16 x 128   (4 channel groups x 32 tokens)
+#   [ 768, 1024)  value zero   fp16 x 128
+#   [1024, 1024 + 512 b)            key payload
+#   [1024 + 512 b, 1024 + 1024 b)   value payload
+# Inside each part the order is the one in which the decode kernel's 32 lanes
+# consume the data; the functions below state it element by element.
 def tile_bytes(bits: int) -> int:
     """Bytes of one 32-token tile of one kv head (K and V together)."""
     return 16384 if bits == 16 else META_BYTES + 2 * TILE_TOKENS * 16 * bits
@@ -293,29 +307,78 @@ def slot_bytes(bits: int, chunk: int) -> int:
     return (chunk // TILE_TOKENS) * tile_bytes(bits)
 
 
-def v_channel_of_position(p: int) -> int:
-    """Value rows store channels interleaved by channel group: position
-    p = 16*u + 4*cg + k holds channel 32*cg + 4*u + k."""
-    u, cg, k = p >> 4, (p >> 2) & 3, p & 3
-    return 32 * cg + 4 * u + k
+def key_code_location(t: int, c: int, bits: int):
+    """(byte offset inside the key payload, bit offset inside that byte) of the
+    code of token row t, channel c.
+
+    Token t = 16*blk + 8*hh + g, channel c = 32*q + cc.  The 32 codes of one
+    (t, q) form a piece of 4*bits bytes, code cc at bits [bits*cc, bits*cc+bits)
+    of the piece taken as a little-endian bit string.  Pieces live in 16-byte
+    units, unit index:
+        bits 2:  32*blk + 4*g + q,                     hh selects bytes [8hh, 8hh+8)
+        bits 4:  32*(2*blk + hh) + 4*g + q
+        bits 8:  32*(2*(2*blk + hh) + j) + 4*g + q,    j = which 16 bytes of the piece
+    """
+    blk, hh, g = t >> 4, (t >> 3) & 1, t & 7
+    q, cc = c >> 5, c & 31
+    byte_in_piece, bit = (cc * bits) >> 3, (cc * bits) & 7
+    if bits == 2:
+        return (32 * blk + 4 * g + q) * 16 + 8 * hh + byte_in_piece, bit
+    if bits == 4:
+        return (32 * (2 * blk + hh) + 4 * g + q) * 16 + byte_in_piece, bit
+    if bits == 8:
+        return (32 * (2 * (2 * blk + hh) + (byte_in_piece >> 4)) + 4 * g + q) * 16 + (byte_in_piece & 15), bit
+    raise ValueError("bits")
 
 
-def code_location(p: int, t: int, bits: int):
-    """(byte offset inside the payload row, bit offset inside the little-endian
-    32-bit word) of position p of token row t, bits in {2, 4, 8}.
+def value_code_location(t: int, c: int, bits: int):
+    """(byte offset of the little-endian 32-bit word inside the value payload,
+    bit offset inside that word) of the code of token row t, channel c.
 
-    A word holds n = 32/bits consecutive positions; position i of a word sits at
-    bit  bits*(i >> 1) + 16*(i & 1)  (even positions fill the low half-word, odd
-    positions the high half-word).  Words are grouped in 16-byte units; rows of
-    128 bytes or more store unit U at  U xor (t mod 8).
+    Token t = 16*blk + 8*half + 2*t4 + e, channel c = 32*cg + 4*g + r4.
+    Lane ln = 4*g + t4 owns, per blk, the 16 channel rows R = 4*cg + r4; row R
+    sits in word w = R*bits/8 of the lane at slot R mod (8/bits); the code is at
+    bit  bits*slot + 8*half + 16*e.  Words are grouped in 16-byte units per lane:
+    byte offset = ((blk*(bits/2) + w/4)*32 + ln)*16 + (w mod 4)*4.
+    """
+    blk, half, t4, e = t >> 4, (t >> 3) & 1, (t >> 1) & 3, t & 1
+    cg, g, r4 = c >> 5, (c >> 2) & 7, c & 3
+    R = 4 * cg + r4
+    w, slot = (R * bits) >> 3, R % (8 // bits)
+    ln = 4 * g + t4
+    return ((blk * (bits // 2) + (w >> 2)) * 32 + ln) * 16 + (w & 3) * 4, bits * slot + 8 * half + 16 * e
+
+
+def key_meta_index(c: int, bits: int) -> int:
+    """Halfword index of channel c in the key scale (and key zero) array.
+
+    With n = 32/bits codes per 32-bit payload word, channel c = 32*q + cc sits in
+    word j = cc / n at position i = cc mod n.  Positions i and i + n/2 share a
+    register of the decode kernel (low / high half); of the n/2 registers of a
+    word the first n/4 come from the word itself, the others from the word
+    shifted right by 8 bits.  Register number r = j*(n/2) + s*(n/4) + m with
+    i mod (n/2) = s*(n/4) + m; index = ((r/4)*4 + q)*8 + (r mod 4)*2 + (i >= n/2).
     """
     n = 32 // bits
-    j, i = divmod(p, n)
-    bit = bits * (i >> 1) + 16 * (i & 1)
-    unit, w_in_unit = j >> 2, j & 3
-    if 16 * bits >= 128:
-        unit ^= (t & 7)
-    return unit * 16 + w_in_unit * 4, bit
+    q, cc = c >> 5, c & 31
+    j, i = cc // n, cc % n
+    hi, i2 = int(i >= n // 2), i % (n // 2)
+    s_, m = i2 // (n // 4), i2 % (n // 4)
+    r = j * (n // 2) + s_ * (n // 4) + m
+    return ((r >> 2) * 4 + q) * 8 + (r & 3) * 2 + hi
+
+
+def value_scale_index(cg: int, t: int) -> int:
+    """Halfword index of (channel group cg, token t) in the value scale array;
+    t = 16*blk + 8*half + 2*t4 + e."""
+    blk, half, t4, e = t >> 4, (t >> 3) & 1, (t >> 1) & 3, t & 1
+    return ((((blk * 2 + (cg >> 1)) * 4 + t4) * 4 + (cg & 1) * 2 + half) * 2) + e
+
+
+def value_zero_index(cg: int, t: int) -> int:
+    """Halfword index of (channel group cg, token t) in the value zero array."""
+    blk, half, t4, e = t >> 4, (t >> 3) & 1, (t >> 1) & 3, t & 1
+    return ((((blk * 4 + cg) * 4 + t4) * 2 + half) * 2) + e
 
 
 def raw_location(c: int, t: int) -> int:
@@ -330,19 +393,25 @@ _TABLES = {}
 
 
 def _tables(bits: int):
-    """Index tables built from `code_location`, cached (pure bookkeeping)."""
+    """Index tables built from the location functions, cached (pure bookkeeping):
+    32-bit word index and shift of every key / value code, halfword index of
+    every metadata entry."""
     if bits in _TABLES:
         return _TABLES[bits]
-    row_words = 4 * bits
-    word = np.zeros((TILE_TOKENS, HEAD_DIM), dtype=np.int64)
-    shift = np.zeros((TILE_TOKENS, HEAD_DIM), dtype=np.uint32)
+    kw = np.zeros((TILE_TOKENS, HEAD_DIM), dtype=np.int64)
+    ks = np.zeros((TILE_TOKENS, HEAD_DIM), dtype=np.uint32)
+    vw = np.zeros((TILE_TOKENS, HEAD_DIM), dtype=np.int64)
+    vs = np.zeros((TILE_TOKENS, HEAD_DIM), dtype=np.uint32)
     for t in range(TILE_TOKENS):
-        for p in range(HEAD_DIM):
-            byte, bit = code_location(p, t, bits)
-            word[t, p] = t * row_words + byte // 4
-            shift[t, p] = bit
-    vperm = np.array([v_channel_of_position(p) for p in range(HEAD_DIM)], dtype=np.int64)
-    _TABLES[bits] = (word, shift, vperm)
+        for c in range(HEAD_DIM):
+            byte, bit = key_code_location(t, c, bits)
+            kw[t, c], ks[t, c] = byte // 4, 8 * (byte % 4) + bit
+            byte, bit = value_code_location(t, c, bits)
+            vw[t, c], vs[t, c] = byte // 4, bit
+    km = np.array([key_meta_index(c, bits) for c in range(HEAD_DIM)], dtype=np.int64)
+    vsi = np.array([[value_scale_index(cg, t) for t in range(TILE_TOKENS)] for cg in range(4)], dtype=np.int64)
+    vzi = np.array([[value_zero_index(cg, t) for t in range(TILE_TOKENS)] for cg in range(4)], dtype=np.int64)
+    _TABLES[bits] = (kw, ks, vw, vs, km, vsi, vzi)
     return _TABLES[bits]
 
 
@@ -356,47 +425,41 @@ def _raw_table():
     return _TABLES["raw"]
 
 
-def _pack_payload(codes_by_position: np.ndarray, bits: int) -> np.ndarray:
-    word, shift, _ = _tables(bits)
+def _pack_payload(codes: np.ndarray, word: np.ndarray, shift: np.ndarray, bits: int) -> np.ndarray:
     out = np.zeros(TILE_TOKENS * 4 * bits, dtype=np.uint32)
-    np.bitwise_or.at(out, word.ravel(),
-                     (codes_by_position.astype(np.uint32) << shift).ravel())
+    np.bitwise_or.at(out, word.ravel(), (codes.astype(np.uint32) << shift).ravel())
     return out.view(np.uint8)
 
 
-def _unpack_payload(payload_u8: np.ndarray, bits: int) -> np.ndarray:
-    word, shift, _ = _tables(bits)
+def _unpack_payload(payload_u8: np.ndarray, word: np.ndarray, shift: np.ndarray, bits: int) -> np.ndarray:
     w = np.ascontiguousarray(payload_u8).view(np.uint32)
     return ((w[word] >> shift) & np.uint32((1 << bits) - 1)).astype(np.uint8)
 
 
 def pack_tile(t: dict, bits: int) -> np.ndarray:
-    """Quantised tile -> bytes.  Layout: K scale fp16[128] | K zero fp16[128] |
-    V scale fp16[4][32] | V zero fp16[4][32] | K payload (32 rows) | V payload."""
-    _, _, vperm = _tables(bits)
+    """Quantised tile (as returned by `quantize_tile`) -> bytes in the storage format."""
+    kw, ks, vw, vs, km, vsi, vzi = _tables(bits)
     out = np.zeros(tile_bytes(bits), dtype=np.uint8)
-    out[0:256] = t["k_scale"].astype(np.float16).view(np.uint8)
-    out[256:512] = t["k_zero"].astype(np.float16).view(np.uint8)
-    out[512:768] = np.ascontiguousarray(t["v_scale"], dtype=np.float16).view(np.uint8).ravel()
-    out[768:1024] = np.ascontiguousarray(t["v_zero"], dtype=np.float16).view(np.uint8).ravel()
+    h = out[:META_BYTES].view(np.uint16)
+    h[0 + km] = np.asarray(t["k_scale"], dtype=np.float16).view(np.uint16)
+    h[128 + km] = np.asarray(t["k_zero"], dtype=np.float16).view(np.uint16)
+    h[256 + vsi] = np.ascontiguousarray(t["v_scale"], dtype=np.float16).view(np.uint16)
+    h[384 + vzi] = np.ascontiguousarray(t["v_zero"], dtype=np.float16).view(np.uint16)
     pb = TILE_TOKENS * 16 * bits
-    out[1024:1024 + pb] = _pack_payload(t["k_codes"], bits)
-    out[1024 + pb:1024 + 2 * pb] = _pack_payload(t["v_codes"][:, vperm], bits)
+    out[1024:1024 + pb] = _pack_payload(t["k_codes"], kw, ks, bits)
+    out[1024 + pb:1024 + 2 * pb] = _pack_payload(t["v_codes"], vw, vs, bits)
     return out
 
 
 def unpack_tile(buf: np.ndarray, bits: int) -> dict:
-    _, _, vperm = _tables(bits)
+    kw, ks, vw, vs, km, vsi, vzi = _tables(bits)
     buf = np.ascontiguousarray(buf, dtype=np.uint8)
     pb = TILE_TOKENS * 16 * bits
-    vcp = _unpack_payload(buf[1024 + pb:1024 + 2 * pb], bits)
-    vc = np.zeros_like(vcp)
-    vc[:, vperm] = vcp
-    return dict(k_scale=buf[0:256].view(np.float16).copy(),
-                k_zero=buf[256:512].view(np.float16).copy(),
-                v_scale=buf[512:768].view(np.float16).reshape(4, 32).copy(),
-                v_zero=buf[768:1024].view(np.float16).reshape(4, 32).copy(),
-                k_codes=_unpack_payload(buf[1024:1024 + pb], bits), v_codes=vc)
+    h = buf[:META_BYTES].view(np.uint16)
+    return dict(k_scale=h[0 + km].view(np.float16).copy(), k_zero=h[128 + km].view(np.float16).copy(),
+                v_scale=h[256 + vsi].view(np.float16).copy(), v_zero=h[384 + vzi].view(np.float16).copy(),
+                k_codes=_unpack_payload(buf[1024:1024 + pb], kw, ks, bits),
+                v_codes=_unpack_payload(buf[1024 + pb:1024 + 2 * pb], vw, vs, bits))
 
 
 def pack_raw_tile(K_u16: np.ndarray, V_u16: np.ndarray) -> np.ndarray:

@@ -115,9 +115,45 @@ def test_scalar_reimplementation_agrees():
             assert ss == s[r] and zz == z[r]
             inv = np.float32(1) / np.float32(ss)
             for i in range(32):
-                t = np.float32(np.float32(x[r, i] - np.float32(zz)) * inv)
-                code = int(min((1 << bits) - 1, max(0, np.rint(t))))
+                from fractions import Fraction
+                prod = Fraction(float(np.float32(x[r, i] - np.float32(zz)))) * Fraction(float(inv))   # exact
+                lo = prod.numerator // prod.denominator
+                frac = prod - lo
+                code = lo + (1 if frac > Fraction(1, 2) or (frac == Fraction(1, 2) and lo % 2 == 1) else 0)
+                code = int(min((1 << bits) - 1, max(0, code)))
                 assert code == c[r, i]
+
+
+def test_negative_zero_minimum_is_stored_as_plus_zero():
+    x = np.zeros((1, 32), np.float32)
+    x[0, 0] = -0.0
+    x[0, 1] = 1.0
+    for bits in BITS:
+        s_, z, c = O.quantize_groups(x, bits)
+        assert z.view(np.uint16)[0] == 0x0000 and c[0, 1] == (1 << bits) - 1 and c[0, 0] == 0
+
+
+@pytest.mark.parametrize("bits", BITS)
+def test_codes_never_need_the_clamp(bits):
+    """z <= min and s >= (max - z)/(2^b - 1) up to one binary32 rounding, so the rounded
+    product already lies in [0, 2^b - 1]: the clamp of the definition is never active on
+    finite inputs (checked on wide-range random groups and on groups built to sit at the edge)."""
+    rs = RS(40 + bits)
+    qmax = (1 << bits) - 1
+    x = np.clip(rs.randn(4000, 32) * np.exp(rs.randn(4000, 1) * 4), -32000, 32000).astype(np.float16).astype(np.float32)
+    edge = np.zeros((2000, 32), np.float32)
+    step = np.clip(np.exp(rs.randn(2000) * 3), 1e-7, 60.0).astype(np.float16).astype(np.float32)
+    edge[:, 1] = step * qmax                   # max exactly qmax steps above the minimum
+    edge[:, 2:] = (rs.randint(0, 2 * qmax + 1, (2000, 30)) * 0.5).astype(np.float32) * step[:, None]
+    for g in (x, edge, -edge):
+        s_, z, c = O.quantize_groups(g, bits)
+        zf, sf = z.astype(np.float32), s_.astype(np.float32)
+        ok = sf > 0
+        inv = (np.float32(1) / sf[ok]).astype(np.float32)
+        d = (g[ok] - zf[ok, None]).astype(np.float32)
+        raw = np.rint(d.astype(np.float64) * inv[:, None].astype(np.float64))
+        assert raw.min() >= 0 and raw.max() <= qmax
+        assert (raw == c[ok]).all()
 
 
 def test_tile_group_orientation():
@@ -149,39 +185,100 @@ def test_pack_round_trip_and_sizes(bits):
         assert (u[k] == t[k]).all(), k
 
 
+def _random_tile(rs, bits):
+    return dict(k_scale=rs.rand(128).astype(np.float16), k_zero=rs.randn(128).astype(np.float16),
+                v_scale=rs.rand(4, 32).astype(np.float16), v_zero=rs.randn(4, 32).astype(np.float16),
+                k_codes=rs.randint(0, 1 << bits, (32, 128)).astype(np.uint8),
+                v_codes=rs.randint(0, 1 << bits, (32, 128)).astype(np.uint8))
+
+
 @pytest.mark.parametrize("bits", BITS)
-def test_pack_bit_positions_independent(bits):
-    """Set one code at a time and find it where the format says it must be, with the
-    location re-derived here from the format's prose rather than from the oracle's tables."""
+def test_pack_layout_seen_from_the_consuming_lanes(bits):
+    """Independent statement of the format: read a packed tile the way the 32 lanes of the
+    decode kernel do (16-byte units per lane, registers = a word, or the word shifted right by
+    8, masked at one code position in both half-words) and find every code and every scale /
+    zero where the tensor-core fragments need it.  Nothing here uses the oracle's location
+    functions."""
     rs = RS(100 + bits)
+    t = _random_tile(rs, bits)
+    blob = O.pack_tile(t, bits)
     n = 32 // bits
-    row_bytes = 16 * bits
-    for _ in range(60):
-        tok, ch = rs.randint(32), rs.randint(128)
-        for which in ("k", "v"):
-            t = dict(k_scale=np.zeros(128, np.float16), k_zero=np.zeros(128, np.float16),
-                     v_scale=np.zeros((4, 32), np.float16), v_zero=np.zeros((4, 32), np.float16),
-                     k_codes=np.zeros((32, 128), np.uint8), v_codes=np.zeros((32, 128), np.uint8))
-            t[which + "_codes"][tok, ch] = (1 << bits) - 1
-            blob = O.pack_tile(t, bits)
-            if which == "k":
-                p = ch
-                base = 1024
-            else:
-                cg, u, k = ch // 32, (ch % 32) // 4, ch % 4      # interleave by channel group
-                p = 16 * u + 4 * cg + k
-                base = 1024 + 32 * row_bytes
-            word, i = p // n, p % n
-            bit = bits * (i // 2) + 16 * (i % 2)
-            unit, win = word // 4, word % 4
-            if row_bytes >= 128:
-                unit ^= tok % 8
-            off = base + tok * row_bytes + unit * 16 + win * 4
-            expect = np.zeros(blob.size, np.uint8)
-            val = ((1 << bits) - 1) << bit
-            for k_ in range(4):
-                expect[off + k_] = (val >> (8 * k_)) & 0xFF
-            assert (blob == expect).all()
+    mask = (1 << bits) - 1
+    hw = blob[:1024].view(np.uint16)
+    kpay = blob[1024:1024 + 512 * bits]
+    vpay = blob[1024 + 512 * bits:]
+
+    def unit(pay, idx):
+        return pay[16 * idx:16 * idx + 16].view(np.uint32)
+
+    for blk in range(2):
+        for g in range(8):
+            for t4 in range(4):
+                lane = 4 * g + t4
+                # ---- key rows 16blk+g (hh = 0) and 16blk+g+8 (hh = 1), channels 32*t4 .. +31
+                for hh in range(2):
+                    tok = 16 * blk + 8 * hh + g
+                    if bits == 2:
+                        words = unit(kpay, 32 * blk + lane)[2 * hh:2 * hh + 2]
+                    elif bits == 4:
+                        words = unit(kpay, 32 * (2 * blk + hh) + lane)
+                    else:
+                        words = np.concatenate([unit(kpay, 32 * (2 * (2 * blk + hh) + j) + lane) for j in range(2)])
+                    assert len(words) == bits
+                    r = 0
+                    for j in range(bits):
+                        for s_ in range(2):
+                            ws = int(words[j]) >> (8 * s_)
+                            for m in range(n // 4):
+                                lo_ch = 32 * t4 + j * n + s_ * (n // 4) + m
+                                hi_ch = lo_ch + n // 2
+                                assert (ws >> (bits * m)) & mask == t["k_codes"][tok, lo_ch]
+                                assert (ws >> (16 + bits * m)) & mask == t["k_codes"][tok, hi_ch]
+                                if blk == 0 and hh == 0 and g == 0:
+                                    # register r of this lane: its scale / zero pair
+                                    base = ((r >> 2) * 4 + t4) * 8 + (r & 3) * 2
+                                    for arr, name in ((hw[0:128], "k_scale"), (hw[128:256], "k_zero")):
+                                        assert arr[base] == t[name][lo_ch].view(np.uint16)
+                                        assert arr[base + 1] == t[name][hi_ch].view(np.uint16)
+                                r += 1
+                    assert r == 16
+                # ---- values: channel rows of this lane, tokens 16blk + 8half + 2t4 + e
+                words = np.concatenate([unit(vpay, (blk * (bits // 2) + u) * 32 + lane) for u in range(bits // 2)])
+                assert len(words) == 2 * bits
+                for w in range(2 * bits):
+                    for slot in range(8 // bits):
+                        R = w * (8 // bits) + slot
+                        ch = 32 * (R >> 2) + 4 * g + (R & 3)
+                        for half in range(2):
+                            ws = int(words[w]) >> (8 * half)
+                            for e in range(2):
+                                tok = 16 * blk + 8 * half + 2 * t4 + e
+                                assert (ws >> (bits * slot + 16 * e)) & mask == t["v_codes"][tok, ch]
+                if g == 0:
+                    for cp in range(2):
+                        base = ((blk * 2 + cp) * 4 + t4) * 8
+                        for k in range(4):
+                            cg, half = 2 * cp + (k >> 1), k & 1
+                            for e in range(2):
+                                tok = 16 * blk + 8 * half + 2 * t4 + e
+                                assert hw[256 + base + 2 * k + e] == t["v_scale"][cg, tok].view(np.uint16)
+                if g < 4:
+                    base = ((blk * 4 + g) * 4 + t4) * 4
+                    for half in range(2):
+                        for e in range(2):
+                            tok = 16 * blk + 8 * half + 2 * t4 + e
+                            assert hw[384 + base + 2 * half + e] == t["v_zero"][g, tok].view(np.uint16)
+
+
+@pytest.mark.parametrize("bits", BITS)
+def test_locations_are_bijections(bits):
+    kb = {O.key_code_location(t, c, bits) for t in range(32) for c in range(128)}
+    vb = {O.value_code_location(t, c, bits) for t in range(32) for c in range(128)}
+    assert len(kb) == len(vb) == 4096
+    assert max(b for b, _ in kb) < 512 * bits and max(b for b, _ in vb) <= 512 * bits - 4
+    assert sorted(O.key_meta_index(c, bits) for c in range(128)) == list(range(128))
+    assert sorted(O.value_scale_index(cg, t) for cg in range(4) for t in range(32)) == list(range(128))
+    assert sorted(O.value_zero_index(cg, t) for cg in range(4) for t in range(32)) == list(range(128))
 
 
 def test_raw_tile_round_trip_and_swizzle():
