@@ -1,204 +1,403 @@
-// Quantise + bit-pack kernels: one warp owns one tile (32 tokens x 128 channels of one kv
-// head), computes the group statistics, the integer codes and the packed words, and stores
-// them into the slot of the tile's chunk.  HBM-bound: 512 B read and 96..512 B written per
-// token and head.
+// Quantise + bit-pack kernels (prefill) and the 16-bit tail writers.
+//
+// quantize_pack_kernel: every warp is an independent tile pipeline.  A tile is 32 tokens x
+// 128 channels of one kv head: 8 KiB of key rows and 8 KiB of value rows, fetched with one
+// 256-byte bulk copy per row into the warp's own shared-memory buffers (mbarrier
+// complete_tx), so the next tile's rows are in flight while the current one is encoded.
+// The encoded tile (metadata + key payload + value payload, 3 / 5 / 9 KiB) is assembled in
+// shared memory in its storage order and leaves with a single bulk store.  16-bit tiles are
+// copied row by row with their 16-byte units swizzled.
+//
+// Arithmetic per element: binary32 subtract of the group's zero, then one fused
+// multiply-add with 1/scale and the constant 1.5 * 2^23: the FMA rounds the exact product
+// to the nearest integer (halves to even) and leaves the code in the low mantissa bits.
+// HBM-bound by design: 512 B read and 96..512 B written per token and head.
 #include "common.cuh"
 
 namespace moqae {
 
 namespace {
 
-constexpr int kWarpsPerBlock = 4;
+constexpr int kQWarps = 4;
+constexpr int kInBytes = 8192;                 // 32 rows x 256 B
+constexpr int kOutBytes = 9216;                // largest quantised tile
+constexpr int kPrmBytes = 1024;                // value groups: [32 tokens][4 groups] (zero, 1/scale)
+constexpr int kWarpSmem = 2 * kInBytes + kOutBytes + kPrmBytes;
+constexpr long long kWaitLimit = 1ll << 22;
+constexpr float kMagic = 12582912.0f;          // 1.5 * 2^23
 
-__device__ __forceinline__ float cvt16(uint32_t u, int dtype) {
-  return load16_as_float(static_cast<uint16_t>(u), dtype);
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, int count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void bulk_store(void* dst, uint32_t src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;\n" ::"l"(dst), "r"(src), "r"(bytes) : "memory");
+  asm volatile("cp.async.bulk.commit_group;\n" ::: "memory");
+}
+__device__ __forceinline__ void bulk_store_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read 0;\n" ::: "memory");
+}
+__device__ __forceinline__ void bulk_store_wait_all() {
+  asm volatile("cp.async.bulk.wait_group 0;\n" ::: "memory");
+}
+__device__ __forceinline__ void fence_async_smem() {
+  asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
+               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+  for (long long i = 0; i < kWaitLimit; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  return false;
 }
 
-// Group parameters from min / max, every step one binary32 operation.
-__device__ __forceinline__ void group_params(float mn, float mx, float qmax, __half& s, __half& z,
-                                             float& zf, float& inv, bool& dead) {
-  z = __float2half_rd(mn);
-  zf = __half2float(z);
+// ---- packed 16-bit min / max (exact: comparisons only) ---------------------------------
+template <bool BF16> __device__ __forceinline__ uint32_t min2(uint32_t a, uint32_t b) {
+  uint32_t d;
+  if (BF16) asm("min.bf16x2 %0, %1, %2;\n" : "=r"(d) : "r"(a), "r"(b));
+  else asm("min.f16x2 %0, %1, %2;\n" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+template <bool BF16> __device__ __forceinline__ uint32_t max2(uint32_t a, uint32_t b) {
+  uint32_t d;
+  if (BF16) asm("max.bf16x2 %0, %1, %2;\n" : "=r"(d) : "r"(a), "r"(b));
+  else asm("max.f16x2 %0, %1, %2;\n" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+template <bool BF16> __device__ __forceinline__ float lo_f(uint32_t w) {
+  if (BF16) return __uint_as_float(w << 16);
+  return __low2float(*reinterpret_cast<const __half2*>(&w));
+}
+template <bool BF16> __device__ __forceinline__ float hi_f(uint32_t w) {
+  if (BF16) return __uint_as_float(w & 0xffff0000u);
+  return __high2float(*reinterpret_cast<const __half2*>(&w));
+}
+
+// Group parameters from min / max.  zf = stored zero as float, inv = 1/scale (0 for a
+// constant group, so that every code comes out 0).
+__device__ __forceinline__ void group_params(float mn, float mx, float qmax, uint16_t& s_bits, uint16_t& z_bits,
+                                             float& zf, float& inv) {
+  uint16_t zb = __half_as_ushort(__float2half_rd(mn));
+  if (zb == 0x8000u) zb = 0;                                   // -0 is stored as +0
+  zf = __half2float(__ushort_as_half(zb));
   const float r = __fsub_rn(mx, zf);
-  s = __float2half_ru(__fdiv_rn(r, qmax));
+  const __half s = __float2half_ru(__fdiv_rn(r, qmax));
   const float sf = __half2float(s);
-  dead = (sf == 0.0f);
-  inv = __frcp_rn(sf);
+  inv = (sf == 0.0f) ? 0.0f : __frcp_rn(sf);
+  s_bits = __half_as_ushort(s);
+  z_bits = zb;
 }
 
-__device__ __forceinline__ uint32_t encode(float x, float zf, float inv, float qmax, bool dead) {
-  float c = rintf(__fmul_rn(__fsub_rn(x, zf), inv));
-  c = fminf(qmax, fmaxf(0.0f, c));
-  return dead ? 0u : static_cast<uint32_t>(c);
+// code + 0x4B400000: the low bits of the result hold rint((x - zf) * inv)
+__device__ __forceinline__ uint32_t encode(float x, float zf, float inv) {
+  return __float_as_uint(__fmaf_rn(__fsub_rn(x, zf), inv, kMagic));
 }
 
-// Partial 32-bit word of the four positions 4*vl .. 4*vl+3 of a row.
+// Four codes of `BITS` bits side by side in the low 4*BITS bits (higher bits: don't care for
+// BITS < 8, exact for BITS == 8).
 template <int BITS>
-__device__ __forceinline__ uint32_t place4(const uint32_t c[4], int vl) {
+__device__ __forceinline__ uint32_t pack4(uint32_t u0, uint32_t u1, uint32_t u2, uint32_t u3) {
+  if (BITS == 8) return __byte_perm(__byte_perm(u0, u1, 0x0040), __byte_perm(u2, u3, 0x0040), 0x5410);
+  return u0 + (u1 << BITS) + (u2 << (2 * BITS)) + (u3 << (3 * BITS));
+}
+
+// halfword index of channel c in the key scale / zero arrays (register order of the decoder)
+template <int BITS> __device__ __forceinline__ int key_meta_index(int c) {
   constexpr int n = 32 / BITS;
-  const int i0 = (4 * vl) & (n - 1);
-  uint32_t w = 0;
-#pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    const int i = i0 + j;
-    w |= c[j] << (BITS * (i >> 1) + 16 * (i & 1));
-  }
-  return w;
+  const int q = c >> 5, cc = c & 31;
+  const int j = cc / n, i = cc % n;
+  const int hi = i >= n / 2 ? 1 : 0, i2 = i % (n / 2);
+  const int s = i2 / (n / 4), m = i2 % (n / 4);
+  const int r = j * (n / 2) + s * (n / 4) + m;
+  return ((r >> 2) * 4 + q) * 8 + (r & 3) * 2 + hi;
 }
 
-// Store one row word: `vl` is the virtual lane (positions 4*vl..4*vl+3), `xor_a/xor_b` the
-// physical-lane distances of the lanes that share a word.
-template <int BITS>
-__device__ __forceinline__ void store_row_word(uint8_t* payload, int t, int vl, uint32_t part, int xor_a,
-                                               int xor_b) {
-  constexpr int lanes_per_word = (32 / BITS) / 4;   // 4, 2, 1
-  if (lanes_per_word >= 2) part |= __shfl_xor_sync(0xffffffffu, part, xor_a);
-  if (lanes_per_word >= 4) part |= __shfl_xor_sync(0xffffffffu, part, xor_b);
-  const int wj = vl / lanes_per_word;
-  int unit = wj >> 2;
-  if (BITS == 8) unit ^= (t & 7);
-  if ((vl % lanes_per_word) == 0)
-    *reinterpret_cast<uint32_t*>(payload + t * 16 * BITS + unit * 16 + (wj & 3) * 4) = part;
-}
-
-template <int BITS>
-__device__ void quantize_tile(const uint16_t* __restrict__ Kg, const uint16_t* __restrict__ Vg,
-                              long long row_stride, uint8_t* __restrict__ tile, int dtype, int lane) {
+// ---- keys: lane owns channels 4*lane .. 4*lane+3 over the tile's 32 tokens --------------
+template <int BITS, bool BF16>
+__device__ __forceinline__ void encode_keys(const uint8_t* __restrict__ in, uint8_t* __restrict__ out, int lane) {
   constexpr float qmax = static_cast<float>((1 << BITS) - 1);
-  uint2 raw[kTileTokens];
-
-  // ---- keys: one group per channel over the 32 tokens; this lane owns channels 4*lane..+3
-#pragma unroll
-  for (int t = 0; t < kTileTokens; ++t)
-    raw[t] = __ldg(reinterpret_cast<const uint2*>(Kg + t * row_stride) + lane);
-  float mn[4], mx[4];
-#pragma unroll
-  for (int j = 0; j < 4; ++j) { mn[j] = INFINITY; mx[j] = -INFINITY; }
-#pragma unroll
-  for (int t = 0; t < kTileTokens; ++t) {
-    const float x0 = cvt16(raw[t].x & 0xffffu, dtype), x1 = cvt16(raw[t].x >> 16, dtype);
-    const float x2 = cvt16(raw[t].y & 0xffffu, dtype), x3 = cvt16(raw[t].y >> 16, dtype);
-    mn[0] = fminf(mn[0], x0); mx[0] = fmaxf(mx[0], x0);
-    mn[1] = fminf(mn[1], x1); mx[1] = fmaxf(mx[1], x1);
-    mn[2] = fminf(mn[2], x2); mx[2] = fmaxf(mx[2], x2);
-    mn[3] = fminf(mn[3], x3); mx[3] = fmaxf(mx[3], x3);
-  }
+  const uint2* rows = reinterpret_cast<const uint2*>(in) + lane;         // row t at rows[32 * t]
+  uint32_t mn01, mn23, mx01, mx23;
   {
-    float zf[4], inv[4];
-    bool dead[4];
-    __half s[4], z[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) group_params(mn[j], mx[j], qmax, s[j], z[j], zf[j], inv[j], dead[j]);
-    uint2 ps, pz;
-    ps.x = __half_as_ushort(s[0]) | (static_cast<uint32_t>(__half_as_ushort(s[1])) << 16);
-    ps.y = __half_as_ushort(s[2]) | (static_cast<uint32_t>(__half_as_ushort(s[3])) << 16);
-    pz.x = __half_as_ushort(z[0]) | (static_cast<uint32_t>(__half_as_ushort(z[1])) << 16);
-    pz.y = __half_as_ushort(z[2]) | (static_cast<uint32_t>(__half_as_ushort(z[3])) << 16);
-    reinterpret_cast<uint2*>(tile)[lane] = ps;
-    reinterpret_cast<uint2*>(tile + 256)[lane] = pz;
-    uint8_t* payload = tile + kMetaBytes;
-#pragma unroll
-    for (int t = 0; t < kTileTokens; ++t) {
-      uint32_t c[4];
-      c[0] = encode(cvt16(raw[t].x & 0xffffu, dtype), zf[0], inv[0], qmax, dead[0]);
-      c[1] = encode(cvt16(raw[t].x >> 16, dtype), zf[1], inv[1], qmax, dead[1]);
-      c[2] = encode(cvt16(raw[t].y & 0xffffu, dtype), zf[2], inv[2], qmax, dead[2]);
-      c[3] = encode(cvt16(raw[t].y >> 16, dtype), zf[3], inv[3], qmax, dead[3]);
-      store_row_word<BITS>(payload, t, lane, place4<BITS>(c, lane), 1, 2);
-    }
+    const uint2 w = rows[0];
+    mn01 = mx01 = w.x; mn23 = mx23 = w.y;
   }
-
-  // ---- values: one group per token over 32 channels = 8 lanes (lane>>3 is the channel group)
 #pragma unroll
-  for (int t = 0; t < kTileTokens; ++t)
-    raw[t] = __ldg(reinterpret_cast<const uint2*>(Vg + t * row_stride) + lane);
-  const int cg = lane >> 3, u = lane & 7;
-  const int vl = 4 * u + cg;                       // value rows are stored channel-group interleaved
-  uint8_t* payload = tile + kMetaBytes + kTileTokens * 16 * BITS;
-  __half keep_s[4], keep_z[4];
+  for (int t = 1; t < kTileTokens; ++t) {
+    const uint2 w = rows[32 * t];
+    mn01 = min2<BF16>(mn01, w.x); mx01 = max2<BF16>(mx01, w.x);
+    mn23 = min2<BF16>(mn23, w.y); mx23 = max2<BF16>(mx23, w.y);
+  }
+  float zf[4], inv[4];
+  uint16_t sb[4], zb[4];
+  group_params(lo_f<BF16>(mn01), lo_f<BF16>(mx01), qmax, sb[0], zb[0], zf[0], inv[0]);
+  group_params(hi_f<BF16>(mn01), hi_f<BF16>(mx01), qmax, sb[1], zb[1], zf[1], inv[1]);
+  group_params(lo_f<BF16>(mn23), lo_f<BF16>(mx23), qmax, sb[2], zb[2], zf[2], inv[2]);
+  group_params(hi_f<BF16>(mn23), hi_f<BF16>(mx23), qmax, sb[3], zb[3], zf[3], inv[3]);
+  uint16_t* meta = reinterpret_cast<uint16_t*>(out);
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const int idx = key_meta_index<BITS>(4 * lane + k);
+    meta[idx] = sb[k];
+    meta[128 + idx] = zb[k];
+  }
+  // payload: this lane's 4 codes of token t are 4*BITS contiguous bits of the (t, quarter) piece
+  uint8_t* pay = out + kMetaBytes;
+  const int q = lane >> 3, l7 = lane & 7;
 #pragma unroll
   for (int t = 0; t < kTileTokens; ++t) {
-    const float x0 = cvt16(raw[t].x & 0xffffu, dtype), x1 = cvt16(raw[t].x >> 16, dtype);
-    const float x2 = cvt16(raw[t].y & 0xffffu, dtype), x3 = cvt16(raw[t].y >> 16, dtype);
-    float lo = fminf(fminf(x0, x1), fminf(x2, x3));
-    float hi = fmaxf(fmaxf(x0, x1), fmaxf(x2, x3));
-#pragma unroll
-    for (int m = 1; m <= 4; m <<= 1) {
-      lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, m));
-      hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, m));
+    const uint2 w = rows[32 * t];
+    const uint32_t p = pack4<BITS>(encode(lo_f<BF16>(w.x), zf[0], inv[0]), encode(hi_f<BF16>(w.x), zf[1], inv[1]),
+                                   encode(lo_f<BF16>(w.y), zf[2], inv[2]), encode(hi_f<BF16>(w.y), zf[3], inv[3]));
+    const int blk = t >> 4, hh = (t >> 3) & 1, g = t & 7;
+    if (BITS == 2) {
+      pay[(32 * blk + 4 * g + q) * 16 + 8 * hh + l7] = static_cast<uint8_t>(p);
+    } else if (BITS == 4) {
+      *reinterpret_cast<uint16_t*>(pay + (32 * (2 * blk + hh) + 4 * g + q) * 16 + 2 * l7) = static_cast<uint16_t>(p);
+    } else {
+      *reinterpret_cast<uint32_t*>(pay + (32 * (2 * (2 * blk + hh) + (l7 >> 2)) + 4 * g + q) * 16 + 4 * (l7 & 3)) = p;
     }
-    __half s, z;
-    float zf, inv;
-    bool dead;
-    group_params(lo, hi, qmax, s, z, zf, inv, dead);
-    if ((t & 7) == u) { keep_s[t >> 3] = s; keep_z[t >> 3] = z; }
-    uint32_t c[4];
-    c[0] = encode(x0, zf, inv, qmax, dead);
-    c[1] = encode(x1, zf, inv, qmax, dead);
-    c[2] = encode(x2, zf, inv, qmax, dead);
-    c[3] = encode(x3, zf, inv, qmax, dead);
-    store_row_word<BITS>(payload, t, vl, place4<BITS>(c, vl), 8, 16);
-  }
-  __half* vs = reinterpret_cast<__half*>(tile + 512) + cg * 32;
-  __half* vz = reinterpret_cast<__half*>(tile + 768) + cg * 32;
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    vs[8 * i + u] = keep_s[i];
-    vz[8 * i + u] = keep_z[i];
   }
 }
 
-// 16-bit tile: rows are copied in the input dtype with 16-byte units swizzled.
-__device__ void copy_raw_tile(const uint16_t* __restrict__ Kg, const uint16_t* __restrict__ Vg,
-                              long long row_stride, uint8_t* __restrict__ tile, int lane) {
-  const int U = lane >> 1;
-#pragma unroll 8
-  for (int t = 0; t < kTileTokens; ++t) {
-    const uint2 k = __ldg(reinterpret_cast<const uint2*>(Kg + t * row_stride) + lane);
-    const uint2 v = __ldg(reinterpret_cast<const uint2*>(Vg + t * row_stride) + lane);
-    const int up = (U & 8) | ((U ^ t) & 7);
-    const int off = t * 256 + up * 16 + (lane & 1) * 8;
-    *reinterpret_cast<uint2*>(tile + off) = k;
-    *reinterpret_cast<uint2*>(tile + 8192 + off) = v;
+// ---- values: groups are 32 channels of one token -----------------------------------------
+template <int BITS, bool BF16>
+__device__ __forceinline__ void encode_values(const uint8_t* __restrict__ in, uint8_t* __restrict__ out,
+                                              float2* __restrict__ prm, int lane) {
+  constexpr float qmax = static_cast<float>((1 << BITS) - 1);
+  uint16_t* meta = reinterpret_cast<uint16_t*>(out);
+  {
+    // statistics: lane = token; its row is read in 16-byte units, rotated inside each channel
+    // group so that neighbouring lanes start on different banks
+    const int t = lane;
+    const uint4* row = reinterpret_cast<const uint4*>(in + t * 256);
+    const int blk = t >> 4, half = (t >> 3) & 1, t4 = (t >> 1) & 3, e = t & 1;
+    float4 pz[2];
+    float* pzf = reinterpret_cast<float*>(pz);
+#pragma unroll
+    for (int cg = 0; cg < 4; ++cg) {
+      uint32_t mn = 0, mx = 0;
+#pragma unroll
+      for (int ii = 0; ii < 4; ++ii) {
+        const uint4 v = row[4 * cg + (ii ^ (t & 3))];
+        const uint32_t a = min2<BF16>(min2<BF16>(v.x, v.y), min2<BF16>(v.z, v.w));
+        const uint32_t b = max2<BF16>(max2<BF16>(v.x, v.y), max2<BF16>(v.z, v.w));
+        mn = ii == 0 ? a : min2<BF16>(mn, a);
+        mx = ii == 0 ? b : max2<BF16>(mx, b);
+      }
+      float zf, inv;
+      uint16_t sb, zb;
+      group_params(fminf(lo_f<BF16>(mn), hi_f<BF16>(mn)), fmaxf(lo_f<BF16>(mx), hi_f<BF16>(mx)), qmax, sb, zb, zf, inv);
+      pzf[2 * cg] = zf;
+      pzf[2 * cg + 1] = inv;
+      meta[256 + ((((blk * 2 + (cg >> 1)) * 4 + t4) * 4 + (cg & 1) * 2 + half) * 2) + e] = sb;
+      meta[384 + ((((blk * 4 + cg) * 4 + t4) * 2 + half) * 2) + e] = zb;
+    }
+    reinterpret_cast<float4*>(prm)[2 * t] = pz[0];
+    reinterpret_cast<float4*>(prm)[2 * t + 1] = pz[1];
+  }
+  __syncwarp();
+  // codes: lane = channels 4*lane .. 4*lane+3 (group p = lane / 8); one word set per 4 tokens
+  const int p = lane >> 3, g = lane & 7;
+  const uint2* rows = reinterpret_cast<const uint2*>(in) + lane;
+  uint8_t* pay = out + kMetaBytes + kTileTokens * 16 * BITS;
+#pragma unroll
+  for (int blk = 0; blk < 2; ++blk) {
+#pragma unroll
+    for (int t4 = 0; t4 < 4; ++t4) {
+      uint32_t u[4][4];                      // [byte position half + 2e][channel]
+#pragma unroll
+      for (int bp = 0; bp < 4; ++bp) {
+        const int t = 16 * blk + 8 * (bp & 1) + 2 * t4 + (bp >> 1);
+        const uint2 w = rows[32 * t];
+        const float2 zi = prm[4 * t + p];
+        u[bp][0] = encode(lo_f<BF16>(w.x), zi.x, zi.y);
+        u[bp][1] = encode(hi_f<BF16>(w.x), zi.x, zi.y);
+        u[bp][2] = encode(lo_f<BF16>(w.y), zi.x, zi.y);
+        u[bp][3] = encode(hi_f<BF16>(w.y), zi.x, zi.y);
+      }
+      const int ln = 4 * g + t4;
+      if (BITS == 2) {
+        uint32_t b[4];
+#pragma unroll
+        for (int bp = 0; bp < 4; ++bp) b[bp] = pack4<2>(u[bp][0], u[bp][1], u[bp][2], u[bp][3]);
+        const uint32_t word = __byte_perm(__byte_perm(b[0], b[1], 0x0040), __byte_perm(b[2], b[3], 0x0040), 0x5410);
+        *reinterpret_cast<uint32_t*>(pay + (blk * 32 + ln) * 16 + p * 4) = word;
+      } else if (BITS == 4) {
+        uint32_t word[2];
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+          uint32_t b[4];
+#pragma unroll
+          for (int bp = 0; bp < 4; ++bp) b[bp] = u[bp][2 * k] + (u[bp][2 * k + 1] << 4);
+          word[k] = __byte_perm(__byte_perm(b[0], b[1], 0x0040), __byte_perm(b[2], b[3], 0x0040), 0x5410);
+        }
+        // words w = 2p, 2p+1 of the lane: unit w/4 = p/2, position 2*(p&1)
+        *reinterpret_cast<uint2*>(pay + ((blk * 2 + (p >> 1)) * 32 + ln) * 16 + (p & 1) * 8) = make_uint2(word[0], word[1]);
+      } else {
+        uint4 word;
+        uint32_t* wp = reinterpret_cast<uint32_t*>(&word);
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          wp[k] = __byte_perm(__byte_perm(u[0][k], u[1][k], 0x0040), __byte_perm(u[2][k], u[3][k], 0x0040), 0x5410);
+        *reinterpret_cast<uint4*>(pay + ((blk * 4 + p) * 32 + ln) * 16) = word;      // words 4p .. 4p+3
+      }
+    }
   }
 }
 
-__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+// 16-bit tile half (keys or values): rows copied in the input dtype, 16-byte units swizzled.
+__device__ __forceinline__ void copy_raw_rows(const uint8_t* __restrict__ in, uint8_t* __restrict__ dst, int lane) {
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    const int idx = i * 32 + lane;
+    const int row = idx >> 4, U = idx & 15;
+    const int up = (U & 8) | ((U ^ row) & 7);
+    *reinterpret_cast<uint4*>(dst + row * 256 + up * 16) = *reinterpret_cast<const uint4*>(in + row * 256 + U * 16);
+  }
+}
+
+struct TileRef {
+  const uint16_t* K;
+  const uint16_t* V;
+  int b, c, j, h;
+};
+
+template <bool BF16>
+__global__ void __launch_bounds__(kQWarps * 32, 2)
 quantize_pack_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ K, const uint16_t* __restrict__ V,
                      int T, int layer, long long n_tiles) {
-  const int lane = threadIdx.x & 31;
-  const long long tile_id = static_cast<long long>(blockIdx.x) * kWarpsPerBlock + (threadIdx.x >> 5);
-  if (tile_id >= n_tiles) return;
+  extern __shared__ __align__(128) uint8_t smem[];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint8_t* bufK = smem + warp * kWarpSmem;
+  uint8_t* bufV = bufK + kInBytes;
+  uint8_t* out = bufV + kInBytes;
+  float2* prm = reinterpret_cast<float2*>(out + kOutBytes);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kQWarps * kWarpSmem) + 2 * warp;
+  const uint32_t barK = smem_u32(bars), barV = smem_u32(bars + 1);
+  if (lane == 0) {
+    mbar_init(barK, 1);
+    mbar_init(barV, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+  }
+  __syncwarp();
+
   const int H = dm.n_kv_heads;
   const int tpc = dm.chunk / kTileTokens;
   const int C = T / dm.chunk;
-  // tile_id = ((b * C + c) * tpc + j) * H + h : heads fastest, so neighbouring warps read
-  // neighbouring 256-byte segments of the same token rows
-  const int h = static_cast<int>(tile_id % H);
-  long long r = tile_id / H;
-  const int j = static_cast<int>(r % tpc);
-  r /= tpc;
-  const int c = static_cast<int>(r % C);
-  const int b = static_cast<int>(r / C);
+  const long long row_stride = static_cast<long long>(H) * kHeadDim;          // elements
+  const long long stride = static_cast<long long>(gridDim.x) * kQWarps;
   const int group = layer / dm.rs_group;
-  const long long tbl = (static_cast<long long>(group) * dm.batch + b) * dm.max_chunks + c;
-  const int w = cv.map[tbl];
-  const int slot = cv.slot[tbl];
-  if (w > 3 || slot < 0 || slot >= cv.capacity[w > 3 ? 0 : w]) {
-    if (lane == 0) set_status(cv.status, MOQAE_ERR_POOL_FULL, w, slot);
-    return;
+
+  auto tile_ref = [&](long long id) {
+    // id = ((b * C + c) * tpc + j) * H + h : heads fastest, so neighbouring warps read
+    // neighbouring 256-byte segments of the same token rows
+    TileRef r;
+    r.h = static_cast<int>(id % H);
+    long long x = id / H;
+    r.j = static_cast<int>(x % tpc);
+    x /= tpc;
+    r.c = static_cast<int>(x % C);
+    r.b = static_cast<int>(x / C);
+    const long long tok0 = static_cast<long long>(r.b) * T + static_cast<long long>(r.c) * dm.chunk + r.j * kTileTokens;
+    r.K = K + tok0 * row_stride + r.h * kHeadDim;
+    r.V = V + tok0 * row_stride + r.h * kHeadDim;
+    return r;
+  };
+  auto fetch = [&](const uint16_t* src, uint8_t* buf, uint32_t bar) {   // one 256-byte row per lane
+    if (lane == 0) mbar_expect_tx(bar, kInBytes);
+    __syncwarp();
+    bulk_load(smem_u32(buf) + lane * 256, src + lane * row_stride, 256, bar);
+  };
+
+  long long id = static_cast<long long>(blockIdx.x) * kQWarps + warp;
+  if (id >= n_tiles) return;
+  TileRef cur = tile_ref(id);
+  fetch(cur.K, bufK, barK);
+  fetch(cur.V, bufV, barV);
+  uint32_t parity = 0;
+  bool store_pending = false;
+  int failed = 0;                             // 1: key rows never arrived, 2: value rows
+
+  for (; id < n_tiles; id += stride) {
+    const long long next = id + stride;
+    TileRef nxt = cur;
+    if (next < n_tiles) nxt = tile_ref(next);
+    const long long tbl = (static_cast<long long>(group) * dm.batch + cur.b) * dm.max_chunks + cur.c;
+    const int w = cv.map[tbl];
+    const int slot = cv.slot[tbl];
+    const bool valid = w <= 3 && slot >= 0 && slot < cv.capacity[w > 3 ? 0 : w];
+    if (!valid && lane == 0) set_status(cv.status, MOQAE_ERR_POOL_FULL, w, slot);
+    uint8_t* tile = nullptr;
+    if (valid) tile = slot_ptr(cv, dm, w, layer, cur.b, cur.h, slot) + static_cast<long long>(cur.j) * tile_bytes_of_expert(w);
+
+    // ---- keys
+    if (!mbar_wait_bounded(barK, parity)) { failed = 1; break; }
+    if (valid) {
+      if (w == 3) {
+        copy_raw_rows(bufK, tile, lane);
+      } else {
+        if (store_pending) {                  // the previous tile's bulk store must have read `out`
+          if (lane == 0) bulk_store_wait_read();
+          __syncwarp();
+          store_pending = false;
+        }
+        if (w == 0) encode_keys<2, BF16>(bufK, out, lane);
+        else if (w == 1) encode_keys<4, BF16>(bufK, out, lane);
+        else encode_keys<8, BF16>(bufK, out, lane);
+      }
+    }
+    __syncwarp();                             // every lane is done reading bufK
+    if (next < n_tiles) fetch(nxt.K, bufK, barK);
+
+    // ---- values
+    if (!mbar_wait_bounded(barV, parity)) { failed = 2; break; }
+    if (valid) {
+      if (w == 3) {
+        copy_raw_rows(bufV, tile + 8192, lane);
+      } else {
+        if (w == 0) encode_values<2, BF16>(bufV, out, prm, lane);
+        else if (w == 1) encode_values<4, BF16>(bufV, out, prm, lane);
+        else encode_values<8, BF16>(bufV, out, prm, lane);
+      }
+    }
+    __syncwarp();
+    if (next < n_tiles) fetch(nxt.V, bufV, barV);
+    if (valid && w != 3) {
+      fence_async_smem();                     // generic-proxy writes to `out` -> visible to the bulk store
+      __syncwarp();
+      if (lane == 0) bulk_store(tile, smem_u32(out), tile_bytes_of_expert(w));
+      store_pending = true;
+    }
+    parity ^= 1u;
+    cur = nxt;
   }
-  const long long row_stride = static_cast<long long>(H) * kHeadDim;
-  const long long tok0 = static_cast<long long>(b) * T + static_cast<long long>(c) * dm.chunk + j * kTileTokens;
-  const uint16_t* Kg = K + tok0 * row_stride + h * kHeadDim;
-  const uint16_t* Vg = V + tok0 * row_stride + h * kHeadDim;
-  uint8_t* tile = slot_ptr(cv, dm, w, layer, b, h, slot) + static_cast<long long>(j) * tile_bytes_of_expert(w);
-  switch (w) {
-    case 0: quantize_tile<2>(Kg, Vg, row_stride, tile, dm.dtype, lane); break;
-    case 1: quantize_tile<4>(Kg, Vg, row_stride, tile, dm.dtype, lane); break;
-    case 2: quantize_tile<8>(Kg, Vg, row_stride, tile, dm.dtype, lane); break;
-    default: copy_raw_tile(Kg, Vg, row_stride, tile, lane); break;
+  if (failed) {
+    // a copy did not land in time: report it, then give the copies still in flight a last
+    // bounded chance to finish before this CTA's shared memory goes away
+    if (lane == 0) set_status(cv.status, MOQAE_ERR_TIMEOUT, blockIdx.x, warp);
+    if (failed == 1) {
+      mbar_wait_bounded(barK, parity);
+      mbar_wait_bounded(barV, parity);
+    } else {
+      if (id + stride < n_tiles) mbar_wait_bounded(barK, parity ^ 1u);   // next tile's key rows
+      mbar_wait_bounded(barV, parity);
+    }
   }
+  if (lane == 0) bulk_store_wait_all();
 }
 
 // Trailing T mod chunk tokens -> tail rows [layer][b][h][t][128]; sets tail_len.
@@ -246,6 +445,16 @@ __global__ void append_kernel(Dims dm, CacheView cv, const uint16_t* __restrict_
   if (threadIdx.x == 0) cv.tail_len[layer * dm.batch + b] = len + 1;
 }
 
+int sm_count() {
+  static int sms = 0;
+  if (sms == 0) {
+    int dev = 0, v = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev);
+    sms = v > 0 ? v : 148;
+  }
+  return sms;
+}
+
 }  // namespace
 
 cudaError_t launch_quantize(const Dims& dm, const CacheView& cv, const void* K, const void* V, int T,
@@ -253,9 +462,24 @@ cudaError_t launch_quantize(const Dims& dm, const CacheView& cv, const void* K, 
   const int C = T / dm.chunk;
   const long long n_tiles = static_cast<long long>(dm.batch) * C * (dm.chunk / kTileTokens) * dm.n_kv_heads;
   if (n_tiles > 0) {
-    const long long blocks = (n_tiles + kWarpsPerBlock - 1) / kWarpsPerBlock;
-    quantize_pack_kernel<<<static_cast<unsigned>(blocks), kWarpsPerBlock * 32, 0, st>>>(
-        dm, cv, static_cast<const uint16_t*>(K), static_cast<const uint16_t*>(V), T, layer, n_tiles);
+    const size_t smem = static_cast<size_t>(kQWarps) * kWarpSmem + kQWarps * 16;
+    const long long want = (n_tiles + kQWarps - 1) / kQWarps;
+    const long long cap = 2ll * sm_count();                    // two resident CTAs per SM, grid-stride
+    const unsigned grid = static_cast<unsigned>(want < cap ? want : cap);
+    cudaError_t e;
+    if (dm.dtype == MOQAE_DTYPE_BF16) {
+      e = cudaFuncSetAttribute(quantize_pack_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+      if (e != cudaSuccess) return e;
+      quantize_pack_kernel<true><<<grid, kQWarps * 32, smem, st>>>(
+          dm, cv, static_cast<const uint16_t*>(K), static_cast<const uint16_t*>(V), T, layer, n_tiles);
+    } else {
+      e = cudaFuncSetAttribute(quantize_pack_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+      if (e != cudaSuccess) return e;
+      quantize_pack_kernel<false><<<grid, kQWarps * 32, smem, st>>>(
+          dm, cv, static_cast<const uint16_t*>(K), static_cast<const uint16_t*>(V), T, layer, n_tiles);
+    }
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
   }
   dim3 g(8, dm.batch);
   tail_copy_kernel<<<g, 256, 0, st>>>(dm, cv, static_cast<const uint16_t*>(K), static_cast<const uint16_t*>(V), T, layer);
