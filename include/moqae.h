@@ -29,17 +29,29 @@
  * Storage format of the cache (what moqae_quantize_kv writes and moqae_decode_attn reads)
  *   tile   = 32 consecutive tokens of one chunk and one kv head.
  *   quantised tile, b in {2, 4, 8} bits, 1024 + 1024*b bytes:
- *       [   0,  256)  key scale   fp16[128]      (one per channel, over the tile's 32 tokens)
- *       [ 256,  512)  key zero    fp16[128]
- *       [ 512,  768)  value scale fp16[4][32]    ([channel group of 32][token])
- *       [ 768, 1024)  value zero  fp16[4][32]
- *       [1024, 1024+512b)         key payload,   32 token rows of 16*b bytes
- *       [1024+512b, 1024+1024b)   value payload, 32 token rows of 16*b bytes
- *     A payload row holds 128 positions of b bits.  Key rows: position p = channel p.  Value
- *     rows: position p = 16*u + 4*cg + k holds channel 32*cg + 4*u + k.  A little-endian 32-bit
- *     word holds n = 32/b consecutive positions; position i of a word sits at bit
- *     b*(i>>1) + 16*(i&1).  Words form 16-byte units; rows of >= 128 bytes (b = 8) store unit
- *     U of token row t at U xor (t mod 8).
+ *       [   0,  256)  key scale    fp16 x 128   (one per channel, over the tile's 32 tokens)
+ *       [ 256,  512)  key zero     fp16 x 128
+ *       [ 512,  768)  value scale  fp16 x 128   (4 channel groups of 32 x 32 tokens)
+ *       [ 768, 1024)  value zero   fp16 x 128
+ *       [1024, 1024+512b)         key payload
+ *       [1024+512b, 1024+1024b)   value payload
+ *     Inside each part the order is the one in which the 32 lanes of the decode kernel consume
+ *     it (lane = 4*g + t4), so that every lane reads whole 16-byte units:
+ *     Key payload.  Token t = 16*blk + 8*hh + g, channel c = 32*q + cc.  The 32 codes of one
+ *       (t, q) form a piece of 4b bytes, code cc at bits [b*cc, b*cc + b) of the piece read as a
+ *       little-endian bit string.  Pieces sit in 16-byte units; unit index
+ *         b = 2:  32*blk + 4*g + q,                   hh selects bytes [8hh, 8hh + 8) of the unit
+ *         b = 4:  32*(2*blk + hh) + 4*g + q
+ *         b = 8:  32*(2*(2*blk + hh) + j) + 4*g + q,  j = which 16 bytes of the piece.
+ *     Value payload.  Token t = 16*blk + 8*half + 2*t4 + e, channel c = 32*cg + 4*g + r4.
+ *       Lane 4*g + t4 owns, per blk, the 16 channel rows R = 4*cg + r4; row R sits in the lane's
+ *       little-endian 32-bit word w = R*b/8 at slot R mod (8/b), its code at bit
+ *       b*slot + 8*half + 16*e.  Word w is at byte ((blk*(b/2) + w/4)*32 + lane)*16 + (w mod 4)*4.
+ *     Key scale / zero.  With n = 32/b codes per payload word, channel c = 32*q + cc is code
+ *       i = cc mod n of word j = cc / n; let i mod (n/2) = s*(n/4) + m and r = j*(n/2) + s*(n/4) + m;
+ *       halfword index = ((r/4)*4 + q)*8 + (r mod 4)*2 + (i >= n/2).
+ *     Value scale of (cg, t): halfword (((blk*2 + cg/2)*4 + t4)*4 + (cg mod 2)*2 + half)*2 + e.
+ *     Value zero  of (cg, t): halfword (((blk*4 + cg)*4 + t4)*2 + half)*2 + e.
  *     Dequantised value = code * scale + zero.
  *   16-bit tile, 16384 bytes: 32 key rows then 32 value rows of 256 bytes in the input dtype;
  *     16-byte unit U of row t is stored at (U & 8) | ((U xor t) & 7).
@@ -162,9 +174,10 @@ int moqae_route(const moqae_config* cfg, const void* hidden, int32_t T, const vo
  *   MOQAE_ERR_POOL_FULL (read it with moqae_poll_status).
  *   Quantiser: group-wise asymmetric min-max, group 32 (keys per channel over the tile's
  *   tokens, values per token over 32 channels); zero = largest fp16 <= min,
- *   scale = smallest fp16 >= (max - zero)/(2^b - 1), code = clamp(rint((x - zero) * (1/scale)))
- *   with every operation a single binary32 operation; inputs must be finite with
- *   |x| < 32752.
+ *   (-0 stored as +0), scale = smallest fp16 >= (max - zero)/(2^b - 1),
+ *   code = rint((x - zero) * (1/scale)): subtraction, division and reciprocal are single
+ *   binary32 operations, the product is rounded once, to the nearest integer (halves to even).
+ *   Inputs must be finite with |x| < 32752.
  */
 int moqae_quantize_kv(const moqae_config* cfg, const void* K, const void* V, int32_t T,
                       int32_t layer, const uint8_t* forced_map, const moqae_cache* cache,

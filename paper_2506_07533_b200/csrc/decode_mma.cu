@@ -5,16 +5,22 @@
 // complete_tx), and it consumes whole tiles from that ring.  Per 32-token tile:
 //
 //   scores   S[t][q] = sum_c code[t][c] * (q[c] s_k[c]) + sum_c q[c] z_k[c]
-//            The codes are never converted: a masked word IS a pair of fp16 subnormals
-//            (code * 4^j * 2^-24), the power of two and the key scale are folded into the
+//            The codes are never converted: a payload word (or the word shifted right by 8)
+//            masked at one code position in both half-words IS a pair of fp16 subnormals
+//            (code * 2^pos * 2^-24), the power of two and the key scale are folded into the
 //            query fragment once per tile, and the product runs on mma.sync m16n8k16
 //            (A = 16 tokens x 16 channels of codes, B = folded queries of the GQA group
 //            padded to 8 columns, fp32 accumulate).  The zero-point term is a second MMA
 //            chain with exact fp16 operands (A = z_k, B = q).
 //   softmax  online, base 2, in registers; the 64x offset keeps p*s_v in fp16 range.
 //   output   out[c][q] = sum_t code[t][c] * (p[t][q] s_v[t][cg]) + sum_t p[t][q] z_v[t][cg]
-//            again with untouched codes as the A operand (A = V^T, 16 channels x 16 tokens),
-//            P transposed in registers with movmatrix, and one extra MMA for the zero term.
+//            again with untouched codes as the A operand (A = V^T, 16 channels x 16 tokens:
+//            the value payload stores, per lane, words of 4 tokens of each channel row it
+//            owns), P transposed in registers with movmatrix, one extra MMA for the zero
+//            term.  Code positions differ only between accumulator rows, so they are undone
+//            once per phase on the accumulators.
+//   The storage format puts every 16-byte unit where the lane that needs it reads it:
+//   all shared-memory reads of a tile are conflict-free 128-bit loads.
 //
 // 16-bit tiles and the 16-bit tail run the same MMAs on the raw values.
 // Every wait on an mbarrier is bounded; on expiry the warp records MOQAE_ERR_TIMEOUT in
@@ -86,12 +92,6 @@ __device__ __forceinline__ uint32_t hmul2_u32(uint32_t a, uint32_t b) {
   asm("mul.rn.f16x2 %0, %1, %2;\n" : "=r"(r) : "r"(a), "r"(b));
   return r;
 }
-// a*b - c in one rounding: with c = round(a*b) this is the exact rounding error of the product
-__device__ __forceinline__ uint32_t hfma2_sub_u32(uint32_t a, uint32_t b, uint32_t c) {
-  uint32_t r;
-  asm("{\n.reg .b32 n;\nneg.f16x2 n, %3;\nfma.rn.f16x2 %0, %1, %2, n;\n}\n" : "=r"(r) : "r"(a), "r"(b), "r"(c));
-  return r;
-}
 __device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
   const __half2 h = __floats2half2_rn(lo, hi);
   return *reinterpret_cast<const uint32_t*>(&h);
@@ -102,18 +102,25 @@ __device__ __forceinline__ uint32_t pack_bf162(float lo, float hi) {
 }
 
 // ---- code extraction: masked words are pairs of fp16 subnormals ------------------------
-template <int BITS> struct Fmt;
-template <> struct Fmt<2> { static constexpr int regs = 8, direct = 5, shift = 10; static constexpr uint32_t mask = 0x00030003u; };
-template <> struct Fmt<4> { static constexpr int regs = 4, direct = 2, shift = 8;  static constexpr uint32_t mask = 0x000F000Fu; };
-template <> struct Fmt<8> { static constexpr int regs = 2, direct = 1, shift = 8;  static constexpr uint32_t mask = 0x00FF00FFu; };
-
-// bit position (inside a half-word) of the code that register m of a word carries
-template <int BITS> __host__ __device__ constexpr int bitpos(int m) {
-  return m < Fmt<BITS>::direct ? BITS * m : BITS * (m - Fmt<BITS>::direct);
+// A 32-bit payload word holds n = 32/BITS codes, code i at bits [BITS*i, BITS*i + BITS).
+// Register (s, m) of a word is ((s ? w >> 8 : w) & (mask << BITS*m)): its low half-word is
+// code s*(n/4) + m, its high half-word code s*(n/4) + m + n/2, both at bit position BITS*m.
+template <int BITS> struct Fmt {
+  static constexpr int n = 32 / BITS;                 // codes per word
+  static constexpr int regs = n / 2;                  // registers per word
+  static constexpr int direct = n / 4;                // of which taken from the unshifted word
+  static constexpr uint32_t mask = ((1u << BITS) - 1u) * 0x00010001u;
+};
+template <int BITS> __device__ __forceinline__ uint32_t ext(uint32_t w, uint32_t wsh, int s, int m) {
+  return (s ? wsh : w) & (Fmt<BITS>::mask << (BITS * m));
 }
-template <int BITS> __device__ __forceinline__ uint32_t ext(uint32_t w, uint32_t wsh, int m) {
-  return m < Fmt<BITS>::direct ? (w & (Fmt<BITS>::mask << (BITS * m)))
-                               : (wsh & (Fmt<BITS>::mask << (BITS * (m - Fmt<BITS>::direct))));
+// register number r (0..15) of a 32-channel key piece -> word j, shifted?, position m
+template <int BITS> __host__ __device__ constexpr int reg_word(int r) { return r / Fmt<BITS>::regs; }
+template <int BITS> __host__ __device__ constexpr int reg_shifted(int r) { return (r % Fmt<BITS>::regs) / Fmt<BITS>::direct; }
+template <int BITS> __host__ __device__ constexpr int reg_m(int r) { return r % Fmt<BITS>::direct; }
+// channel (inside the piece) of the low half of register r; the high half is n/2 further
+template <int BITS> __host__ __device__ constexpr int reg_channel_lo(int r) {
+  return reg_word<BITS>(r) * Fmt<BITS>::n + reg_shifted<BITS>(r) * Fmt<BITS>::direct + reg_m<BITS>(r);
 }
 // fp16 constant 2^e as a half2 bit pattern (e in the normal range)
 __host__ __device__ constexpr uint32_t half2_pow2(int e) {
@@ -167,89 +174,85 @@ __device__ __forceinline__ void softmax_update(State& st, float x[NV][4]) {
 }
 
 // ---- one quantised tile (32 tokens) from shared memory ---------------------------------
-// qc[r], r = 0..15: fp16 pair q[32*t4 + 2r], q[.. + 1] of query g (zero for g >= G), times the
-// power of two that undoes the bit position of the codes register r multiplies.  qsm: the
-// same pairs unscaled, in shared memory.
+// Lane (g, t4) = (lane / 4, lane % 4).  qb[r], r = 0..15: fp16 pair (q[c_lo(r)], q[c_hi(r)])
+// of query g (zero for g >= G) for the channels 32*t4 + .. that key register r carries;
+// qc[r] = qb[r] times the power of two that undoes the register's bit position.
 template <int BITS>
 __device__ __forceinline__ void process_qtile(const uint8_t* __restrict__ tile, State& st,
-                                              const uint32_t (&qc)[16], const uint16_t* __restrict__ qsm,
+                                              const uint32_t (&qc)[16], const uint32_t (&qb)[16],
                                               float c_score, float c_bias, int lane) {
   using F = Fmt<BITS>;
   const int g = lane >> 2, t4 = lane & 3;
-  constexpr int kRowBytes = 16 * BITS;
   const uint8_t* kpay = tile + kMetaBytes;
-  const uint8_t* vpay = kpay + kTileTokens * kRowBytes;
+  const uint8_t* vpay = kpay + kTileTokens * 16 * BITS;
 
-  // fold the key scales into the query fragment: q*s = hi + lo exactly (two fp16 each)
-  uint32_t qf[16], ql[16];
+  // fold the key scales into the query fragment
+  uint32_t qf[16];
   {
-    const uint4* sp = reinterpret_cast<const uint4*>(tile + 64 * t4);
+    const uint4* sp = reinterpret_cast<const uint4*>(tile) + t4;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      const uint4 s4 = sp[i];
-      const uint32_t sv[4] = {s4.x, s4.y, s4.z, s4.w};
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const int r = 4 * i + j;
-        qf[r] = hmul2_u32(qc[r], sv[j]);
-        ql[r] = hfma2_sub_u32(qc[r], sv[j], qf[r]);
-      }
+      const uint4 s4 = sp[4 * i];
+      qf[4 * i] = hmul2_u32(qc[4 * i], s4.x);
+      qf[4 * i + 1] = hmul2_u32(qc[4 * i + 1], s4.y);
+      qf[4 * i + 2] = hmul2_u32(qc[4 * i + 2], s4.z);
+      qf[4 * i + 3] = hmul2_u32(qc[4 * i + 3], s4.w);
     }
   }
   // zero-point term of the scores: bias[q] = sum_c z_k[c] q[c], exact products (row 0 only)
   float bz[4] = {0.f, 0.f, 0.f, 0.f}, bz2[4] = {0.f, 0.f, 0.f, 0.f};
   {
-    const uint4* zp = reinterpret_cast<const uint4*>(tile + 256 + 64 * t4);
-    const uint4* qp = reinterpret_cast<const uint4*>(qsm + g * kHeadDim + 32 * t4);
+    const uint4* zp = reinterpret_cast<const uint4*>(tile + 256) + t4;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       uint4 z4 = make_uint4(0u, 0u, 0u, 0u);
-      if (g == 0) z4 = zp[i];
-      const uint4 q4 = qp[i];
-      mma16816<false>(bz, z4.x, 0u, z4.y, 0u, q4.x, q4.y);
-      mma16816<false>(bz2, z4.z, 0u, z4.w, 0u, q4.z, q4.w);
+      if (g == 0) z4 = zp[4 * i];
+      mma16816<false>(bz, z4.x, 0u, z4.y, 0u, qb[4 * i], qb[4 * i + 1]);
+      mma16816<false>(bz2, z4.z, 0u, z4.w, 0u, qb[4 * i + 2], qb[4 * i + 3]);
     }
   }
   const float bias0 = __shfl_sync(0xffffffffu, bz[0] + bz2[0], t4) * c_bias;
   const float bias1 = __shfl_sync(0xffffffffu, bz[1] + bz2[1], t4) * c_bias;
 
-  // scores of the two 16-token blocks
+  // scores of the two 16-token blocks: rows g and g + 8 of each
   float x[2][4];
 #pragma unroll
   for (int blk = 0; blk < 2; ++blk) {
+    uint32_t w[2][BITS];           // words of the two row pieces
+    if (BITS == 2) {
+      const uint4 v = *reinterpret_cast<const uint4*>(kpay + (blk * 32 + lane) * 16);
+      w[0][0] = v.x; w[0][1] = v.y; w[1][0] = v.z; w[1][1] = v.w;
+    } else if (BITS == 4) {
+#pragma unroll
+      for (int hh = 0; hh < 2; ++hh) {
+        const uint4 v = *reinterpret_cast<const uint4*>(kpay + ((2 * blk + hh) * 32 + lane) * 16);
+        w[hh][0] = v.x; w[hh][1] = v.y; w[hh][2 % BITS] = v.z; w[hh][3 % BITS] = v.w;
+      }
+    } else {
+#pragma unroll
+      for (int hh = 0; hh < 2; ++hh)
+#pragma unroll
+        for (int j2 = 0; j2 < 2; ++j2) {
+          const uint4 v = *reinterpret_cast<const uint4*>(kpay + (((2 * blk + hh) * 2 + j2) * 32 + lane) * 16);
+          w[hh][(4 * j2) % BITS] = v.x; w[hh][(4 * j2 + 1) % BITS] = v.y;
+          w[hh][(4 * j2 + 2) % BITS] = v.z; w[hh][(4 * j2 + 3) % BITS] = v.w;
+        }
+    }
     uint32_t a[2][16];
 #pragma unroll
-    for (int hh = 0; hh < 2; ++hh) {
-      const int row = 16 * blk + g + 8 * hh;
-      const uint8_t* rp = kpay + row * kRowBytes;
-      uint32_t w[BITS];           // 2, 4 or 8 words per thread and row
-      if (BITS == 2) {
-        const uint2 v = *reinterpret_cast<const uint2*>(rp + 8 * t4);
-        w[0] = v.x; w[1] = v.y;
-      } else if (BITS == 4) {
-        const uint4 v = *reinterpret_cast<const uint4*>(rp + 16 * t4);
-        w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
-      } else {
-#pragma unroll
-        for (int j = 0; j < 2; ++j) {
-          const uint4 v = *reinterpret_cast<const uint4*>(rp + (((2 * t4 + j) ^ (row & 7)) << 4));
-          w[4 * j] = v.x; w[4 * j + 1] = v.y; w[4 * j + 2] = v.z; w[4 * j + 3] = v.w;
-        }
-      }
+    for (int hh = 0; hh < 2; ++hh)
 #pragma unroll
       for (int j = 0; j < BITS; ++j) {
-        const uint32_t wsh = w[j] >> F::shift;
+        const uint32_t wsh = w[hh][j] >> 8;
 #pragma unroll
-        for (int m = 0; m < F::regs; ++m) a[hh][j * F::regs + m] = ext<BITS>(w[j], wsh, m);
+        for (int rr = 0; rr < F::regs; ++rr)
+          a[hh][j * F::regs + rr] = ext<BITS>(w[hh][j], wsh, rr / F::direct, rr % F::direct);
       }
-    }
     float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
     for (int ks = 0; ks < 8; ks += 2) {
       mma16816<false>(s0, a[0][2 * ks], a[1][2 * ks], a[0][2 * ks + 1], a[1][2 * ks + 1], qf[2 * ks], qf[2 * ks + 1]);
       mma16816<false>(s1, a[0][2 * ks + 2], a[1][2 * ks + 2], a[0][2 * ks + 3], a[1][2 * ks + 3], qf[2 * ks + 2], qf[2 * ks + 3]);
-      mma16816<false>(s0, a[0][2 * ks], a[1][2 * ks], a[0][2 * ks + 1], a[1][2 * ks + 1], ql[2 * ks], ql[2 * ks + 1]);
-      mma16816<false>(s1, a[0][2 * ks + 2], a[1][2 * ks + 2], a[0][2 * ks + 3], a[1][2 * ks + 3], ql[2 * ks + 2], ql[2 * ks + 3]);
     }
     x[blk][0] = fmaf(s0[0] + s1[0], c_score, bias0);
     x[blk][1] = fmaf(s0[1] + s1[1], c_score, bias1);
@@ -258,75 +261,72 @@ __device__ __forceinline__ void process_qtile(const uint8_t* __restrict__ tile, 
   }
   softmax_update<2>(st, x);
 
-  const __half* vs = reinterpret_cast<const __half*>(tile + 512);
-  const __half* vz = reinterpret_cast<const __half*>(tile + 768);
 #pragma unroll
   for (int blk = 0; blk < 2; ++blk) {
-    const uint32_t p0 = movmatrix_trans(pack_half2(x[blk][0], x[blk][1]));   // tokens 2t4, 2t4+1 of query g
-    const uint32_t p1 = movmatrix_trans(pack_half2(x[blk][2], x[blk][3]));   // tokens 2t4+8, 2t4+9
-    const int tk = 16 * blk + 2 * t4;
+    const uint32_t p0 = movmatrix_trans(pack_half2(x[blk][0], x[blk][1]));   // tokens 16blk + 2t4, +1 of query g
+    const uint32_t p1 = movmatrix_trans(pack_half2(x[blk][2], x[blk][3]));   // tokens 16blk + 8 + 2t4, +1
     {  // zero-point term: rows = channel groups (lanes g < 4)
       uint32_t z0 = (g == 4) ? 0x3C003C00u : 0u, z1 = z0;      // row 4: ones -> sum of the weights
       if (g < 4) {
-        z0 = *reinterpret_cast<const uint32_t*>(vz + g * 32 + tk);
-        z1 = *reinterpret_cast<const uint32_t*>(vz + g * 32 + tk + 8);
+        const uint2 z = *reinterpret_cast<const uint2*>(tile + 768 + ((blk * 4 + g) * 4 + t4) * 8);
+        z0 = z.x; z1 = z.y;
       }
       mma16816<false>(st.oz, z0, 0u, z1, 0u, p0, p1);
     }
     uint32_t pb[4][2];
 #pragma unroll
-    for (int cg = 0; cg < 4; ++cg) {
-      pb[cg][0] = hmul2_u32(p0, *reinterpret_cast<const uint32_t*>(vs + cg * 32 + tk));
-      pb[cg][1] = hmul2_u32(p1, *reinterpret_cast<const uint32_t*>(vs + cg * 32 + tk + 8));
+    for (int cp = 0; cp < 2; ++cp) {
+      const uint4 sv = *reinterpret_cast<const uint4*>(tile + 512 + ((blk * 2 + cp) * 4 + t4) * 16);
+      pb[2 * cp][0] = hmul2_u32(p0, sv.x); pb[2 * cp][1] = hmul2_u32(p1, sv.y);
+      pb[2 * cp + 1][0] = hmul2_u32(p0, sv.z); pb[2 * cp + 1][1] = hmul2_u32(p1, sv.w);
     }
-    // value codes of token rows tk, tk+1, tk+8, tk+9: this lane's 16 positions 16g..16g+15
-    constexpr int NWV = BITS / 2;
-    uint32_t wv[4][NWV];
+    // value words of this lane: channel rows R = 0..15 (channel 32*(R/4) + 4g + R%4), 4 tokens each
+    constexpr int NW = 2 * BITS;
+    uint32_t wv[NW];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const int row = tk + (i & 1) + 8 * (i >> 1);
-      const uint8_t* rp = vpay + row * kRowBytes;
-      if (BITS == 2) {
-        wv[i][0] = *reinterpret_cast<const uint32_t*>(rp + 4 * g);
-      } else if (BITS == 4) {
-        const uint2 v = *reinterpret_cast<const uint2*>(rp + 8 * g);
-        wv[i][0] = v.x; wv[i][NWV - 1] = v.y;
-      } else {
-        const uint4 v = *reinterpret_cast<const uint4*>(rp + ((g ^ (row & 7)) << 4));
-        wv[i][0] = v.x; wv[i][1 % NWV] = v.y; wv[i][2 % NWV] = v.z; wv[i][3 % NWV] = v.w;
-      }
+    for (int u = 0; u < BITS / 2; ++u) {
+      const uint4 v = *reinterpret_cast<const uint4*>(vpay + ((blk * (BITS / 2) + u) * 32 + lane) * 16);
+      wv[4 * u] = v.x; wv[4 * u + 1] = v.y; wv[4 * u + 2] = v.z; wv[4 * u + 3] = v.w;
     }
 #pragma unroll
-    for (int jv = 0; jv < NWV; ++jv) {
-      const uint32_t lo01 = __byte_perm(wv[0][jv], wv[1][jv], 0x5410), hi01 = __byte_perm(wv[0][jv], wv[1][jv], 0x7632);
-      const uint32_t lo23 = __byte_perm(wv[2][jv], wv[3][jv], 0x5410), hi23 = __byte_perm(wv[2][jv], wv[3][jv], 0x7632);
-      const uint32_t lo01s = lo01 >> F::shift, hi01s = hi01 >> F::shift, lo23s = lo23 >> F::shift, hi23s = hi23 >> F::shift;
-#pragma unroll
-      for (int m = 0; m < F::regs; ++m) {
-        // register m of word jv holds positions jv*n + 2m (low halves) and + 2m + 1 (high halves)
-        constexpr int n = 32 / BITS;
-        const int i16 = jv * n + 2 * m;
-        const int cg = i16 >> 2, hf = (i16 & 3) >> 1;
-        mma16816<false>(st.acc[2 * cg + hf], ext<BITS>(lo01, lo01s, m), ext<BITS>(hi01, hi01s, m),
-                        ext<BITS>(lo23, lo23s, m), ext<BITS>(hi23, hi23s, m), pb[cg][0], pb[cg][1]);
-      }
+    for (int mt = 0; mt < 8; ++mt) {
+      // rows R = 2mt (accumulator row g) and 2mt + 1 (row g + 8)
+      constexpr int per = 8 / BITS;                      // rows per word
+      const int w0 = (2 * mt) / per, sl0 = (2 * mt) % per;
+      const int w1 = (2 * mt + 1) / per, sl1 = (2 * mt + 1) % per;
+      const uint32_t m0 = F::mask << (BITS * sl0), m1 = F::mask << (BITS * sl1);
+      mma16816<false>(st.acc[mt], wv[w0] & m0, wv[w1] & m1, (wv[w0] >> 8) & m0, (wv[w1] >> 8) & m1,
+                      pb[mt >> 1][0], pb[mt >> 1][1]);
     }
   }
 }
 
-// power of two that M-tile mt's accumulator carries inside a quantised phase (code unit / 2^-24)
-template <int BITS> __host__ __device__ constexpr int v_bitpos_of_mtile(int mt) {
-  // i16 = 4*cg + 2*hf with mt = 2*cg + hf;  word jv = i16 / n, register m = (i16 % n) / 2
-  return bitpos<BITS>(((2 * mt) % (32 / BITS)) / 2);
+// power of two that accumulator row `hi` (0: row g, 1: row g + 8) of M-tile mt carries inside
+// a quantised phase, in units of one code (the codes themselves are 2^-24 subnormals)
+template <int BITS> __host__ __device__ constexpr int v_bitpos(int mt, int hi) {
+  return BITS * ((2 * mt + hi) % (8 / BITS));
 }
 template <int BITS>
 __device__ __forceinline__ void phase_scale(State& st, bool enter) {
 #pragma unroll
-  for (int mt = 0; mt < 8; ++mt) {
-    const int e = v_bitpos_of_mtile<BITS>(mt) - 24;          // accumulator = true * 2^e
-    const float f = enter ? exp2f(static_cast<float>(e)) : exp2f(static_cast<float>(-e));
+  for (int mt = 0; mt < 8; ++mt)
 #pragma unroll
-    for (int i = 0; i < 4; ++i) st.acc[mt][i] *= f;
+    for (int i = 0; i < 4; ++i) {
+      const int e = v_bitpos<BITS>(mt, i >> 1) - 24;          // accumulator = true * 2^e
+      st.acc[mt][i] *= enter ? exp2f(static_cast<float>(e)) : exp2f(static_cast<float>(-e));
+    }
+}
+
+// Query fragments of a quantised phase: qb[r] = (q[c_lo(r)], q[c_hi(r)]) of query g as fp16,
+// qc[r] = qb[r] * 2^(4 - bit position of register r).
+template <int BITS>
+__device__ __forceinline__ void load_q_phase(uint32_t (&qb)[16], uint32_t (&qc)[16], const uint16_t* q_h, int g, int t4) {
+  const uint16_t* qrow = q_h + g * kHeadDim + 32 * t4;
+#pragma unroll
+  for (int r = 0; r < 16; ++r) {
+    const int lo = reg_channel_lo<BITS>(r);
+    qb[r] = static_cast<uint32_t>(qrow[lo]) | (static_cast<uint32_t>(qrow[lo + Fmt<BITS>::n / 2]) << 16);
+    qc[r] = hmul2_u32(qb[r], half2_pow2(4 - BITS * reg_m<BITS>(r)));
   }
 }
 
@@ -460,14 +460,6 @@ __device__ __forceinline__ void stream_units(Pipe& pp, int n_units, int lane, Sr
   }
 }
 
-__device__ __forceinline__ void load_qraw(uint32_t (&qraw)[16], const uint16_t* qsrc, int g, int t4) {
-  const uint4* p = reinterpret_cast<const uint4*>(qsrc + g * kHeadDim + 32 * t4);
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const uint4 v = p[i];
-    qraw[4 * i] = v.x; qraw[4 * i + 1] = v.y; qraw[4 * i + 2] = v.z; qraw[4 * i + 3] = v.w;
-  }
-}
 __device__ __forceinline__ void load_qraw_rawset(uint32_t (&qr)[16], const uint16_t* qsrc, int g, int t4) {
 #pragma unroll
   for (int jj = 0; jj < 4; ++jj) {
@@ -529,9 +521,7 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
   const float c_qscore = c_bias * 1048576.0f;      // scores of quantised tiles carry 2^-20
   const uint8_t* my_ring = rings + warp * kRingBytes;
 
-  uint32_t qraw[16];
-  load_qraw(qraw, q_h, g, t4);
-  uint32_t qc[16];
+  uint32_t qb[16], qc[16];
 
   // ---- quantised phases
   {
@@ -540,11 +530,10 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
     if (n > 0) {
       const uint8_t* stream = slot_ptr(cv, dm, 0, layer, b, h, 0);
       phase_scale<2>(st, true);
-#pragma unroll
-      for (int r = 0; r < 16; ++r) qc[r] = hmul2_u32(qraw[r], half2_pow2(4 - bitpos<2>(r % Fmt<2>::regs)));
+      load_q_phase<2>(qb, qc, q_h, g, t4);
       stream_units<6, 3072, 1>(pp, n, lane,
           [&](int u, int) { return stream + static_cast<long long>(first + u * kWarps) * 3072; },
-          [&](const uint8_t* tile, int) { process_qtile<2>(tile, st, qc, q_h, c_qscore, c_bias, lane); }, my_ring);
+          [&](const uint8_t* tile, int) { process_qtile<2>(tile, st, qc, qb, c_qscore, c_bias, lane); }, my_ring);
       phase_scale<2>(st, false);
     }
   }
@@ -554,11 +543,10 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
     if (n > 0) {
       const uint8_t* stream = slot_ptr(cv, dm, 1, layer, b, h, 0);
       phase_scale<4>(st, true);
-#pragma unroll
-      for (int r = 0; r < 16; ++r) qc[r] = hmul2_u32(qraw[r], half2_pow2(4 - bitpos<4>(r % Fmt<4>::regs)));
+      load_q_phase<4>(qb, qc, q_h, g, t4);
       stream_units<3, 5120, 1>(pp, n, lane,
           [&](int u, int) { return stream + static_cast<long long>(first + u * kWarps) * 5120; },
-          [&](const uint8_t* tile, int) { process_qtile<4>(tile, st, qc, q_h, c_qscore, c_bias, lane); }, my_ring);
+          [&](const uint8_t* tile, int) { process_qtile<4>(tile, st, qc, qb, c_qscore, c_bias, lane); }, my_ring);
       phase_scale<4>(st, false);
     }
   }
@@ -568,11 +556,10 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
     if (n > 0) {
       const uint8_t* stream = slot_ptr(cv, dm, 2, layer, b, h, 0);
       phase_scale<8>(st, true);
-#pragma unroll
-      for (int r = 0; r < 16; ++r) qc[r] = hmul2_u32(qraw[r], half2_pow2(4 - bitpos<8>(r % Fmt<8>::regs)));
+      load_q_phase<8>(qb, qc, q_h, g, t4);
       stream_units<2, 9216, 1>(pp, n, lane,
           [&](int u, int) { return stream + static_cast<long long>(first + u * kWarps) * 9216; },
-          [&](const uint8_t* tile, int) { process_qtile<8>(tile, st, qc, q_h, c_qscore, c_bias, lane); }, my_ring);
+          [&](const uint8_t* tile, int) { process_qtile<8>(tile, st, qc, qb, c_qscore, c_bias, lane); }, my_ring);
       phase_scale<8>(st, false);
     }
   }
