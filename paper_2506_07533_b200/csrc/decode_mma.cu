@@ -92,6 +92,12 @@ __device__ __forceinline__ uint32_t hmul2_u32(uint32_t a, uint32_t b) {
   asm("mul.rn.f16x2 %0, %1, %2;\n" : "=r"(r) : "r"(a), "r"(b));
   return r;
 }
+// a*b - c in one rounding: with c = round(a*b) this is the exact rounding error of the product
+__device__ __forceinline__ uint32_t hfma2_sub_u32(uint32_t a, uint32_t b, uint32_t c) {
+  uint32_t r;
+  asm("{\n.reg .b32 n;\nneg.f16x2 n, %3;\nfma.rn.f16x2 %0, %1, %2, n;\n}\n" : "=r"(r) : "r"(a), "r"(b), "r"(c));
+  return r;
+}
 __device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
   const __half2 h = __floats2half2_rn(lo, hi);
   return *reinterpret_cast<const uint32_t*>(&h);
@@ -186,17 +192,20 @@ __device__ __forceinline__ void process_qtile(const uint8_t* __restrict__ tile, 
   const uint8_t* kpay = tile + kMetaBytes;
   const uint8_t* vpay = kpay + kTileTokens * 16 * BITS;
 
-  // fold the key scales into the query fragment
-  uint32_t qf[16];
+  // fold the key scales into the query fragment: q*s = qf + ql exactly (two fp16 each), so the
+  // scores carry no rounding besides the fp32 accumulation
+  uint32_t qf[16], ql[16];
   {
     const uint4* sp = reinterpret_cast<const uint4*>(tile) + t4;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const uint4 s4 = sp[4 * i];
-      qf[4 * i] = hmul2_u32(qc[4 * i], s4.x);
-      qf[4 * i + 1] = hmul2_u32(qc[4 * i + 1], s4.y);
-      qf[4 * i + 2] = hmul2_u32(qc[4 * i + 2], s4.z);
-      qf[4 * i + 3] = hmul2_u32(qc[4 * i + 3], s4.w);
+      const uint32_t sv[4] = {s4.x, s4.y, s4.z, s4.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        qf[4 * i + j] = hmul2_u32(qc[4 * i + j], sv[j]);
+        ql[4 * i + j] = hfma2_sub_u32(qc[4 * i + j], sv[j], qf[4 * i + j]);
+      }
     }
   }
   // zero-point term of the scores: bias[q] = sum_c z_k[c] q[c], exact products (row 0 only)
@@ -253,6 +262,8 @@ __device__ __forceinline__ void process_qtile(const uint8_t* __restrict__ tile, 
     for (int ks = 0; ks < 8; ks += 2) {
       mma16816<false>(s0, a[0][2 * ks], a[1][2 * ks], a[0][2 * ks + 1], a[1][2 * ks + 1], qf[2 * ks], qf[2 * ks + 1]);
       mma16816<false>(s1, a[0][2 * ks + 2], a[1][2 * ks + 2], a[0][2 * ks + 3], a[1][2 * ks + 3], qf[2 * ks + 2], qf[2 * ks + 3]);
+      mma16816<false>(s0, a[0][2 * ks], a[1][2 * ks], a[0][2 * ks + 1], a[1][2 * ks + 1], ql[2 * ks], ql[2 * ks + 1]);
+      mma16816<false>(s1, a[0][2 * ks + 2], a[1][2 * ks + 2], a[0][2 * ks + 3], a[1][2 * ks + 3], ql[2 * ks + 2], ql[2 * ks + 3]);
     }
     x[blk][0] = fmaf(s0[0] + s1[0], c_score, bias0);
     x[blk][1] = fmaf(s0[1] + s1[1], c_score, bias1);

@@ -13,9 +13,9 @@ pytestmark = pytest.mark.gpu
 
 def run_case(B, T, Hkv, chunk, dtype, bmap, seed, n_layers=1, layer=0, rs_group=1, scale=1.0):
     K, V = H.make_kv(B, T, Hkv, dtype, seed)
-    if scale != 1.0:
-        K = (K.float() * scale).to(K.dtype)
-        V = (V.float() * scale).to(V.dtype)
+    if scale != 1.0:                        # the quantiser's input domain is |x| < 32752
+        K = (K.float() * scale).clamp(-32000.0, 32000.0).to(K.dtype)
+        V = (V.float() * scale).clamp(-32000.0, 32000.0).to(V.dtype)
     ocache = O.quantize_kv(synth.to_u16(K), synth.to_u16(V), dtype, chunk, bmap)
     cfg = mq.make_config(n_layers=n_layers, n_q_heads=Hkv, n_kv_heads=Hkv, chunk=chunk, dtype=dtype,
                          d_in=64, max_tokens=max(T, chunk), batch=B, rs_group=rs_group)
