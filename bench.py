@@ -14,6 +14,7 @@ time.
 from __future__ import annotations
 
 import argparse
+import dataclasses
 import json
 import os
 import subprocess
@@ -103,7 +104,7 @@ class Job:
 
     N_DISTINCT = 4      # distinct per-layer K/V inputs; layer l reads input l mod 4 (each > L2)
 
-    def __init__(self, wl, device, seed=1234, context=None):
+    def __init__(self, wl, device, seed=1234, context=None, force_map=False):
         import torch
 
         from paper_2506_07533_b200 import binding as mq
@@ -117,7 +118,8 @@ class Job:
         nd = min(self.N_DISTINCT, wl.n_layers)
         self.kv = [synth.keys_values(B, T, Hkv, 128, wl.dtype, seed + 10 * i, device,
                                      outlier_frac=wl.outlier_frac) for i in range(nd)]
-        nh = min(2, wl.n_groups)
+        self.force_map = force_map
+        nh = 0 if force_map else min(2, wl.n_groups)
         self.hidden = [synth.hidden_states(B, T, wl.d_in, wl.chunk, wl.dtype, seed + 100 + i, device)
                        for i in range(nh)]
         self.W1, self.W2, self.W3, self.bias = synth.router_weights(wl.d_in, 4, wl.dtype, seed + 7, device,
@@ -144,7 +146,7 @@ class Job:
         target = np.asarray(wl.mix, dtype=np.float64)
         bias = np.zeros(4)
         ok = False
-        for it in range(60):
+        for it in range(0 if self.force_map else 60):
             self.bias.copy_(torch.tensor(bias, dtype=torch.float32))
             mq.moqae_route(probe_cfg, self.hidden[0], self.T, self.W1, self.W2, self.W3, self.bias, 0, probe)
             cnt = probe.count[0].sum(0).cpu().numpy().astype(np.float64)
@@ -237,7 +239,11 @@ def run_ours(args):
     if world > 1:
         dist.barrier()
     wl = W.WORKLOADS[args.workload]
-    job = Job(wl, device, seed=1234 + rank, context=args.context)
+    if args.layers:
+        wl = dataclasses.replace(wl, n_layers=args.layers)
+    if args.mix:
+        wl = dataclasses.replace(wl, mix=tuple(float(x) for x in args.mix.split(",")))
+    job = Job(wl, device, seed=1234 + rank, context=args.context, force_map=bool(args.mix))
     torch.cuda.synchronize()
 
     def one_step(ev=None):
@@ -283,7 +289,10 @@ def run_ours(args):
     ms_dec = sum(e[2].elapsed_time(e[3]) for e in events) / args.steps
 
     # end to end: inputs start in pinned host memory, result read back, every step
-    e2e = measure_e2e(job, args, torch)
+    if args.e2e_steps > 0:
+        e2e = measure_e2e(job, args, torch)
+    else:
+        e2e = {"ms_dec": float("nan"), "ms_step": float("nan"), "h2d": 0, "d2h": 0, "steps": 0}
 
     times = torch.tensor([total_ms, ms_route, ms_quant, ms_dec, e2e["ms_dec"], e2e["ms_step"]],
                          dtype=torch.float64, device=device)
@@ -352,7 +361,7 @@ def measure_e2e(job, args, torch):
     h_q = job.q.cpu().pin_memory()
     h_out = torch.empty(job.out.shape, dtype=torch.float32).pin_memory()
     d_K, d_V = torch.empty_like(job.kv[0][0]), torch.empty_like(job.kv[0][1])
-    d_h = torch.empty_like(job.hidden[0])
+    d_h = torch.empty_like(job.hidden[0]) if job.hidden else None
     d_q = torch.empty_like(job.q)
     h2d = 0
     ms_dec, ms_step = 0.0, 0.0
@@ -470,6 +479,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg4", choices=["cfg1", "cfg2", "cfg3", "cfg4"])
     ap.add_argument("--context", type=int, default=None, help="override the context length (profiling)")
+    ap.add_argument("--layers", type=int, default=None, help="override the layer count (profiling)")
+    ap.add_argument("--mix", default=None,
+                    help="four comma-separated shares: skip the router and force a seeded multinomial map "
+                         "with this 2/4/8/16-bit mix (e.g. 1,0,0,0 = uniform 2-bit)")
     ap.add_argument("--e2e-steps", type=int, default=1)
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--reference-tokens", type=int, default=32768)
@@ -477,7 +490,7 @@ def main():
     ap.add_argument("--traffic", type=float, default=None,
                     help="dram bytes per decode launch from an ncu capture (recorded in the JSON line)")
     args = ap.parse_args()
-    if args.warmup < 3 and args.impl == "ours" and args.context is None:
+    if args.warmup < 3 and args.impl == "ours" and args.context is None and args.layers is None:
         args.warmup = 3
     if args.impl == "reference":
         run_reference(args)

@@ -4,8 +4,8 @@
 // Softmax attention does not depend on the order of the keys, so a CTA does not walk the
 // chunks in sequence order: for its (sequence, kv head) it walks pool by pool - all 2-bit
 // tiles, then the 4-bit, 8-bit and 16-bit ones, then (last split only) the 16-bit tail.
-// Each (sequence, kv head) is cut into n_splits pieces of equal COST, a tile costing its
-// size in KiB (3, 5, 9, 16), so every CTA streams about the same number of bytes.
+// Each (sequence, kv head) is cut into n_splits pieces, every piece taking the same share
+// of every pool, so all CTAs stream the same bytes AND the same mix of widths.
 // Each CTA writes, per query head of the group, a partial (max, sum, 128 weighted values)
 // (decode_mma.cu); decode_combine_kernel merges the partials with the log-sum-exp rule.
 #include "common.cuh"

@@ -405,28 +405,19 @@ __device__ __forceinline__ void process_raw16(const uint8_t* __restrict__ ks, co
 
 struct SplitRange { int lo[4], hi[4]; };
 
+// Split `split` of n_splits takes the same share of EVERY pool, so all CTAs of a (sequence,
+// kv head) stream the same mix of widths: they finish together whatever a tile of each
+// width costs, and the demand on HBM is even over the launch.
 __device__ __forceinline__ SplitRange split_range(const int32_t* cnt_in, const long long* capacity,
                                                   int tiles_per_chunk, int split, int n_splits) {
-  int cnt[4];   // never walk past a pool's end, whatever the table says
-#pragma unroll
-  for (int w = 0; w < 4; ++w) cnt[w] = static_cast<int>(min(static_cast<long long>(max(cnt_in[w], 0)), capacity[w]));
-  long long base[5];
-  base[0] = 0;
-#pragma unroll
-  for (int w = 0; w < 4; ++w)
-    base[w + 1] = base[w] + static_cast<long long>(cnt[w]) * tiles_per_chunk * tile_cost_of_expert(w);
-  const long long total = base[4];
-  const long long lo_c = total * split / n_splits, hi_c = total * (split + 1) / n_splits;
   SplitRange r;
 #pragma unroll
   for (int w = 0; w < 4; ++w) {
-    const long long cost = tile_cost_of_expert(w);
-    const long long n = static_cast<long long>(cnt[w]) * tiles_per_chunk;
-    long long a = lo_c - base[w], b = hi_c - base[w];
-    a = a <= 0 ? 0 : (a + cost - 1) / cost;
-    b = b <= 0 ? 0 : (b + cost - 1) / cost;
-    r.lo[w] = static_cast<int>(a < n ? a : n);
-    r.hi[w] = static_cast<int>(b < n ? b : n);
+    // never walk past a pool's end, whatever the table says
+    const long long cnt = min(static_cast<long long>(max(cnt_in[w], 0)), capacity[w]);
+    const long long n = cnt * tiles_per_chunk;
+    r.lo[w] = static_cast<int>(n * split / n_splits);
+    r.hi[w] = static_cast<int>(n * (split + 1) / n_splits);
   }
   return r;
 }
@@ -533,10 +524,12 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
   const uint8_t* my_ring = rings + warp * kRingBytes;
 
   uint32_t qb[16], qc[16];
+  // the CTA's tiles, pool after pool, are dealt to its warps round robin: `dealt` tiles so far
+  int dealt = 0;
 
   // ---- quantised phases
   {
-    const int first = rg.lo[0] + warp;
+    const int first = rg.lo[0] + (warp + kWarps - dealt % kWarps) % kWarps;
     const int n = first < rg.hi[0] ? (rg.hi[0] - first + kWarps - 1) / kWarps : 0;
     if (n > 0) {
       const uint8_t* stream = slot_ptr(cv, dm, 0, layer, b, h, 0);
@@ -547,9 +540,10 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
           [&](const uint8_t* tile, int) { process_qtile<2>(tile, st, qc, qb, c_qscore, c_bias, lane); }, my_ring);
       phase_scale<2>(st, false);
     }
+    dealt += rg.hi[0] - rg.lo[0];
   }
   {
-    const int first = rg.lo[1] + warp;
+    const int first = rg.lo[1] + (warp + kWarps - dealt % kWarps) % kWarps;
     const int n = first < rg.hi[1] ? (rg.hi[1] - first + kWarps - 1) / kWarps : 0;
     if (n > 0) {
       const uint8_t* stream = slot_ptr(cv, dm, 1, layer, b, h, 0);
@@ -560,9 +554,10 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
           [&](const uint8_t* tile, int) { process_qtile<4>(tile, st, qc, qb, c_qscore, c_bias, lane); }, my_ring);
       phase_scale<4>(st, false);
     }
+    dealt += rg.hi[1] - rg.lo[1];
   }
   {
-    const int first = rg.lo[2] + warp;
+    const int first = rg.lo[2] + (warp + kWarps - dealt % kWarps) % kWarps;
     const int n = first < rg.hi[2] ? (rg.hi[2] - first + kWarps - 1) / kWarps : 0;
     if (n > 0) {
       const uint8_t* stream = slot_ptr(cv, dm, 2, layer, b, h, 0);
@@ -573,12 +568,13 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
           [&](const uint8_t* tile, int) { process_qtile<8>(tile, st, qc, qb, c_qscore, c_bias, lane); }, my_ring);
       phase_scale<8>(st, false);
     }
+    dealt += rg.hi[2] - rg.lo[2];
   }
   // ---- 16-bit tiles: units of 16 tokens (4 KiB of key rows + 4 KiB of value rows)
   uint32_t qr[16];
   load_qraw_rawset(qr, q_in, g, t4);
   {
-    const int first = rg.lo[3] + warp;
+    const int first = rg.lo[3] + (warp + kWarps - dealt % kWarps) % kWarps;
     const int n = first < rg.hi[3] ? (rg.hi[3] - first + kWarps - 1) / kWarps : 0;
     if (n > 0) {
       const uint8_t* stream = slot_ptr(cv, dm, 3, layer, b, h, 0);
