@@ -49,7 +49,8 @@
  *       b*slot + 8*half + 16*e.  Word w is at byte ((blk*(b/2) + w/4)*32 + lane)*16 + (w mod 4)*4.
  *     Key scale / zero.  With n = 32/b codes per payload word, channel c = 32*q + cc is code
  *       i = cc mod n of word j = cc / n; let i mod (n/2) = s*(n/4) + m and r = j*(n/2) + s*(n/4) + m;
- *       halfword index = ((r/4)*4 + q)*8 + (r mod 4)*2 + (i >= n/2).
+ *       halfword index = ((r/4)*4 + q)*8 + p*2 + (i >= n/2), with p = r mod 4 for the scales and
+ *       p = (0, 2, 1, 3)[r mod 4] for the zeros.
  *     Value scale of (cg, t): halfword (((blk*2 + cg/2)*4 + t4)*4 + (cg mod 2)*2 + half)*2 + e.
  *     Value zero  of (cg, t): halfword (((blk*4 + cg)*4 + t4)*2 + half)*2 + e.
  *     Dequantised value = code * scale + zero.

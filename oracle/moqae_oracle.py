@@ -368,6 +368,15 @@ def key_meta_index(c: int, bits: int) -> int:
     return ((r >> 2) * 4 + q) * 8 + (r & 3) * 2 + hi
 
 
+def key_zero_index(c: int, bits: int) -> int:
+    """Halfword index of channel c in the key zero array: as `key_meta_index`, but
+    inside each group of four registers the registers are stored in the order
+    0, 2, 1, 3 (so that registers r and r + 2 are neighbours)."""
+    i = key_meta_index(c, bits)
+    r4 = (i >> 1) & 3
+    return (i & ~6) | ((0, 2, 1, 3)[r4] << 1)
+
+
 def value_scale_index(cg: int, t: int) -> int:
     """Halfword index of (channel group cg, token t) in the value scale array;
     t = 16*blk + 8*half + 2*t4 + e."""
@@ -409,9 +418,10 @@ def _tables(bits: int):
             byte, bit = value_code_location(t, c, bits)
             vw[t, c], vs[t, c] = byte // 4, bit
     km = np.array([key_meta_index(c, bits) for c in range(HEAD_DIM)], dtype=np.int64)
+    kz = np.array([key_zero_index(c, bits) for c in range(HEAD_DIM)], dtype=np.int64)
     vsi = np.array([[value_scale_index(cg, t) for t in range(TILE_TOKENS)] for cg in range(4)], dtype=np.int64)
     vzi = np.array([[value_zero_index(cg, t) for t in range(TILE_TOKENS)] for cg in range(4)], dtype=np.int64)
-    _TABLES[bits] = (kw, ks, vw, vs, km, vsi, vzi)
+    _TABLES[bits] = (kw, ks, vw, vs, km, kz, vsi, vzi)
     return _TABLES[bits]
 
 
@@ -438,11 +448,11 @@ def _unpack_payload(payload_u8: np.ndarray, word: np.ndarray, shift: np.ndarray,
 
 def pack_tile(t: dict, bits: int) -> np.ndarray:
     """Quantised tile (as returned by `quantize_tile`) -> bytes in the storage format."""
-    kw, ks, vw, vs, km, vsi, vzi = _tables(bits)
+    kw, ks, vw, vs, km, kz, vsi, vzi = _tables(bits)
     out = np.zeros(tile_bytes(bits), dtype=np.uint8)
     h = out[:META_BYTES].view(np.uint16)
     h[0 + km] = np.asarray(t["k_scale"], dtype=np.float16).view(np.uint16)
-    h[128 + km] = np.asarray(t["k_zero"], dtype=np.float16).view(np.uint16)
+    h[128 + kz] = np.asarray(t["k_zero"], dtype=np.float16).view(np.uint16)
     h[256 + vsi] = np.ascontiguousarray(t["v_scale"], dtype=np.float16).view(np.uint16)
     h[384 + vzi] = np.ascontiguousarray(t["v_zero"], dtype=np.float16).view(np.uint16)
     pb = TILE_TOKENS * 16 * bits
@@ -452,11 +462,11 @@ def pack_tile(t: dict, bits: int) -> np.ndarray:
 
 
 def unpack_tile(buf: np.ndarray, bits: int) -> dict:
-    kw, ks, vw, vs, km, vsi, vzi = _tables(bits)
+    kw, ks, vw, vs, km, kz, vsi, vzi = _tables(bits)
     buf = np.ascontiguousarray(buf, dtype=np.uint8)
     pb = TILE_TOKENS * 16 * bits
     h = buf[:META_BYTES].view(np.uint16)
-    return dict(k_scale=h[0 + km].view(np.float16).copy(), k_zero=h[128 + km].view(np.float16).copy(),
+    return dict(k_scale=h[0 + km].view(np.float16).copy(), k_zero=h[128 + kz].view(np.float16).copy(),
                 v_scale=h[256 + vsi].view(np.float16).copy(), v_zero=h[384 + vzi].view(np.float16).copy(),
                 k_codes=_unpack_payload(buf[1024:1024 + pb], kw, ks, bits),
                 v_codes=_unpack_payload(buf[1024 + pb:1024 + 2 * pb], vw, vs, bits))

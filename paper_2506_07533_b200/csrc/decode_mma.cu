@@ -68,11 +68,11 @@ template <bool BF16>
 __device__ __forceinline__ void mma16816(float d[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                          uint32_t b0, uint32_t b1) {
   if (BF16) {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
                  : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
   } else {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
                  : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
   }
@@ -183,7 +183,10 @@ __device__ __forceinline__ void softmax_update(State& st, float x[NV][4]) {
 // Lane (g, t4) = (lane / 4, lane % 4).  qb[r], r = 0..15: fp16 pair (q[c_lo(r)], q[c_hi(r)])
 // of query g (zero for g >= G) for the channels 32*t4 + .. that key register r carries;
 // qc[r] = qb[r] times the power of two that undoes the register's bit position.
-template <int BITS>
+// G4 (query group of at most 4): B columns 4..7 carry the low parts of the folded queries
+// 0..3, so one MMA chain yields both halves of the exact product and the score of query c
+// is column c plus column c + 4; columns 4..7 then simply mirror 0..3 in everything after.
+template <int BITS, bool G4>
 __device__ __forceinline__ void process_qtile(const uint8_t* __restrict__ tile, State& st,
                                               const uint32_t (&qc)[16], const uint32_t (&qb)[16],
                                               float c_score, float c_bias, int lane) {
@@ -192,36 +195,46 @@ __device__ __forceinline__ void process_qtile(const uint8_t* __restrict__ tile, 
   const uint8_t* kpay = tile + kMetaBytes;
   const uint8_t* vpay = kpay + kTileTokens * 16 * BITS;
 
-  // fold the key scales into the query fragment: q*s = qf + ql exactly (two fp16 each), so the
+  // fold the key scales into the query fragment: q*s = hi + lo exactly (two fp16 each), so the
   // scores carry no rounding besides the fp32 accumulation
-  uint32_t qf[16], ql[16];
+  uint32_t qf[16], ql[G4 ? 1 : 16];
   {
     const uint4* sp = reinterpret_cast<const uint4*>(tile) + t4;
+    const uint32_t lo_lane = (G4 && g >= 4) ? 0xffffffffu : 0u;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const uint4 s4 = sp[4 * i];
       const uint32_t sv[4] = {s4.x, s4.y, s4.z, s4.w};
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        qf[4 * i + j] = hmul2_u32(qc[4 * i + j], sv[j]);
-        ql[4 * i + j] = hfma2_sub_u32(qc[4 * i + j], sv[j], qf[4 * i + j]);
+        const uint32_t hi = hmul2_u32(qc[4 * i + j], sv[j]);
+        if (G4) {
+          // lanes of columns 0..3: fma(q, s, -0) = hi; lanes of columns 4..7: fma(q, s, -hi) = lo
+          qf[4 * i + j] = hfma2_sub_u32(qc[4 * i + j], sv[j], hi & lo_lane);
+        } else {
+          qf[4 * i + j] = hi;
+          ql[(4 * i + j) % (G4 ? 1 : 16)] = hfma2_sub_u32(qc[4 * i + j], sv[j], hi);
+        }
       }
     }
   }
-  // zero-point term of the scores: bias[q] = sum_c z_k[c] q[c], exact products (row 0 only)
-  float bz[4] = {0.f, 0.f, 0.f, 0.f}, bz2[4] = {0.f, 0.f, 0.f, 0.f};
+  // zero-point term of the scores: bias[q] = sum_c z_k[c] q[c], exact products.  Here the
+  // queries are the A operand (rows) and the zeros the B operand, the same in every column:
+  // registers 4i, 4i+2 accumulate in row g of `ba`, registers 4i+1, 4i+3 in row g + 8 of `bb`
+  // (the zero array stores each group of four registers in the order 0, 2, 1, 3).
+  float ba[4] = {0.f, 0.f, 0.f, 0.f}, bb[4] = {0.f, 0.f, 0.f, 0.f};
   {
     const uint4* zp = reinterpret_cast<const uint4*>(tile + 256) + t4;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      uint4 z4 = make_uint4(0u, 0u, 0u, 0u);
-      if (g == 0) z4 = zp[4 * i];
-      mma16816<false>(bz, z4.x, 0u, z4.y, 0u, qb[4 * i], qb[4 * i + 1]);
-      mma16816<false>(bz2, z4.z, 0u, z4.w, 0u, qb[4 * i + 2], qb[4 * i + 3]);
+      const uint4 z4 = zp[4 * i];
+      mma16816<false>(ba, qb[4 * i], qb[4 * i + 1], qb[4 * i + 2], qb[4 * i + 3], z4.x, z4.y);
+      mma16816<false>(bb, qb[4 * i], qb[4 * i + 1], qb[4 * i + 2], qb[4 * i + 3], z4.z, z4.w);
     }
   }
-  const float bias0 = __shfl_sync(0xffffffffu, bz[0] + bz2[0], t4) * c_bias;
-  const float bias1 = __shfl_sync(0xffffffffu, bz[1] + bz2[1], t4) * c_bias;
+  const float bq = (ba[0] + bb[2]) * c_bias;                 // query g, whatever the column
+  const float bias0 = __shfl_sync(0xffffffffu, bq, 8 * t4);
+  const float bias1 = __shfl_sync(0xffffffffu, bq, 8 * t4 + 4);
 
   // scores of the two 16-token blocks: rows g and g + 8 of each
   float x[2][4];
@@ -262,13 +275,18 @@ __device__ __forceinline__ void process_qtile(const uint8_t* __restrict__ tile, 
     for (int ks = 0; ks < 8; ks += 2) {
       mma16816<false>(s0, a[0][2 * ks], a[1][2 * ks], a[0][2 * ks + 1], a[1][2 * ks + 1], qf[2 * ks], qf[2 * ks + 1]);
       mma16816<false>(s1, a[0][2 * ks + 2], a[1][2 * ks + 2], a[0][2 * ks + 3], a[1][2 * ks + 3], qf[2 * ks + 2], qf[2 * ks + 3]);
-      mma16816<false>(s0, a[0][2 * ks], a[1][2 * ks], a[0][2 * ks + 1], a[1][2 * ks + 1], ql[2 * ks], ql[2 * ks + 1]);
-      mma16816<false>(s1, a[0][2 * ks + 2], a[1][2 * ks + 2], a[0][2 * ks + 3], a[1][2 * ks + 3], ql[2 * ks + 2], ql[2 * ks + 3]);
+      if (!G4) {
+        constexpr int M = G4 ? 1 : 16;
+        mma16816<false>(s0, a[0][2 * ks], a[1][2 * ks], a[0][2 * ks + 1], a[1][2 * ks + 1], ql[(2 * ks) % M], ql[(2 * ks + 1) % M]);
+        mma16816<false>(s1, a[0][2 * ks + 2], a[1][2 * ks + 2], a[0][2 * ks + 3], a[1][2 * ks + 3], ql[(2 * ks + 2) % M], ql[(2 * ks + 3) % M]);
+      }
     }
-    x[blk][0] = fmaf(s0[0] + s1[0], c_score, bias0);
-    x[blk][1] = fmaf(s0[1] + s1[1], c_score, bias1);
-    x[blk][2] = fmaf(s0[2] + s1[2], c_score, bias0);
-    x[blk][3] = fmaf(s0[3] + s1[3], c_score, bias1);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      float v = s0[i] + s1[i];
+      if (G4) v += __shfl_xor_sync(0xffffffffu, v, 2);       // column c + column c ^ 4
+      x[blk][i] = fmaf(v, c_score, (i & 1) ? bias1 : bias0);
+    }
   }
   softmax_update<2>(st, x);
 
@@ -471,7 +489,7 @@ __device__ __forceinline__ void load_qraw_rawset(uint32_t (&qr)[16], const uint1
   }
 }
 
-template <bool BF16>
+template <bool BF16, bool G4>
 __global__ void __launch_bounds__(kThreads, 2)
 decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int layer, float scale,
                   float* __restrict__ ws_o, float* __restrict__ ws_ml, int n_splits) {
@@ -489,7 +507,8 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
   for (int i = threadIdx.x; i < 8 * kHeadDim; i += kThreads) {
     const int qi = i / kHeadDim, c = i % kHeadDim;
     uint16_t raw = 0;
-    if (qi < G) raw = q[(static_cast<long long>(b) * dm.n_q_heads + h * G + qi) * kHeadDim + c];
+    const int qs = G4 ? (qi & 3) : qi;                        // G4: rows 4..7 mirror rows 0..3
+    if (qs < G) raw = q[(static_cast<long long>(b) * dm.n_q_heads + h * G + qs) * kHeadDim + c];
     q_in[i] = raw;
     q_h[i] = BF16 ? __half_as_ushort(__float2half_rn(__uint_as_float(static_cast<uint32_t>(raw) << 16))) : raw;
   }
@@ -537,7 +556,7 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
       load_q_phase<2>(qb, qc, q_h, g, t4);
       stream_units<6, 3072, 1>(pp, n, lane,
           [&](int u, int) { return stream + static_cast<long long>(first + u * kWarps) * 3072; },
-          [&](const uint8_t* tile, int) { process_qtile<2>(tile, st, qc, qb, c_qscore, c_bias, lane); }, my_ring);
+          [&](const uint8_t* tile, int) { process_qtile<2, G4>(tile, st, qc, qb, c_qscore, c_bias, lane); }, my_ring);
       phase_scale<2>(st, false);
     }
     dealt += rg.hi[0] - rg.lo[0];
@@ -551,7 +570,7 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
       load_q_phase<4>(qb, qc, q_h, g, t4);
       stream_units<3, 5120, 1>(pp, n, lane,
           [&](int u, int) { return stream + static_cast<long long>(first + u * kWarps) * 5120; },
-          [&](const uint8_t* tile, int) { process_qtile<4>(tile, st, qc, qb, c_qscore, c_bias, lane); }, my_ring);
+          [&](const uint8_t* tile, int) { process_qtile<4, G4>(tile, st, qc, qb, c_qscore, c_bias, lane); }, my_ring);
       phase_scale<4>(st, false);
     }
     dealt += rg.hi[1] - rg.lo[1];
@@ -565,7 +584,7 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
       load_q_phase<8>(qb, qc, q_h, g, t4);
       stream_units<2, 9216, 1>(pp, n, lane,
           [&](int u, int) { return stream + static_cast<long long>(first + u * kWarps) * 9216; },
-          [&](const uint8_t* tile, int) { process_qtile<8>(tile, st, qc, qb, c_qscore, c_bias, lane); }, my_ring);
+          [&](const uint8_t* tile, int) { process_qtile<8, G4>(tile, st, qc, qb, c_qscore, c_bias, lane); }, my_ring);
       phase_scale<8>(st, false);
     }
     dealt += rg.hi[2] - rg.lo[2];
@@ -658,16 +677,17 @@ cudaError_t launch_decode_mma(const Dims& dm, const CacheView& cv, const void* q
                               float* ws_o, float* ws_ml, int n_splits, cudaStream_t st) {
   const size_t smem = static_cast<size_t>(kWarps) * kRingBytes + 2 * kQBytes + kWarps * 6 * 8;
   dim3 grid(n_splits, dm.n_kv_heads, dm.batch);
+  const bool g4 = dm.n_q_heads / dm.n_kv_heads <= 4;
+  auto launch = [&](auto kernel) -> cudaError_t {
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (e != cudaSuccess) return e;
+    kernel<<<grid, kThreads, smem, st>>>(dm, cv, static_cast<const uint16_t*>(q), layer, scale, ws_o, ws_ml, n_splits);
+    return cudaSuccess;
+  };
   cudaError_t e;
-  if (dm.dtype == MOQAE_DTYPE_BF16) {
-    e = cudaFuncSetAttribute(decode_mma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-    if (e != cudaSuccess) return e;
-    decode_mma_kernel<true><<<grid, kThreads, smem, st>>>(dm, cv, static_cast<const uint16_t*>(q), layer, scale, ws_o, ws_ml, n_splits);
-  } else {
-    e = cudaFuncSetAttribute(decode_mma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-    if (e != cudaSuccess) return e;
-    decode_mma_kernel<false><<<grid, kThreads, smem, st>>>(dm, cv, static_cast<const uint16_t*>(q), layer, scale, ws_o, ws_ml, n_splits);
-  }
+  if (dm.dtype == MOQAE_DTYPE_BF16) e = g4 ? launch(decode_mma_kernel<true, true>) : launch(decode_mma_kernel<true, false>);
+  else e = g4 ? launch(decode_mma_kernel<false, true>) : launch(decode_mma_kernel<false, false>);
+  if (e != cudaSuccess) return e;
   return cudaGetLastError();
 }
 

@@ -152,7 +152,8 @@ __device__ __forceinline__ void encode_keys(const uint8_t* __restrict__ in, uint
   for (int k = 0; k < 4; ++k) {
     const int idx = key_meta_index<BITS>(4 * lane + k);
     meta[idx] = sb[k];
-    meta[128 + idx] = zb[k];
+    // zeros: inside each group of four registers the order is 0, 2, 1, 3 (bits 1 and 2 of the index swap)
+    meta[128 + ((idx & ~6) | ((idx & 2) << 1) | ((idx & 4) >> 1))] = zb[k];
   }
   // payload: this lane's 4 codes of token t are 4*BITS contiguous bits of the (t, quarter) piece
   uint8_t* pay = out + kMetaBytes;

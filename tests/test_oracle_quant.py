@@ -236,10 +236,14 @@ def test_pack_layout_seen_from_the_consuming_lanes(bits):
                                 assert (ws >> (16 + bits * m)) & mask == t["k_codes"][tok, hi_ch]
                                 if blk == 0 and hh == 0 and g == 0:
                                     # register r of this lane: its scale / zero pair
-                                    base = ((r >> 2) * 4 + t4) * 8 + (r & 3) * 2
-                                    for arr, name in ((hw[0:128], "k_scale"), (hw[128:256], "k_zero")):
-                                        assert arr[base] == t[name][lo_ch].view(np.uint16)
-                                        assert arr[base + 1] == t[name][hi_ch].view(np.uint16)
+                                    # scales: the lane's i-th 16-byte unit holds registers 4i .. 4i+3;
+                                    # zeros: the same unit holds them in the order 4i, 4i+2, 4i+1, 4i+3
+                                    unit_hw = ((r >> 2) * 4 + t4) * 8
+                                    spos, zpos = (r & 3), (0, 2, 1, 3)[r & 3]
+                                    assert hw[unit_hw + 2 * spos] == t["k_scale"][lo_ch].view(np.uint16)
+                                    assert hw[unit_hw + 2 * spos + 1] == t["k_scale"][hi_ch].view(np.uint16)
+                                    assert hw[128 + unit_hw + 2 * zpos] == t["k_zero"][lo_ch].view(np.uint16)
+                                    assert hw[128 + unit_hw + 2 * zpos + 1] == t["k_zero"][hi_ch].view(np.uint16)
                                 r += 1
                     assert r == 16
                 # ---- values: channel rows of this lane, tokens 16blk + 8half + 2t4 + e
@@ -277,6 +281,7 @@ def test_locations_are_bijections(bits):
     assert len(kb) == len(vb) == 4096
     assert max(b for b, _ in kb) < 512 * bits and max(b for b, _ in vb) <= 512 * bits - 4
     assert sorted(O.key_meta_index(c, bits) for c in range(128)) == list(range(128))
+    assert sorted(O.key_zero_index(c, bits) for c in range(128)) == list(range(128))
     assert sorted(O.value_scale_index(cg, t) for cg in range(4) for t in range(32)) == list(range(128))
     assert sorted(O.value_zero_index(cg, t) for cg in range(4) for t in range(32)) == list(range(128))
 
