@@ -1,9 +1,10 @@
 // Quantise + bit-pack kernels (prefill) and the 16-bit tail writers.
 //
 // quantize_pack_kernel: every warp is an independent tile pipeline.  A tile is 32 tokens x
-// 128 channels of one kv head: 8 KiB of key rows and 8 KiB of value rows, fetched with one
-// 256-byte bulk copy per row into the warp's own shared-memory buffers (mbarrier
-// complete_tx), so the next tile's rows are in flight while the current one is encoded.
+// 128 channels of one kv head: 8 KiB of key rows and 8 KiB of value rows, each fetched by ONE
+// tiled TMA copy (a 128 x 32 box of the [batch*T][heads*128] tensor) into the warp's own
+// shared-memory buffers (mbarrier complete_tx), so the next tile's rows are in flight while
+// the current one is encoded.
 // The encoded tile (metadata + key payload + value payload, 3 / 5 / 9 KiB) is assembled in
 // shared memory in its storage order and leaves with a single bulk store.  16-bit tiles are
 // copied row by row with their 16-byte units swizzled.
@@ -12,6 +13,8 @@
 // multiply-add with 1/scale and the constant 1.5 * 2^23: the FMA rounds the exact product
 // to the nearest integer (halves to even) and leaves the code in the low mantissa bits.
 // HBM-bound by design: 512 B read and 96..512 B written per token and head.
+#include <cuda.h>
+
 #include "common.cuh"
 
 namespace moqae {
@@ -35,9 +38,10 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, int count) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n"
-               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+// tiled TMA load of the box whose corner is (x = element column, y = token row)
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];\n"
+               ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
 }
 __device__ __forceinline__ void bulk_store(void* dst, uint32_t src, uint32_t bytes) {
   asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;\n" ::"l"(dst), "r"(src), "r"(bytes) : "memory");
@@ -272,15 +276,15 @@ __device__ __forceinline__ void copy_raw_rows(const uint8_t* __restrict__ in, ui
 }
 
 struct TileRef {
-  const uint16_t* K;
-  const uint16_t* V;
-  int b, c, j, h;
+  int x, y;            // TMA coordinates: column h*128, token row b*T + c*chunk + j*32
+  int b, j, h;
+  int w, slot;         // routed width and slot of the tile's chunk
 };
 
 template <bool BF16>
 __global__ void __launch_bounds__(kQWarps * 32, 2)
-quantize_pack_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ K, const uint16_t* __restrict__ V,
-                     int T, int layer, long long n_tiles) {
+quantize_pack_kernel(Dims dm, CacheView cv, const __grid_constant__ CUtensorMap mapK,
+                     const __grid_constant__ CUtensorMap mapV, int T, int layer, long long n_tiles) {
   extern __shared__ __align__(128) uint8_t smem[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   uint8_t* bufK = smem + warp * kWarpSmem;
@@ -299,9 +303,10 @@ quantize_pack_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ K, cons
   const int H = dm.n_kv_heads;
   const int tpc = dm.chunk / kTileTokens;
   const int C = T / dm.chunk;
-  const long long row_stride = static_cast<long long>(H) * kHeadDim;          // elements
   const long long stride = static_cast<long long>(gridDim.x) * kQWarps;
   const int group = layer / dm.rs_group;
+  const uint8_t* map_g = cv.map + static_cast<long long>(group) * dm.batch * dm.max_chunks;
+  const int32_t* slot_g = cv.slot + static_cast<long long>(group) * dm.batch * dm.max_chunks;
 
   auto tile_ref = [&](long long id) {
     // id = ((b * C + c) * tpc + j) * H + h : heads fastest, so neighbouring warps read
@@ -311,24 +316,27 @@ quantize_pack_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ K, cons
     long long x = id / H;
     r.j = static_cast<int>(x % tpc);
     x /= tpc;
-    r.c = static_cast<int>(x % C);
+    const int c = static_cast<int>(x % C);
     r.b = static_cast<int>(x / C);
-    const long long tok0 = static_cast<long long>(r.b) * T + static_cast<long long>(r.c) * dm.chunk + r.j * kTileTokens;
-    r.K = K + tok0 * row_stride + r.h * kHeadDim;
-    r.V = V + tok0 * row_stride + r.h * kHeadDim;
+    r.x = r.h * kHeadDim;
+    r.y = r.b * T + c * dm.chunk + r.j * kTileTokens;
+    const long long tbl = static_cast<long long>(r.b) * dm.max_chunks + c;
+    r.w = map_g[tbl];                      // loaded one tile ahead of their use
+    r.slot = slot_g[tbl];
     return r;
   };
-  auto fetch = [&](const uint16_t* src, uint8_t* buf, uint32_t bar) {   // one 256-byte row per lane
-    if (lane == 0) mbar_expect_tx(bar, kInBytes);
-    __syncwarp();
-    bulk_load(smem_u32(buf) + lane * 256, src + lane * row_stride, 256, bar);
+  auto fetch = [&](const CUtensorMap* map, const TileRef& r, uint8_t* buf, uint32_t bar) {
+    if (lane == 0) {
+      mbar_expect_tx(bar, kInBytes);
+      tma_load_2d(smem_u32(buf), map, r.x, r.y, bar);
+    }
   };
 
   long long id = static_cast<long long>(blockIdx.x) * kQWarps + warp;
   if (id >= n_tiles) return;
   TileRef cur = tile_ref(id);
-  fetch(cur.K, bufK, barK);
-  fetch(cur.V, bufV, barV);
+  fetch(&mapK, cur, bufK, barK);
+  fetch(&mapV, cur, bufV, barV);
   uint32_t parity = 0;
   bool store_pending = false;
   int failed = 0;                             // 1: key rows never arrived, 2: value rows
@@ -337,13 +345,21 @@ quantize_pack_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ K, cons
     const long long next = id + stride;
     TileRef nxt = cur;
     if (next < n_tiles) nxt = tile_ref(next);
-    const long long tbl = (static_cast<long long>(group) * dm.batch + cur.b) * dm.max_chunks + cur.c;
-    const int w = cv.map[tbl];
-    const int slot = cv.slot[tbl];
-    const bool valid = w <= 3 && slot >= 0 && slot < cv.capacity[w > 3 ? 0 : w];
+    const int w = cur.w, slot = cur.slot;
+    long long cap = 0;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) cap = (w == k) ? cv.capacity[k] : cap;
+    const bool valid = w <= 3 && slot >= 0 && slot < cap;
     if (!valid && lane == 0) set_status(cv.status, MOQAE_ERR_POOL_FULL, w, slot);
     uint8_t* tile = nullptr;
-    if (valid) tile = slot_ptr(cv, dm, w, layer, cur.b, cur.h, slot) + static_cast<long long>(cur.j) * tile_bytes_of_expert(w);
+    if (valid) {
+      const long long tb = tile_bytes_of_expert(w);
+      const long long idx = ((static_cast<long long>(layer) * dm.batch + cur.b) * H + cur.h) * cap + slot;
+      uint8_t* pool = cv.pool[0];
+#pragma unroll
+      for (int k = 1; k < 4; ++k) pool = (w == k) ? cv.pool[k] : pool;
+      tile = pool + (idx * tpc + cur.j) * tb;
+    }
 
     // ---- keys
     if (!mbar_wait_bounded(barK, parity)) { failed = 1; break; }
@@ -362,7 +378,7 @@ quantize_pack_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ K, cons
       }
     }
     __syncwarp();                             // every lane is done reading bufK
-    if (next < n_tiles) fetch(nxt.K, bufK, barK);
+    if (next < n_tiles) fetch(&mapK, nxt, bufK, barK);
 
     // ---- values
     if (!mbar_wait_bounded(barV, parity)) { failed = 2; break; }
@@ -376,7 +392,7 @@ quantize_pack_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ K, cons
       }
     }
     __syncwarp();
-    if (next < n_tiles) fetch(nxt.V, bufV, barV);
+    if (next < n_tiles) fetch(&mapV, nxt, bufV, barV);
     if (valid && w != 3) {
       fence_async_smem();                     // generic-proxy writes to `out` -> visible to the bulk store
       __syncwarp();
@@ -458,11 +474,44 @@ int sm_count() {
 
 }  // namespace
 
+// cuTensorMapEncodeTiled through the runtime's driver entry-point lookup (no link against libcuda)
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess)
+      p = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
+  return fn;
+}
+
+// [rows][cols] 16-bit tensor, boxes of 128 columns x 32 rows (one tile), no swizzle
+static bool make_tile_map(CUtensorMap* m, const void* base, long long rows, long long cols) {
+  EncodeTiledFn enc = encode_tiled_fn();
+  if (!enc) return false;
+  const cuuint64_t gdim[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
+  const cuuint64_t gstride[1] = {static_cast<cuuint64_t>(cols) * 2};
+  const cuuint32_t box[2] = {kHeadDim, kTileTokens};
+  const cuuint32_t estr[2] = {1, 1};
+  return enc(m, CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, const_cast<void*>(base), gdim, gstride, box, estr,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 cudaError_t launch_quantize(const Dims& dm, const CacheView& cv, const void* K, const void* V, int T,
                             int layer, cudaStream_t st) {
   const int C = T / dm.chunk;
   const long long n_tiles = static_cast<long long>(dm.batch) * C * (dm.chunk / kTileTokens) * dm.n_kv_heads;
   if (n_tiles > 0) {
+    CUtensorMap mapK, mapV;
+    const long long rows = static_cast<long long>(dm.batch) * T, cols = static_cast<long long>(dm.n_kv_heads) * kHeadDim;
+    if (!make_tile_map(&mapK, K, rows, cols) || !make_tile_map(&mapV, V, rows, cols)) return cudaErrorNotSupported;
     const size_t smem = static_cast<size_t>(kQWarps) * kWarpSmem + kQWarps * 16;
     const long long want = (n_tiles + kQWarps - 1) / kQWarps;
     const long long cap = 2ll * sm_count();                    // two resident CTAs per SM, grid-stride
@@ -471,13 +520,11 @@ cudaError_t launch_quantize(const Dims& dm, const CacheView& cv, const void* K, 
     if (dm.dtype == MOQAE_DTYPE_BF16) {
       e = cudaFuncSetAttribute(quantize_pack_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
       if (e != cudaSuccess) return e;
-      quantize_pack_kernel<true><<<grid, kQWarps * 32, smem, st>>>(
-          dm, cv, static_cast<const uint16_t*>(K), static_cast<const uint16_t*>(V), T, layer, n_tiles);
+      quantize_pack_kernel<true><<<grid, kQWarps * 32, smem, st>>>(dm, cv, mapK, mapV, T, layer, n_tiles);
     } else {
       e = cudaFuncSetAttribute(quantize_pack_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
       if (e != cudaSuccess) return e;
-      quantize_pack_kernel<false><<<grid, kQWarps * 32, smem, st>>>(
-          dm, cv, static_cast<const uint16_t*>(K), static_cast<const uint16_t*>(V), T, layer, n_tiles);
+      quantize_pack_kernel<false><<<grid, kQWarps * 32, smem, st>>>(dm, cv, mapK, mapV, T, layer, n_tiles);
     }
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
