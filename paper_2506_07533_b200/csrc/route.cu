@@ -1,15 +1,19 @@
 // Chunk router (Section 3.2, Eq. 1 and Eq. 2; Section 3.4 routing freezing).
 //
-// route_score_vote_kernel: a warp scores 16 tokens at a time.  The two first-layer products
-// C*W1 and C*W2 are one skinny GEMM with N = 2*M = 8 output columns, which is exactly the
-// m16n8k16 tensor-core shape: A = 16 token rows x 16 channels straight from global memory,
-// B = the transposed weights staged once per CTA in shared memory, float32 accumulators.
-// The epilogue applies the product, SiLU, W3 and the bias, takes the per-token arg-max and
-// adds the 16 choices to the chunk's histogram with integer atomics (order-independent).
+// route_score_vote_kernel: every warp is an independent stream over 16-token blocks.  The
+// hidden rows arrive through tiled TMA copies (boxes of 64 channels x 16 tokens, 128-byte
+// swizzle, four boxes per pipeline stage) into the warp's own two-stage ring, so 16 KiB per
+// warp are always in flight.  The two first-layer products C*W1 and C*W2 are one skinny GEMM
+// with N = 2*M = 8 output columns, which is exactly the m16n8k16 tensor-core shape: A = 16
+// token rows x 16 channels read with ldmatrix (conflict-free under the swizzle), B = the
+// transposed weights staged once per CTA in shared memory, float32 accumulators.  The
+// epilogue applies the product, SiLU, W3 and the bias, takes the per-token arg-max and adds
+// the 16 choices to the chunk's histogram with integer atomics (order-independent).
 // HBM-bound: every hidden row is read once.
 //
 // finalize_map_kernel: per sequence, chunk winner (first maximum), routing freezing,
 // per-width counts and slot = rank among earlier chunks of the same width.
+#include <cuda.h>
 #include <cuda_bf16.h>
 
 #include "common.cuh"
@@ -18,17 +22,52 @@ namespace moqae {
 
 namespace {
 
-constexpr int kRouteWarps = 8;
-constexpr int kWPad = 32;   // elements of padding per transposed weight row (bank spread)
+constexpr int kMaxRouteWarps = 8;
+constexpr int kWPad = 8;             // elements of padding per transposed weight row (bank spread)
+constexpr int kBoxCols = 64;         // channels per TMA box (128 bytes: the swizzle span)
+constexpr int kBoxBytes = 16 * 128;  // 16 token rows
+constexpr int kBoxesPerStage = 4;
+constexpr int kStageBytes = kBoxesPerStage * kBoxBytes;
+constexpr int kStages = 2;
+constexpr long long kWaitLimit = 1ll << 22;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, int count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];\n"
+               ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
+               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+  for (long long i = 0; i < kWaitLimit; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  return false;
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&a)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(a[0]), "=r"(a[1]), "=r"(a[2]), "=r"(a[3]) : "r"(addr));
+}
 
 template <bool BF16>
 __device__ __forceinline__ void mma16816(float d[4], const uint32_t a[4], uint32_t b0, uint32_t b1) {
   if (BF16) {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
                  : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
   } else {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
                  : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
   }
@@ -47,22 +86,34 @@ __device__ __forceinline__ int argmax4(float p0, float p1, float p2, float p3) {
 }
 
 template <bool BF16>
-__global__ void __launch_bounds__(kRouteWarps * 32)
+__global__ void __launch_bounds__(kMaxRouteWarps * 32)
 route_score_vote_kernel(Dims dm, int32_t* __restrict__ votes /* [batch][max_chunks][4] of the group */,
-                        const uint16_t* __restrict__ hidden, int T, const uint16_t* __restrict__ W1,
+                        const __grid_constant__ CUtensorMap map_hidden, int T, const uint16_t* __restrict__ W1,
                         const uint16_t* __restrict__ W2, const float* __restrict__ W3,
-                        const float* __restrict__ bias, long long n_blocks16, int first_chunk) {
-  extern __shared__ __align__(16) uint16_t wt[];   // [8][d_in + kWPad], row n<4: W1[:,n]; n>=4: W2[:,n-4]
+                        const float* __restrict__ bias, long long n_blocks16, int first_chunk, int32_t* status) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  // the swizzled TMA boxes want 1024-byte alignment: round the base up (the launch adds the slack)
+  uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   const int D = dm.d_in;
-  const int ld = D + kWPad;
-  for (int i = threadIdx.x; i < D * 4; i += blockDim.x) {
+  const int n_boxes = (D + kBoxCols - 1) / kBoxCols;
+  const int Dpad = n_boxes * kBoxCols;
+  const int ld = Dpad + kWPad;
+  const int n_warps = blockDim.x >> 5;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint8_t* ring = smem + warp * (kStages * kStageBytes);
+  uint16_t* wt = reinterpret_cast<uint16_t*>(smem + n_warps * (kStages * kStageBytes));   // [8][ld]: W1^T then W2^T
+  uint64_t* bars = reinterpret_cast<uint64_t*>(wt + 8 * ld) + kStages * warp;
+  for (int i = threadIdx.x; i < Dpad * 4; i += blockDim.x) {
     const int c = i >> 2, n = i & 3;
-    wt[n * ld + c] = W1[i];
-    wt[(4 + n) * ld + c] = W2 ? W2[i] : static_cast<uint16_t>(0);
+    wt[n * ld + c] = c < D ? W1[i] : static_cast<uint16_t>(0);
+    wt[(4 + n) * ld + c] = (W2 && c < D) ? W2[i] : static_cast<uint16_t>(0);
+  }
+  if (lane == 0) {
+    for (int s = 0; s < kStages; ++s) mbar_init(smem_u32(bars + s), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
   }
   __syncthreads();
 
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = lane >> 2, t4 = lane & 3;
   const int C = T / dm.chunk;
   const int blocks_per_chunk = dm.chunk / 16;
@@ -74,30 +125,71 @@ route_score_vote_kernel(Dims dm, int32_t* __restrict__ votes /* [batch][max_chun
 #pragma unroll
     for (int j = 0; j < 4; ++j) w3[i][j] = W3 ? W3[i * 4 + j] : 0.0f;
   }
+  const int n_stages = (n_boxes + kBoxesPerStage - 1) / kBoxesPerStage;     // per 16-token block
+  const long long blk0 = static_cast<long long>(blockIdx.x) * n_warps + warp;
+  const long long blk_stride = static_cast<long long>(gridDim.x) * n_warps;
+  const long long my_blocks = blk0 < n_blocks16 ? (n_blocks16 - blk0 + blk_stride - 1) / blk_stride : 0;
+  const long long total_units = my_blocks * n_stages;                      // this warp's stream of stages
 
-  for (long long blk = static_cast<long long>(blockIdx.x) * kRouteWarps + warp; blk < n_blocks16;
-       blk += static_cast<long long>(gridDim.x) * kRouteWarps) {
+  auto block_coords = [&](long long blk, int& b, int& c, int& row) {
     const int sub = static_cast<int>(blk % blocks_per_chunk);
-    long long r = blk / blocks_per_chunk;
-    const int c = first_chunk + static_cast<int>(r % routed_chunks);
-    const int b = static_cast<int>(r / routed_chunks);
-    const long long tok0 = static_cast<long long>(b) * T + static_cast<long long>(c) * dm.chunk + sub * 16;
-    const uint4* row_lo = reinterpret_cast<const uint4*>(hidden + (tok0 + g) * D) + t4;
-    const uint4* row_hi = reinterpret_cast<const uint4*>(hidden + (tok0 + g + 8) * D) + t4;
-    const uint16_t* wrow = wt + g * ld + 8 * t4;
+    const long long r = blk / blocks_per_chunk;
+    c = first_chunk + static_cast<int>(r % routed_chunks);
+    b = static_cast<int>(r / routed_chunks);
+    row = b * T + c * dm.chunk + sub * 16;
+  };
+  auto issue = [&](long long u) {       // lane 0: stage u of this warp's stream
+    const long long blk = blk0 + (u / n_stages) * blk_stride;
+    const int st = static_cast<int>(u % n_stages);
+    int b, c, row;
+    block_coords(blk, b, c, row);
+    const int slot = static_cast<int>(u % kStages);
+    const int box0 = st * kBoxesPerStage;
+    const int nb = min(kBoxesPerStage, n_boxes - box0);
+    const uint32_t bar = smem_u32(bars + slot);
+    mbar_expect_tx(bar, nb * kBoxBytes);
+    for (int i = 0; i < nb; ++i)
+      tma_load_2d(smem_u32(ring + slot * kStageBytes + i * kBoxBytes), &map_hidden, (box0 + i) * kBoxCols, row, bar);
+  };
+  if (lane == 0)
+    for (long long u = 0; u < kStages && u < total_units; ++u) issue(u);
+
+  // ldmatrix row address of this lane inside a box: matrices (rows 0-7 | 8-15) x (k 0-7 | 8-15)
+  const int lm_row = (lane & 7) + ((lane >> 3) & 1) * 8;
+  const int lm_half = lane >> 4;
+  const uint16_t* wrow = wt + g * ld + 2 * t4;
+  uint32_t parity = 0;                  // bit s: parity to wait for on stage s
+  bool ok = true;
+  long long u = 0;
+  for (long long ib = 0; ib < my_blocks && ok; ++ib) {
+    const long long blk = blk0 + ib * blk_stride;
+    int b, c, row;
+    block_coords(blk, b, c, row);
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
     float acc2[4] = {0.f, 0.f, 0.f, 0.f};
-    const int n_win = D / 32;
-#pragma unroll 4
-    for (int w = 0; w < n_win; ++w) {
-      const uint4 lo = __ldg(row_lo + 4 * w);
-      const uint4 hi = __ldg(row_hi + 4 * w);
-      const uint4 bw = *reinterpret_cast<const uint4*>(wrow + 32 * w);
-      const uint32_t a1[4] = {lo.x, hi.x, lo.y, hi.y};
-      const uint32_t a2[4] = {lo.z, hi.z, lo.w, hi.w};
-      mma16816<BF16>(acc, a1, bw.x, bw.y);
-      mma16816<BF16>(acc2, a2, bw.z, bw.w);
+    for (int st = 0; st < n_stages; ++st, ++u) {
+      const int slot = static_cast<int>(u % kStages);
+      if (!mbar_wait_bounded(smem_u32(bars + slot), (parity >> slot) & 1u)) { ok = false; break; }
+      parity ^= 1u << slot;
+      const int box0 = st * kBoxesPerStage;
+      const int nb = min(kBoxesPerStage, n_boxes - box0);
+      const uint32_t stage_base = smem_u32(ring + slot * kStageBytes);
+      for (int i = 0; i < nb; ++i) {
+        const uint32_t box_base = stage_base + i * kBoxBytes + lm_row * 128;
+        const uint16_t* wk = wrow + (box0 + i) * kBoxCols;
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {
+          uint32_t a[4];
+          ldmatrix_x4(a, box_base + (((2 * kk + lm_half) ^ (lm_row & 7)) << 4));
+          const uint32_t b0 = *reinterpret_cast<const uint32_t*>(wk + 16 * kk);
+          const uint32_t b1 = *reinterpret_cast<const uint32_t*>(wk + 16 * kk + 8);
+          mma16816<BF16>((kk & 1) ? acc2 : acc, a, b0, b1);
+        }
+      }
+      __syncwarp();
+      if (lane == 0 && u + kStages < total_units) issue(u + kStages);
     }
+    if (!ok) break;
 #pragma unroll
     for (int i = 0; i < 4; ++i) acc[i] += acc2[i];
     // acc[0], acc[1]: token g, columns 2*t4, 2*t4+1; acc[2], acc[3]: token g+8.
@@ -140,6 +232,11 @@ route_score_vote_kernel(Dims dm, int32_t* __restrict__ votes /* [batch][max_chun
       const int cnt = __popc(m1) + __popc(m2);
       if (lane == 0 && cnt) atomicAdd(vrow + k, cnt);
     }
+  }
+  if (!ok) {
+    // a copy did not land in time: report it and give the copies in flight a last bounded chance
+    if (lane == 0) set_status(status, MOQAE_ERR_TIMEOUT, blockIdx.x, warp);
+    for (int s = 0; s < kStages; ++s) mbar_wait_bounded(smem_u32(bars + s), (parity >> s) & 1u);
   }
 }
 
@@ -197,6 +294,22 @@ finalize_map_kernel(Dims dm, CacheView cv, int group, int n_chunks, const uint8_
 
 }  // namespace
 
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess)
+      p = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
+  return fn;
+}
+
 cudaError_t launch_route(const Dims& dm, const CacheView& cv, const void* hidden, int T, const void* W1,
                          const void* W2, const float* W3, const float* bias, int group,
                          int32_t* votes_out, cudaStream_t st) {
@@ -208,25 +321,44 @@ cudaError_t launch_route(const Dims& dm, const CacheView& cv, const void* hidden
   const int first = dm.rf_first_chunk ? 1 : 0;
   const long long n_blocks16 = static_cast<long long>(dm.batch) * (C > first ? C - first : 0) * (dm.chunk / 16);
   if (n_blocks16 > 0) {
-    int dev = 0, sms = 148;
+    int dev = 0, sms = 148, smem_max = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const size_t smem = sizeof(uint16_t) * 8 * static_cast<size_t>(dm.d_in + kWPad);
-    long long want = (n_blocks16 + kRouteWarps - 1) / kRouteWarps;
-    const long long cap = static_cast<long long>(sms) * 2;
-    const unsigned grid = static_cast<unsigned>(want < cap ? want : cap);
+    cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    // [batch*T][d_in] 16-bit tensor, boxes of 64 channels x 16 tokens, 128-byte swizzle
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return cudaErrorNotSupported;
+    CUtensorMap map;
+    const cuuint64_t gdim[2] = {static_cast<cuuint64_t>(dm.d_in), static_cast<cuuint64_t>(dm.batch) * T};
+    const cuuint64_t gstride[1] = {static_cast<cuuint64_t>(dm.d_in) * 2};
+    const cuuint32_t box[2] = {kBoxCols, 16};
+    const cuuint32_t estr[2] = {1, 1};
+    if (enc(&map, CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, const_cast<void*>(hidden), gdim, gstride, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cudaErrorInvalidValue;
+    const int n_boxes = (dm.d_in + kBoxCols - 1) / kBoxCols;
+    const size_t wt_bytes = sizeof(uint16_t) * 8 * static_cast<size_t>(n_boxes * kBoxCols + kWPad);
+    // as many warps (each with its own ring) as fit beside the weights, one CTA per SM
+    int warps = kMaxRouteWarps;
+    auto smem_for = [&](int w) { return static_cast<size_t>(w) * kStages * kStageBytes + wt_bytes + 8 * kStages * w + 1024; };
+    while (warps > 1 && smem_for(warps) > static_cast<size_t>(smem_max)) --warps;
+    if (smem_for(warps) > static_cast<size_t>(smem_max)) return cudaErrorInvalidConfiguration;
+    const size_t smem = smem_for(warps);
+    long long want = (n_blocks16 + warps - 1) / warps;
+    const unsigned grid = static_cast<unsigned>(want < sms ? want : sms);
     if (dm.dtype == MOQAE_DTYPE_BF16) {
       e = cudaFuncSetAttribute(route_score_vote_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
       if (e != cudaSuccess) return e;
-      route_score_vote_kernel<true><<<grid, kRouteWarps * 32, smem, st>>>(
-          dm, votes, static_cast<const uint16_t*>(hidden), T, static_cast<const uint16_t*>(W1),
-          static_cast<const uint16_t*>(W2), W3, bias, n_blocks16, first);
+      route_score_vote_kernel<true><<<grid, warps * 32, smem, st>>>(
+          dm, votes, map, T, static_cast<const uint16_t*>(W1), static_cast<const uint16_t*>(W2), W3, bias,
+          n_blocks16, first, cv.status);
     } else {
       e = cudaFuncSetAttribute(route_score_vote_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
       if (e != cudaSuccess) return e;
-      route_score_vote_kernel<false><<<grid, kRouteWarps * 32, smem, st>>>(
-          dm, votes, static_cast<const uint16_t*>(hidden), T, static_cast<const uint16_t*>(W1),
-          static_cast<const uint16_t*>(W2), W3, bias, n_blocks16, first);
+      route_score_vote_kernel<false><<<grid, warps * 32, smem, st>>>(
+          dm, votes, map, T, static_cast<const uint16_t*>(W1), static_cast<const uint16_t*>(W2), W3, bias,
+          n_blocks16, first, cv.status);
     }
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
