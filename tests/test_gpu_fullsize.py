@@ -1,0 +1,117 @@
+"""GPU parity at the full size of the 128k-context workload (batch 4, 131072 (+ tail) tokens,
+8 kv heads / 32 query heads, chunk 256, bf16, d_in 4096), one layer, in the launch
+configuration the benchmark times.  Inputs are drawn on the device; sampled pieces are copied
+to the host and recomputed by the oracle one by one:
+  * router: sampled chunks (vote histograms away from near-ties, winner),
+  * quantise+pack: every tile of sampled (sequence, kv head, chunk) slots, byte for byte,
+  * decode attention: sampled (sequence, kv head) pairs over the whole context, all four
+    query heads of the group, against the oracle run on the GPU's own packed cache and map.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import moqae_oracle as O
+from paper_2506_07533_b200 import binding as mq
+from paper_2506_07533_b200 import synth
+from paper_2506_07533_b200 import workloads as W
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+TAU = 1e-4
+
+
+@pytest.fixture(scope="module")
+def job():
+    wl = W.WORKLOADS["cfg4"]
+    B, Hkv, Hq, chunk, D, dtype = wl.batch, wl.n_kv_heads, wl.n_q_heads, wl.chunk, wl.d_in, wl.dtype
+    T = wl.context + 37                                   # a ragged tail on top of 512 chunks
+    dev = "cuda"
+    cfg = mq.make_config(n_layers=1, n_q_heads=Hq, n_kv_heads=Hkv, chunk=chunk, dtype=dtype, d_in=D,
+                         max_tokens=T, batch=B, rs_group=1, rf_first_chunk=1, tail_capacity=chunk)
+    hidden = synth.hidden_states(B, T, D, chunk, dtype, 4242, dev)
+    W1, W2, W3, bias = synth.router_weights(D, 4, dtype, 4243, dev)
+    K, V = synth.keys_values(B, T, Hkv, 128, dtype, 4244, dev, outlier_frac=wl.outlier_frac)
+    q = synth.normal((B, Hq, 128), dtype, 4245, dev)
+    C = T // chunk
+    cache = mq.moqae_cache_bind(cfg, [C, C, C, C])
+    mq.moqae_route(cfg, hidden, T, W1, W2, W3, bias, 0, cache)
+    torch.cuda.synchronize()
+    routed = dict(map=cache.map[0, :, :C].cpu().numpy().copy(), votes=cache.votes[0, :, :C].cpu().numpy().copy(),
+                  slot=cache.slot[0, :, :C].cpu().numpy().copy(), count=cache.count[0].cpu().numpy().copy())
+    # the cache itself is built from a seeded map with the workload's 60/30/5/5 mix, so that every
+    # width is present whatever the untrained synthetic router prefers
+    forced = torch.from_numpy(synth.multinomial_map(B, C, wl.mix, 77)).to(dev)
+    mq.moqae_quantize_kv(cfg, K, V, T, 0, cache, forced_map=forced)
+    ws = torch.empty(mq.moqae_decode_attn_workspace(cfg), dtype=torch.uint8, device=dev)
+    out = torch.full((B, Hq, 128), float("nan"), dtype=torch.float32, device=dev)
+    mq.moqae_decode_attn(cfg, q, 0, cache, out, ws)
+    torch.cuda.synchronize()
+    assert mq.moqae_poll_status(cache) == 0
+    return dict(wl=wl, cfg=cfg, T=T, C=C, hidden=hidden, routed=routed, W=(W1, W2, W3, bias), K=K, V=V, q=q, cache=cache, out=out)
+
+
+def test_router_sampled_chunks(job):
+    wl, T, C, cache = job["wl"], job["T"], job["C"], job["cache"]
+    W1, W2, W3, bias = job["W"]
+    gmap, gvotes = job["routed"]["map"], job["routed"]["votes"]
+    assert (gmap[:, 0] == 3).all()                        # routing freezing
+    w1, w2 = synth.to_u16(W1), synth.to_u16(W2)
+    rs = np.random.RandomState(5)
+    picks = [(b, c) for b in range(wl.batch) for c in rs.choice(np.arange(1, C), 6, replace=False)]
+    picks += [(0, 1), (wl.batch - 1, C - 1)]
+    for b, c in picks:
+        rows = job["hidden"][b, c * wl.chunk:(c + 1) * wl.chunk].unsqueeze(0)
+        ref = O.route(synth.to_u16(rows), wl.dtype, wl.chunk, w1, w2, W3.cpu().numpy(), bias.cpu().numpy(),
+                      rf_first_chunk=False)
+        frag = np.where(ref["margin"][0] < TAU * np.maximum(ref["pmax"][0], 1e-30))[0]
+        diff = gvotes[b, c].astype(np.int64) - ref["votes"][0, 0]
+        assert diff.sum() == 0 and np.abs(diff).sum() // 2 <= len(frag), (b, c, diff, len(frag))
+        if len(frag) == 0:
+            assert gmap[b, c] == ref["map"][0, 0]
+    slot, count = O.assign_slots(gmap)
+    assert (job["routed"]["slot"] == slot).all() and (job["routed"]["count"] == count).all()
+
+
+def test_quantize_sampled_slots_byte_exact(job):
+    wl, C, cache = job["wl"], job["C"], job["cache"]
+    gmap = cache.map[0, :, :C].cpu().numpy()
+    slot, _ = O.assign_slots(gmap)
+    rs = np.random.RandomState(6)
+    for w in range(4):                                    # ten slots of every width
+        where = np.argwhere(gmap == w)
+        assert len(where) >= 10
+        for b, c in where[rs.choice(len(where), 10, replace=False)]:
+            h = rs.randint(wl.n_kv_heads)
+            Kc = job["K"][b, c * wl.chunk:(c + 1) * wl.chunk, h].unsqueeze(0).unsqueeze(2)
+            Vc = job["V"][b, c * wl.chunk:(c + 1) * wl.chunk, h].unsqueeze(0).unsqueeze(2)
+            ref = O.quantize_kv(synth.to_u16(Kc), synth.to_u16(Vc), wl.dtype, wl.chunk, gmap[b:b + 1, c:c + 1])
+            got = cache.pool(w)[0, b, h, int(slot[b, c])].cpu().numpy()
+            assert (got == ref["pools"][w][0, 0, 0]).all(), (b, h, c, w)
+    r = job["T"] % wl.chunk
+    assert (cache.tail_len[0].cpu().numpy() == r).all()
+    tk = cache.tail("k")[0, 1, 3, :r].cpu().numpy().view(np.uint16)
+    assert (tk == synth.to_u16(job["K"][1, C * wl.chunk:, 3])).all()
+
+
+def test_decode_sampled_heads_whole_context(job):
+    wl, C, T, cache = job["wl"], job["C"], job["T"], job["cache"]
+    G = wl.n_q_heads // wl.n_kv_heads
+    gmap = cache.map[0, :, :C].cpu().numpy()
+    slot, count = O.assign_slots(gmap)
+    out = job["out"].cpu().numpy()
+    r = T % wl.chunk
+    for b, h in [(0, 0), (3, 7), (2, 5)]:
+        # the oracle reads the GPU's own packed bytes of this (sequence, head)
+        pools = []
+        for w in range(4):
+            n = int(count[b, w])
+            pools.append(cache.pool(w)[0, b, h, :max(n, 1)].cpu().numpy()[None, None])
+        oc = dict(pools=pools, slot=slot[b:b + 1], count=count[b:b + 1], tail_len=r,
+                  tail_k=cache.tail("k")[0, b, h, :r].cpu().numpy().view(np.uint16)[None, None],
+                  tail_v=cache.tail("v")[0, b, h, :r].cpu().numpy().view(np.uint16)[None, None])
+        qh = synth.to_u16(job["q"][b, h * G:(h + 1) * G]).reshape(1, G, 128)
+        ref = O.decode_attn(qh, wl.dtype, oc, wl.chunk)
+        ok, e_abs, e_rel = H.attn_tolerance_ok(out[b, h * G:(h + 1) * G][None], ref)
+        assert ok, (b, h, e_abs, e_rel)
