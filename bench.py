@@ -125,6 +125,9 @@ class Job:
         self.W1, self.W2, self.W3, self.bias = synth.router_weights(wl.d_in, 4, wl.dtype, seed + 7, device,
                                                                     gated=wl.gated_router)
         self.q = synth.normal((wl.n_layers, B, Hq, 128), wl.dtype, seed + 9, device)
+        if wl.decode_steps > 1:
+            self.k_new = synth.normal((wl.decode_steps, wl.n_layers, B, Hkv, 128), wl.dtype, seed + 11, device)
+            self.v_new = synth.normal((wl.decode_steps, wl.n_layers, B, Hkv, 128), wl.dtype, seed + 12, device)
         self.out = torch.zeros((wl.n_layers, B, Hq, 128), dtype=torch.float32, device=device)
         self.ws = torch.empty(mq.moqae_decode_attn_workspace(self.cfg), dtype=torch.uint8, device=device)
         self.n_splits = self.ws.numel() // (B * Hq * 130 * 4)
@@ -197,8 +200,17 @@ class Job:
             self.mq.moqae_quantize_kv(self.cfg, K, V, self.T, l, self.cache, forced_map=fm)
 
     def decode_all(self):
-        for l in range(self.wl.n_layers):
-            self.mq.moqae_decode_attn(self.cfg, self.q[l], l, self.cache, self.out[l], self.ws)
+        wl = self.wl
+        if wl.decode_steps == 1:
+            for l in range(wl.n_layers):
+                self.mq.moqae_decode_attn(self.cfg, self.q[l], l, self.cache, self.out[l], self.ws)
+            return
+        # generation loop: every step appends one token per sequence to each layer's 16-bit tail
+        # (routing is not re-run) and attends over the grown cache
+        for s in range(wl.decode_steps):
+            for l in range(wl.n_layers):
+                self.mq.moqae_append_kv(self.cfg, self.k_new[s, l], self.v_new[s, l], l, self.cache)
+                self.mq.moqae_decode_attn(self.cfg, self.q[l], l, self.cache, self.out[l], self.ws)
 
     def counts(self):
         return self.cache.count.cpu().numpy()           # [groups, batch, 4]
@@ -209,15 +221,19 @@ class Job:
         tail = self.T % wl.chunk
         route = 0 if self.forced is not None else wl.n_groups * W.route_bytes_per_group(wl, self.T)
         quant = sum(W.quantize_bytes_per_layer(cnt[l // wl.rs_group], wl, self.T) for l in range(wl.n_layers))
-        dec = sum(W.decode_bytes_per_layer(cnt[l // wl.rs_group], wl, self.n_splits, tail)
-                  for l in range(wl.n_layers))
+        dec = 0
+        for st in range(wl.decode_steps):
+            t_len = tail + (st + 1 if wl.decode_steps > 1 else 0)
+            dec += sum(W.decode_bytes_per_layer(cnt[l // wl.rs_group], wl, self.n_splits, t_len)
+                       for l in range(wl.n_layers))
         return route, quant, dec
 
     def launches_per_step(self):
         wl = self.wl
         route = 0 if self.forced is not None else 2 * wl.n_groups        # score+vote, finalise
         quant = 2 * wl.n_layers + (wl.n_groups if self.forced is not None else 0)
-        return route + quant + 2 * wl.n_layers                            # + split-K and combine
+        per_decode = 2 + (1 if wl.decode_steps > 1 else 0)                # split-K, combine (+ append)
+        return route + quant + per_decode * wl.n_layers * wl.decode_steps
 
 
 def run_ours(args):
@@ -241,6 +257,8 @@ def run_ours(args):
     wl = W.WORKLOADS[args.workload]
     if args.layers:
         wl = dataclasses.replace(wl, n_layers=args.layers)
+    if args.chunk:
+        wl = dataclasses.replace(wl, chunk=args.chunk)
     if args.mix:
         wl = dataclasses.replace(wl, mix=tuple(float(x) for x in args.mix.split(",")))
     job = Job(wl, device, seed=1234 + rank, context=args.context, force_map=bool(args.mix))
@@ -303,8 +321,8 @@ def run_ours(args):
     if rank == 0:
         peak, peak_kind = read_peaks()
         dec_gbs = world * b_dec / (ms_dec * 1e6)
-        per_launch_bytes = b_dec / wl.n_layers
-        per_launch_ms = ms_dec / wl.n_layers
+        per_launch_bytes = b_dec / (wl.n_layers * wl.decode_steps)
+        per_launch_ms = ms_dec / (wl.n_layers * wl.decode_steps)
         achieved = per_launch_bytes / (per_launch_ms * 1e6)
         cnt = job.counts().astype(np.float64)
         mix = (cnt.sum((0, 1)) / max(cnt.sum(), 1)).round(4).tolist()
@@ -323,12 +341,12 @@ def run_ours(args):
                        "n_splits": job.n_splits},
             "phase_ms": {"route": round(ms_route, 4), "quantize_pack": round(ms_quant, 4),
                          "decode_attn": round(ms_dec, 4)},
-            "context_tokens_per_s": round(world * wl.batch * job.T / (ms_dec * 1e-3), 1),
+            "context_tokens_per_s": round(world * wl.batch * job.T * wl.decode_steps / (ms_dec * 1e-3), 1),
             "quantize_route_gbs": round(world * (b_route + b_quant) / ((ms_route + ms_quant) * 1e6), 1),
             "bytes_per_step": {"route": b_route, "quantize_pack": b_quant, "decode_attn": b_dec},
             "gpu_launches": job.launches_per_step() * args.steps,
             "clocks": clocks,
-            "roofline": {"bound": "hbm", "kernel": "decode_splitk_kernel (+combine)",
+            "roofline": {"bound": "hbm", "kernel": "decode_mma_kernel (+ decode_combine_kernel)",
                          "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
                          "frac": round(achieved / peak, 4), "peak_source": f"of {peak_kind}",
                          "frac_of_8TBs_spec": round(achieved / 8000.0, 4),
@@ -363,6 +381,9 @@ def measure_e2e(job, args, torch):
     d_K, d_V = torch.empty_like(job.kv[0][0]), torch.empty_like(job.kv[0][1])
     d_h = torch.empty_like(job.hidden[0]) if job.hidden else None
     d_q = torch.empty_like(job.q)
+    new_tok = []
+    if wl.decode_steps > 1:                          # the generated tokens' K/V rows also start on the host
+        new_tok = [(job.k_new, job.k_new.cpu().pin_memory()), (job.v_new, job.v_new.cpu().pin_memory())]
     h2d = 0
     ms_dec, ms_step = 0.0, 0.0
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
@@ -385,8 +406,13 @@ def measure_e2e(job, args, torch):
         ev[1].record()
         d_q.copy_(h_q, non_blocking=True)
         h2d += h_q.numel() * 2
-        for l in range(wl.n_layers):
-            job.mq.moqae_decode_attn(job.cfg, d_q[l], l, job.cache, job.out[l], job.ws)
+        for d_t, h_t in new_tok:
+            d_t.copy_(h_t, non_blocking=True)
+            h2d += h_t.numel() * 2
+        saved = job.q
+        job.q = d_q
+        job.decode_all()
+        job.q = saved
         h_out.copy_(job.out, non_blocking=True)
         ev[2].record()
         torch.cuda.synchronize()
@@ -424,18 +450,25 @@ def oracle_sample(wl, tokens: int, seed=77):
 
 
 def cpu_baseline(wl, budget_s=20.0):
+    """The oracle as it stands on about `budget_s` seconds of work: whole-context (sequence, kv head)
+    pairs of one layer, one after the other (quantise+pack, then decode for the head's query group)."""
     import threadpoolctl
-    tokens = 4 * wl.chunk
-    r = oracle_sample(wl, tokens)
-    per_tok = (r["quant_s"] + r["decode_s"]) / tokens
-    tokens = int(min(wl.context, max(tokens, budget_s / max(per_tok, 1e-9))) // wl.chunk * wl.chunk)
-    r = oracle_sample(wl, tokens)
+    probe = oracle_sample(wl, 4 * wl.chunk)
+    per_tok = (probe["quant_s"] + probe["decode_s"]) / probe["tokens"]
+    tokens = int(min(wl.context, max(4 * wl.chunk, budget_s / max(per_tok, 1e-9))) // wl.chunk * wl.chunk)
+    runs, spent = [], 0.0
+    while spent < budget_s and len(runs) < wl.batch * wl.n_kv_heads:
+        r = oracle_sample(wl, tokens, seed=77 + len(runs))
+        runs.append(r)
+        spent += r["quant_s"] + r["decode_s"]
+    dec_s = sum(r["decode_s"] for r in runs)
+    q_s = sum(r["quant_s"] for r in runs)
     threads = max([p.get("num_threads", 1) for p in threadpoolctl.threadpool_info()] or [1])
-    return {"value": round(r["decode_bytes"] / r["decode_s"] / 1e9, 5), "unit": "GB/s", "cores": int(threads),
-            "kind": "oracle",
-            "sample": f"decode attention of 1 sequence x 1 kv head x {r['tokens']} context tokens of {wl.name} "
-                      f"(numpy float64 oracle, {r['decode_s']:.1f} s); its quantise+pack ran at "
-                      f"{r['quant_bytes'] / r['quant_s'] / 1e9:.5f} GB/s ({r['quant_s']:.1f} s)",
+    return {"value": round(sum(r["decode_bytes"] for r in runs) / dec_s / 1e9, 5), "unit": "GB/s",
+            "cores": int(threads), "kind": "oracle",
+            "sample": f"decode attention of {len(runs)} (sequence, kv head) pairs x {tokens} context tokens of one "
+                      f"layer of {wl.name} (numpy float64 oracle, {dec_s:.1f} s); their quantise+pack ran at "
+                      f"{sum(r['quant_bytes'] for r in runs) / q_s / 1e9:.5f} GB/s ({q_s:.1f} s)",
             "host_cpus": os.cpu_count()}
 
 
@@ -477,9 +510,10 @@ def main():
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg4", choices=["cfg1", "cfg2", "cfg3", "cfg4"])
+    ap.add_argument("--workload", default="cfg4", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
     ap.add_argument("--context", type=int, default=None, help="override the context length (profiling)")
     ap.add_argument("--layers", type=int, default=None, help="override the layer count (profiling)")
+    ap.add_argument("--chunk", type=int, default=None, help="override the chunk size (chunk-size sweep)")
     ap.add_argument("--mix", default=None,
                     help="four comma-separated shares: skip the router and force a seeded multinomial map "
                          "with this 2/4/8/16-bit mix (e.g. 1,0,0,0 = uniform 2-bit)")

@@ -44,6 +44,9 @@ WORKLOADS = {
                      decode_steps=16),
     # Llama-3-8B-shaped GQA, the 128k-context target
     "cfg4": Workload("cfg4", 32, 32, 8, 4096, 4, 131072, 256, 1, 3, (0.60, 0.30, 0.05, 0.05), 0.01),
+    # prefill quantise+route sweep: one layer, 32 kv heads, 131072 tokens; the chunk size and the
+    # map (forced uniform widths or router-chosen) are varied by the caller
+    "cfg5": Workload("cfg5", 1, 32, 32, 4096, 1, 131072, 128, 1, 1, (0.25, 0.25, 0.25, 0.25), 0.01),
 }
 
 
