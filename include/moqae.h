@@ -192,6 +192,26 @@ int moqae_quantize_kv(const moqae_config* cfg, const void* K, const void* V, int
 int moqae_append_kv(const moqae_config* cfg, const void* k_new, const void* v_new,
                     int32_t layer, const moqae_cache* cache, void* stream);
 
+/*
+ * Turn the full 16-bit tails of one routing-sharing group into one more routed, quantised
+ * chunk during generation.  Section 3.2 keeps the tokens that do not fill a chunk in 16 bits;
+ * once `chunk` tokens have been appended they are a complete chunk and go through the same
+ * router (Eq. 1, Eq. 2) and quantiser as a prefill chunk.  (The paper does not say when this
+ * happens during decoding; this call is the reading "as soon as the chunk is complete".)
+ *   hidden_tail [batch][chunk][d_in] input dtype: the hidden states (router inputs of the group's
+ *   first layer) of the tail's tokens, buffered by the caller as the tokens were generated.
+ *   W1, W2, W3, bias as in moqae_route.
+ *   A sequence takes part only if tail_len of the group's first layer equals `chunk` exactly;
+ *   the others are left untouched.  For a participating sequence the new chunk gets index
+ *   n = chunks so far, map[n] = winner of the vote (16-bit if n = 0 and rf_first_chunk),
+ *   slot[n] / count are updated, the tails of ALL layers of the group are packed into that slot
+ *   of their pools, and their tail_len becomes 0.  Needs tail_capacity >= chunk.  A full table or
+ *   pool sets status[0] = MOQAE_ERR_POOL_FULL and leaves the sequence untouched.
+ */
+int moqae_flush_tail(const moqae_config* cfg, const void* hidden_tail, const void* W1, const void* W2,
+                     const float* W3, const float* bias, int32_t layer_group, const moqae_cache* cache,
+                     void* stream);
+
 /* Bytes of scratch moqae_decode_attn needs for `cfg` on the current device (host out). */
 int moqae_decode_attn_workspace(const moqae_config* cfg, int64_t* out_bytes);
 

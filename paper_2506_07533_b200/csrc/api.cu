@@ -199,6 +199,30 @@ int moqae_append_kv(const moqae_config* cfg, const void* k_new, const void* v_ne
   return e == cudaSuccess ? MOQAE_OK : cuda_fail(e);
 }
 
+int moqae_flush_tail(const moqae_config* cfg, const void* hidden_tail, const void* W1, const void* W2,
+                     const float* W3, const float* bias, int32_t layer_group, const moqae_cache* cache,
+                     void* stream) {
+  int rc = check_config(cfg);
+  if (rc != MOQAE_OK) return rc;
+  moqae::CacheView cv;
+  rc = check_cache(cache, &cv);
+  if (rc != MOQAE_OK) return rc;
+  if (!hidden_tail || !W1) return MOQAE_ERR_INVALID_ARG;
+  if ((W2 == nullptr) != (W3 == nullptr)) return MOQAE_ERR_INVALID_ARG;
+  if (layer_group < 0 || layer_group >= n_groups(cfg)) return MOQAE_ERR_INVALID_ARG;
+  if (cfg->tail_capacity < cfg->chunk || !cache->tail_k || !cache->tail_v) return MOQAE_ERR_POOL_FULL;
+  if (!aligned16(hidden_tail) || !aligned16(W1) || !aligned16(W2) || !aligned16(W3) || !aligned16(bias))
+    return MOQAE_ERR_MISALIGNED;
+  const moqae::Dims dm = dims_of(cfg);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  cudaError_t e = moqae::launch_flush_route(dm, cv, hidden_tail, W1, W2, W3, bias, layer_group, st);
+  const int l0 = layer_group * cfg->rs_group;
+  for (int l = l0; e == cudaSuccess && l < l0 + cfg->rs_group && l < cfg->n_layers; ++l)
+    e = moqae::launch_flush_quantize(dm, cv, l, st);
+  if (e == cudaSuccess) e = moqae::launch_flush_reset(dm, cv, layer_group, st);
+  return e == cudaSuccess ? MOQAE_OK : cuda_fail(e);
+}
+
 int moqae_decode_attn_workspace(const moqae_config* cfg, int64_t* out_bytes) {
   int rc = check_config(cfg);
   if (rc != MOQAE_OK) return rc;

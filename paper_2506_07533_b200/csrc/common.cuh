@@ -71,6 +71,10 @@ void record_cuda_error(cudaError_t e);
 cudaError_t launch_route(const Dims& dm, const CacheView& cv, const void* hidden, int T, const void* W1,
                          const void* W2, const float* W3, const float* bias, int group,
                          int32_t* votes_out, cudaStream_t st);
+cudaError_t launch_flush_route(const Dims& dm, const CacheView& cv, const void* hidden_tail, const void* W1,
+                               const void* W2, const float* W3, const float* bias, int group, cudaStream_t st);
+cudaError_t launch_flush_quantize(const Dims& dm, const CacheView& cv, int layer, cudaStream_t st);
+cudaError_t launch_flush_reset(const Dims& dm, const CacheView& cv, int group, cudaStream_t st);
 cudaError_t launch_finalize_map(const Dims& dm, const CacheView& cv, int group, int n_chunks,
                                 const uint8_t* forced_map, cudaStream_t st);
 cudaError_t launch_quantize(const Dims& dm, const CacheView& cv, const void* K, const void* V, int T,

@@ -28,6 +28,7 @@ constexpr int kPrmBytes = 1024;                // value groups: [32 tokens][4 gr
 constexpr int kWarpSmem = 2 * kInBytes + kOutBytes + kPrmBytes;
 constexpr long long kWaitLimit = 1ll << 22;
 constexpr float kMagic = 12582912.0f;          // 1.5 * 2^23
+constexpr int kSkipTile = 0xfe;                // width marker: nothing to do for this tile
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -284,7 +285,7 @@ struct TileRef {
 template <bool BF16>
 __global__ void __launch_bounds__(kQWarps * 32, 2)
 quantize_pack_kernel(Dims dm, CacheView cv, const __grid_constant__ CUtensorMap mapK,
-                     const __grid_constant__ CUtensorMap mapV, int T, int layer, long long n_tiles) {
+                     const __grid_constant__ CUtensorMap mapV, int T, int layer, long long n_tiles, int flush) {
   extern __shared__ __align__(128) uint8_t smem[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   uint8_t* bufK = smem + warp * kWarpSmem;
@@ -308,6 +309,7 @@ quantize_pack_kernel(Dims dm, CacheView cv, const __grid_constant__ CUtensorMap 
   const uint8_t* map_g = cv.map + static_cast<long long>(group) * dm.batch * dm.max_chunks;
   const int32_t* slot_g = cv.slot + static_cast<long long>(group) * dm.batch * dm.max_chunks;
 
+  const int32_t* count_g = cv.count + static_cast<long long>(group) * dm.batch * 4;
   auto tile_ref = [&](long long id) {
     // id = ((b * C + c) * tpc + j) * H + h : heads fastest, so neighbouring warps read
     // neighbouring 256-byte segments of the same token rows
@@ -316,13 +318,29 @@ quantize_pack_kernel(Dims dm, CacheView cv, const __grid_constant__ CUtensorMap 
     long long x = id / H;
     r.j = static_cast<int>(x % tpc);
     x /= tpc;
-    const int c = static_cast<int>(x % C);
-    r.b = static_cast<int>(x / C);
-    r.x = r.h * kHeadDim;
-    r.y = r.b * T + c * dm.chunk + r.j * kTileTokens;
-    const long long tbl = static_cast<long long>(r.b) * dm.max_chunks + c;
-    r.w = map_g[tbl];                      // loaded one tile ahead of their use
-    r.slot = slot_g[tbl];
+    if (!flush) {
+      const int c = static_cast<int>(x % C);
+      r.b = static_cast<int>(x / C);
+      r.x = r.h * kHeadDim;
+      r.y = r.b * T + c * dm.chunk + r.j * kTileTokens;
+      const long long tbl = static_cast<long long>(r.b) * dm.max_chunks + c;
+      r.w = map_g[tbl];                      // loaded one tile ahead of their use
+      r.slot = slot_g[tbl];
+    } else {
+      // flush of a full tail: the source is the tail itself ([layer][b][h][row][128]); the target is
+      // the sequence's newest chunk, marked with bit 7 in the map while its rows are being packed
+      r.b = static_cast<int>(x);
+      r.x = 0;
+      r.y = ((layer * dm.batch + r.b) * H + r.h) * dm.tail_capacity + r.j * kTileTokens;
+      const int c = count_g[4 * r.b] + count_g[4 * r.b + 1] + count_g[4 * r.b + 2] + count_g[4 * r.b + 3] - 1;
+      r.w = kSkipTile;
+      r.slot = 0;
+      if (c >= 0) {
+        const long long tbl = static_cast<long long>(r.b) * dm.max_chunks + c;
+        const int e = map_g[tbl];
+        if (e & 0x80) { r.w = e & 0x7f; r.slot = slot_g[tbl]; }
+      }
+    }
     return r;
   };
   auto fetch = [&](const CUtensorMap* map, const TileRef& r, uint8_t* buf, uint32_t bar) {
@@ -350,7 +368,7 @@ quantize_pack_kernel(Dims dm, CacheView cv, const __grid_constant__ CUtensorMap 
 #pragma unroll
     for (int k = 0; k < 4; ++k) cap = (w == k) ? cv.capacity[k] : cap;
     const bool valid = w <= 3 && slot >= 0 && slot < cap;
-    if (!valid && lane == 0) set_status(cv.status, MOQAE_ERR_POOL_FULL, w, slot);
+    if (!valid && w != kSkipTile && lane == 0) set_status(cv.status, MOQAE_ERR_POOL_FULL, w, slot);
     uint8_t* tile = nullptr;
     if (valid) {
       const long long tb = tile_bytes_of_expert(w);
@@ -462,6 +480,19 @@ __global__ void append_kernel(Dims dm, CacheView cv, const uint16_t* __restrict_
   if (threadIdx.x == 0) cv.tail_len[layer * dm.batch + b] = len + 1;
 }
 
+__global__ void flush_reset_kernel(Dims dm, CacheView cv, int group) {
+  const int b = blockIdx.x;
+  const int32_t* count = cv.count + (static_cast<long long>(group) * dm.batch + b) * 4;
+  const int c = count[0] + count[1] + count[2] + count[3] - 1;
+  if (c < 0) return;
+  uint8_t* entry = cv.map + (static_cast<long long>(group) * dm.batch + b) * dm.max_chunks + c;
+  if (!(*entry & 0x80)) return;
+  __syncwarp();
+  if (threadIdx.x == 0) *entry &= 0x7f;
+  for (int l = group * dm.rs_group + threadIdx.x; l < min(dm.n_layers, (group + 1) * dm.rs_group); l += 32)
+    cv.tail_len[l * dm.batch + b] = 0;
+}
+
 int sm_count() {
   static int sms = 0;
   if (sms == 0) {
@@ -520,17 +551,47 @@ cudaError_t launch_quantize(const Dims& dm, const CacheView& cv, const void* K, 
     if (dm.dtype == MOQAE_DTYPE_BF16) {
       e = cudaFuncSetAttribute(quantize_pack_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
       if (e != cudaSuccess) return e;
-      quantize_pack_kernel<true><<<grid, kQWarps * 32, smem, st>>>(dm, cv, mapK, mapV, T, layer, n_tiles);
+      quantize_pack_kernel<true><<<grid, kQWarps * 32, smem, st>>>(dm, cv, mapK, mapV, T, layer, n_tiles, 0);
     } else {
       e = cudaFuncSetAttribute(quantize_pack_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
       if (e != cudaSuccess) return e;
-      quantize_pack_kernel<false><<<grid, kQWarps * 32, smem, st>>>(dm, cv, mapK, mapV, T, layer, n_tiles);
+      quantize_pack_kernel<false><<<grid, kQWarps * 32, smem, st>>>(dm, cv, mapK, mapV, T, layer, n_tiles, 0);
     }
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }
   dim3 g(8, dm.batch);
   tail_copy_kernel<<<g, 256, 0, st>>>(dm, cv, static_cast<const uint16_t*>(K), static_cast<const uint16_t*>(V), T, layer);
+  return cudaGetLastError();
+}
+
+// Pack the full tails of `layer` into the chunk that launch_flush_route has just added to the tables.
+cudaError_t launch_flush_quantize(const Dims& dm, const CacheView& cv, int layer, cudaStream_t st) {
+  const long long n_tiles = static_cast<long long>(dm.batch) * (dm.chunk / kTileTokens) * dm.n_kv_heads;
+  CUtensorMap mapK, mapV;
+  const long long rows = static_cast<long long>(dm.n_layers) * dm.batch * dm.n_kv_heads * dm.tail_capacity;
+  if (!make_tile_map(&mapK, cv.tail_k, rows, kHeadDim) || !make_tile_map(&mapV, cv.tail_v, rows, kHeadDim))
+    return cudaErrorNotSupported;
+  const size_t smem = static_cast<size_t>(kQWarps) * kWarpSmem + kQWarps * 16;
+  const long long want = (n_tiles + kQWarps - 1) / kQWarps;
+  const long long cap = 2ll * sm_count();
+  const unsigned grid = static_cast<unsigned>(want < cap ? want : cap);
+  cudaError_t e;
+  if (dm.dtype == MOQAE_DTYPE_BF16) {
+    e = cudaFuncSetAttribute(quantize_pack_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (e != cudaSuccess) return e;
+    quantize_pack_kernel<true><<<grid, kQWarps * 32, smem, st>>>(dm, cv, mapK, mapV, 0, layer, n_tiles, 1);
+  } else {
+    e = cudaFuncSetAttribute(quantize_pack_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (e != cudaSuccess) return e;
+    quantize_pack_kernel<false><<<grid, kQWarps * 32, smem, st>>>(dm, cv, mapK, mapV, 0, layer, n_tiles, 1);
+  }
+  return cudaGetLastError();
+}
+
+// After every layer of the group has packed its rows: clear the marker and empty the tails.
+cudaError_t launch_flush_reset(const Dims& dm, const CacheView& cv, int group, cudaStream_t st) {
+  flush_reset_kernel<<<dm.batch, 32, 0, st>>>(dm, cv, group);
   return cudaGetLastError();
 }
 

@@ -90,7 +90,8 @@ __global__ void __launch_bounds__(kMaxRouteWarps * 32)
 route_score_vote_kernel(Dims dm, int32_t* __restrict__ votes /* [batch][max_chunks][4] of the group */,
                         const __grid_constant__ CUtensorMap map_hidden, int T, const uint16_t* __restrict__ W1,
                         const uint16_t* __restrict__ W2, const float* __restrict__ W3,
-                        const float* __restrict__ bias, long long n_blocks16, int first_chunk, int32_t* status) {
+                        const float* __restrict__ bias, long long n_blocks16, int first_chunk, int32_t* status,
+                        const int32_t* __restrict__ append_after /* nullable: [batch][4] chunk counts */) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   // the swizzled TMA boxes want 1024-byte alignment: round the base up (the launch adds the slack)
   uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -224,7 +225,11 @@ route_score_vote_kernel(Dims dm, int32_t* __restrict__ votes /* [batch][max_chun
       e_lo = argmax4(acc[0] + bs[0], acc[1] + bs[1], o0 + bs[2], o1 + bs[3]);
       e_hi = argmax4(acc[2] + bs[0], acc[3] + bs[1], o2 + bs[2], o3 + bs[3]);
     }
-    int32_t* vrow = votes + (static_cast<long long>(b) * dm.max_chunks + c) * 4;
+    // prefill: the chunk's own row; flush of a full tail: the row after the sequence's last chunk
+    int c_row = c;
+    if (append_after) c_row = append_after[4 * b] + append_after[4 * b + 1] + append_after[4 * b + 2] + append_after[4 * b + 3];
+    if (c_row >= dm.max_chunks) continue;
+    int32_t* vrow = votes + (static_cast<long long>(b) * dm.max_chunks + c_row) * 4;
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
       const unsigned m1 = __ballot_sync(0xffffffffu, t4 == 0 && e_lo == k);
@@ -292,6 +297,39 @@ finalize_map_kernel(Dims dm, CacheView cv, int group, int n_chunks, const uint8_
   }
 }
 
+// flush step 1: clear the vote row the new chunk of every sequence will use
+__global__ void flush_prepare_kernel(Dims dm, int32_t* __restrict__ votes, const int32_t* __restrict__ count_g) {
+  const int b = blockIdx.x;
+  const int c = count_g[4 * b] + count_g[4 * b + 1] + count_g[4 * b + 2] + count_g[4 * b + 3];
+  if (threadIdx.x < 4 && c < dm.max_chunks) votes[(static_cast<long long>(b) * dm.max_chunks + c) * 4 + threadIdx.x] = 0;
+}
+
+// flush step 3: winner of the new chunk, its slot, tables.  A sequence takes part only if the
+// tail of the group's first layer is exactly full.  The map entry carries bit 7 until the
+// chunk's rows have been packed (flush_reset_kernel clears it), which is how the packing
+// kernels know that the sequence is being flushed.
+__global__ void flush_finalize_kernel(Dims dm, CacheView cv, int group) {
+  if (threadIdx.x != 0) return;
+  const int b = blockIdx.x;
+  const int layer0 = group * dm.rs_group;
+  if (cv.tail_len[layer0 * dm.batch + b] != dm.chunk) return;
+  int32_t* count = cv.count + (static_cast<long long>(group) * dm.batch + b) * 4;
+  const int c = count[0] + count[1] + count[2] + count[3];
+  if (c >= dm.max_chunks) { set_status(cv.status, MOQAE_ERR_POOL_FULL, -3, c); return; }
+  const long long base = (static_cast<long long>(group) * dm.batch + b) * dm.max_chunks;
+  const int32_t* v = cv.votes + (base + c) * 4;
+  int w = 0, m = v[0];
+  if (v[1] > m) { m = v[1]; w = 1; }
+  if (v[2] > m) { m = v[2]; w = 2; }
+  if (v[3] > m) { m = v[3]; w = 3; }
+  if (c == 0 && dm.rf_first_chunk) w = 3;                  // routing freezing: the first chunk stays 16-bit
+  const int slot = count[w];
+  if (slot >= cv.capacity[w]) { set_status(cv.status, MOQAE_ERR_POOL_FULL, w, slot); return; }
+  cv.map[base + c] = static_cast<uint8_t>(w | 0x80);
+  cv.slot[base + c] = slot;
+  count[w] = slot + 1;
+}
+
 }  // namespace
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -310,6 +348,56 @@ static EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
+// Launch the scoring + voting kernel over hidden [batch][T][d_in]: chunks first..C-1 of every sequence.
+static cudaError_t launch_score_vote(const Dims& dm, const CacheView& cv, const void* hidden, int T, int first,
+                                     const void* W1, const void* W2, const float* W3, const float* bias,
+                                     int32_t* votes, const int32_t* append_after, cudaStream_t st) {
+  const int C = T / dm.chunk;
+  const long long n_blocks16 = static_cast<long long>(dm.batch) * (C > first ? C - first : 0) * (dm.chunk / 16);
+  if (n_blocks16 <= 0) return cudaSuccess;
+  int dev = 0, sms = 148, smem_max = 0;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+  // [batch*T][d_in] 16-bit tensor, boxes of 64 channels x 16 tokens, 128-byte swizzle
+  EncodeTiledFn enc = encode_tiled_fn();
+  if (!enc) return cudaErrorNotSupported;
+  CUtensorMap map;
+  const cuuint64_t gdim[2] = {static_cast<cuuint64_t>(dm.d_in), static_cast<cuuint64_t>(dm.batch) * T};
+  const cuuint64_t gstride[1] = {static_cast<cuuint64_t>(dm.d_in) * 2};
+  const cuuint32_t box[2] = {kBoxCols, 16};
+  const cuuint32_t estr[2] = {1, 1};
+  if (enc(&map, CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, const_cast<void*>(hidden), gdim, gstride, box, estr,
+          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return cudaErrorInvalidValue;
+  const int n_boxes = (dm.d_in + kBoxCols - 1) / kBoxCols;
+  const size_t wt_bytes = sizeof(uint16_t) * 8 * static_cast<size_t>(n_boxes * kBoxCols + kWPad);
+  // as many warps (each with its own ring) as fit beside the weights, one CTA per SM
+  int warps = kMaxRouteWarps;
+  auto smem_for = [&](int w) { return static_cast<size_t>(w) * kStages * kStageBytes + wt_bytes + 8 * kStages * w + 1024; };
+  while (warps > 1 && smem_for(warps) > static_cast<size_t>(smem_max)) --warps;
+  if (smem_for(warps) > static_cast<size_t>(smem_max)) return cudaErrorInvalidConfiguration;
+  const size_t smem = smem_for(warps);
+  long long want = (n_blocks16 + warps - 1) / warps;
+  const unsigned grid = static_cast<unsigned>(want < sms ? want : sms);
+  cudaError_t e;
+  if (dm.dtype == MOQAE_DTYPE_BF16) {
+    e = cudaFuncSetAttribute(route_score_vote_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (e != cudaSuccess) return e;
+    route_score_vote_kernel<true><<<grid, warps * 32, smem, st>>>(
+        dm, votes, map, T, static_cast<const uint16_t*>(W1), static_cast<const uint16_t*>(W2), W3, bias,
+        n_blocks16, first, cv.status, append_after);
+  } else {
+    e = cudaFuncSetAttribute(route_score_vote_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (e != cudaSuccess) return e;
+    route_score_vote_kernel<false><<<grid, warps * 32, smem, st>>>(
+        dm, votes, map, T, static_cast<const uint16_t*>(W1), static_cast<const uint16_t*>(W2), W3, bias,
+        n_blocks16, first, cv.status, append_after);
+  }
+  return cudaGetLastError();
+}
+
 cudaError_t launch_route(const Dims& dm, const CacheView& cv, const void* hidden, int T, const void* W1,
                          const void* W2, const float* W3, const float* bias, int group,
                          int32_t* votes_out, cudaStream_t st) {
@@ -318,51 +406,8 @@ cudaError_t launch_route(const Dims& dm, const CacheView& cv, const void* hidden
   int32_t* votes = cv.votes + tbl * 4;
   cudaError_t e = cudaMemsetAsync(votes, 0, sizeof(int32_t) * 4 * static_cast<size_t>(dm.batch) * dm.max_chunks, st);
   if (e != cudaSuccess) return e;
-  const int first = dm.rf_first_chunk ? 1 : 0;
-  const long long n_blocks16 = static_cast<long long>(dm.batch) * (C > first ? C - first : 0) * (dm.chunk / 16);
-  if (n_blocks16 > 0) {
-    int dev = 0, sms = 148, smem_max = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
-    // [batch*T][d_in] 16-bit tensor, boxes of 64 channels x 16 tokens, 128-byte swizzle
-    EncodeTiledFn enc = encode_tiled_fn();
-    if (!enc) return cudaErrorNotSupported;
-    CUtensorMap map;
-    const cuuint64_t gdim[2] = {static_cast<cuuint64_t>(dm.d_in), static_cast<cuuint64_t>(dm.batch) * T};
-    const cuuint64_t gstride[1] = {static_cast<cuuint64_t>(dm.d_in) * 2};
-    const cuuint32_t box[2] = {kBoxCols, 16};
-    const cuuint32_t estr[2] = {1, 1};
-    if (enc(&map, CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, const_cast<void*>(hidden), gdim, gstride, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-      return cudaErrorInvalidValue;
-    const int n_boxes = (dm.d_in + kBoxCols - 1) / kBoxCols;
-    const size_t wt_bytes = sizeof(uint16_t) * 8 * static_cast<size_t>(n_boxes * kBoxCols + kWPad);
-    // as many warps (each with its own ring) as fit beside the weights, one CTA per SM
-    int warps = kMaxRouteWarps;
-    auto smem_for = [&](int w) { return static_cast<size_t>(w) * kStages * kStageBytes + wt_bytes + 8 * kStages * w + 1024; };
-    while (warps > 1 && smem_for(warps) > static_cast<size_t>(smem_max)) --warps;
-    if (smem_for(warps) > static_cast<size_t>(smem_max)) return cudaErrorInvalidConfiguration;
-    const size_t smem = smem_for(warps);
-    long long want = (n_blocks16 + warps - 1) / warps;
-    const unsigned grid = static_cast<unsigned>(want < sms ? want : sms);
-    if (dm.dtype == MOQAE_DTYPE_BF16) {
-      e = cudaFuncSetAttribute(route_score_vote_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-      if (e != cudaSuccess) return e;
-      route_score_vote_kernel<true><<<grid, warps * 32, smem, st>>>(
-          dm, votes, map, T, static_cast<const uint16_t*>(W1), static_cast<const uint16_t*>(W2), W3, bias,
-          n_blocks16, first, cv.status);
-    } else {
-      e = cudaFuncSetAttribute(route_score_vote_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-      if (e != cudaSuccess) return e;
-      route_score_vote_kernel<false><<<grid, warps * 32, smem, st>>>(
-          dm, votes, map, T, static_cast<const uint16_t*>(W1), static_cast<const uint16_t*>(W2), W3, bias,
-          n_blocks16, first, cv.status);
-    }
-    e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-  }
+  e = launch_score_vote(dm, cv, hidden, T, dm.rf_first_chunk ? 1 : 0, W1, W2, W3, bias, votes, nullptr, st);
+  if (e != cudaSuccess) return e;
   e = launch_finalize_map(dm, cv, group, C, nullptr, st);
   if (e != cudaSuccess) return e;
   if (votes_out && C > 0) {
@@ -370,6 +415,22 @@ cudaError_t launch_route(const Dims& dm, const CacheView& cv, const void* hidden
                           sizeof(int32_t) * 4 * C, dm.batch, cudaMemcpyDeviceToDevice, st);
   }
   return e;
+}
+
+// ---- flush of a full 16-bit tail: the tail's tokens become one more routed chunk -------------
+cudaError_t launch_flush_route(const Dims& dm, const CacheView& cv, const void* hidden_tail, const void* W1,
+                               const void* W2, const float* W3, const float* bias, int group, cudaStream_t st) {
+  const long long tbl = static_cast<long long>(group) * dm.batch * dm.max_chunks;
+  int32_t* votes = cv.votes + tbl * 4;
+  const int32_t* count_g = cv.count + static_cast<long long>(group) * dm.batch * 4;
+  flush_prepare_kernel<<<dm.batch, 32, 0, st>>>(dm, votes, count_g);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  // the tail is one chunk per sequence: T = chunk, nothing frozen here (chunk 0 is handled below)
+  e = launch_score_vote(dm, cv, hidden_tail, dm.chunk, 0, W1, W2, W3, bias, votes, count_g, st);
+  if (e != cudaSuccess) return e;
+  flush_finalize_kernel<<<dm.batch, 32, 0, st>>>(dm, cv, group);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_finalize_map(const Dims& dm, const CacheView& cv, int group, int n_chunks,
