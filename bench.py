@@ -242,6 +242,22 @@ class Job:
         return route + quant + per_decode * wl.n_layers * wl.decode_steps
 
 
+def max_over_ranks(values, device, world):
+    """Element-wise maximum of `values` over all ranks (replicas share no data: the slowest rank's
+    device time is the job's time).  world == 1: the values themselves."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(v) for v in values], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t.cpu()]
+
+
+def whole_job_gbs(bytes_per_rank, ms, world):
+    """Aggregate throughput of `world` replicas that each move `bytes_per_rank` in at most `ms`."""
+    return world * bytes_per_rank / (ms * 1e6)
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -318,15 +334,12 @@ def run_ours(args):
     else:
         e2e = {"ms_dec": float("nan"), "ms_step": float("nan"), "h2d": 0, "d2h": 0, "steps": 0}
 
-    times = torch.tensor([total_ms, ms_route, ms_quant, ms_dec, e2e["ms_dec"], e2e["ms_step"]],
-                         dtype=torch.float64, device=device)
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    total_ms, ms_route, ms_quant, ms_dec, e2e_ms_dec, e2e_ms_step = [float(x) for x in times.cpu()]
+    total_ms, ms_route, ms_quant, ms_dec, e2e_ms_dec, e2e_ms_step = max_over_ranks(
+        [total_ms, ms_route, ms_quant, ms_dec, e2e["ms_dec"], e2e["ms_step"]], device, world)
 
     if rank == 0:
         peak, peak_kind = read_peaks()
-        dec_gbs = world * b_dec / (ms_dec * 1e6)
+        dec_gbs = whole_job_gbs(b_dec, ms_dec, world)
         per_launch_bytes = b_dec / (wl.n_layers * wl.decode_steps)
         per_launch_ms = ms_dec / (wl.n_layers * wl.decode_steps)
         achieved = per_launch_bytes / (per_launch_ms * 1e6)

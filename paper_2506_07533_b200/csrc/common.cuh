@@ -21,8 +21,6 @@ __host__ __device__ constexpr int bits_of_expert(int w) { return 2 << w; }   // 
 __host__ __device__ constexpr int tile_bytes_of_expert(int w) {
   return w == 3 ? kRawTileBytes : kMetaBytes + 1024 * (2 << w);
 }
-// Cost of one tile in KiB (3, 5, 9, 16): the unit in which decode work is balanced.
-__host__ __device__ constexpr int tile_cost_of_expert(int w) { return tile_bytes_of_expert(w) >> 10; }
 
 // Everything a kernel needs to find its way around a cache (passed by value).
 struct CacheView {
