@@ -452,31 +452,28 @@ struct Pipe {
 // UNIT_BYTES / STAGES are compile-time; src(u, piece) gives each piece's global address.
 template <int STAGES, int STAGE_BYTES, int PIECES, typename SrcFn, typename ConsumeFn>
 __device__ __forceinline__ void stream_units(Pipe& pp, int n_units, int lane, SrcFn src, ConsumeFn consume,
-                                             const uint8_t* ring_generic) {
+                                             const uint8_t* ring_generic, uint32_t last_unit_bytes = STAGE_BYTES) {
   if (n_units <= 0 || !pp.ok) return;
-  constexpr uint32_t piece_bytes = STAGE_BYTES / PIECES;
+  auto issue = [&](int u) {              // lane 0; the last unit of the stream may be shorter
+    const uint32_t bytes = (u == n_units - 1) ? last_unit_bytes : STAGE_BYTES;
+    const uint32_t piece_bytes = bytes / PIECES;
+    const int s = u % STAGES;
+    const uint32_t bar = pp.bars + 8 * s;
+    mbar_expect_tx(bar, bytes);
+#pragma unroll
+    for (int p = 0; p < PIECES; ++p) bulk_load(pp.ring + s * STAGE_BYTES + p * piece_bytes, src(u, p), piece_bytes, bar);
+  };
   if (lane == 0) {
     const int pre = n_units < STAGES ? n_units : STAGES;
-    for (int u = 0; u < pre; ++u) {
-      const uint32_t bar = pp.bars + 8 * u;
-      mbar_expect_tx(bar, STAGE_BYTES);
-#pragma unroll
-      for (int p = 0; p < PIECES; ++p) bulk_load(pp.ring + u * STAGE_BYTES + p * piece_bytes, src(u, p), piece_bytes, bar);
-    }
+    for (int u = 0; u < pre; ++u) issue(u);
   }
   for (int u = 0; u < n_units; ++u) {
     const int s = u % STAGES;
-    const uint32_t bar = pp.bars + 8 * s;
-    if (!mbar_wait_bounded(bar, (pp.parity >> s) & 1u)) { pp.ok = false; return; }
+    if (!mbar_wait_bounded(pp.bars + 8 * s, (pp.parity >> s) & 1u)) { pp.ok = false; return; }
     pp.parity ^= (1u << s);
     consume(ring_generic + s * STAGE_BYTES, u);
     __syncwarp();
-    if (lane == 0 && u + STAGES < n_units) {
-      mbar_expect_tx(bar, STAGE_BYTES);
-#pragma unroll
-      for (int p = 0; p < PIECES; ++p)
-        bulk_load(pp.ring + s * STAGE_BYTES + p * piece_bytes, src(u + STAGES, p), piece_bytes, bar);
-    }
+    if (lane == 0 && u + STAGES < n_units) issue(u + STAGES);
   }
 }
 
@@ -548,18 +545,27 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
 
   // ---- quantised phases
   {
-    const int first = rg.lo[0] + (warp + kWarps - dealt % kWarps) % kWarps;
-    const int n = first < rg.hi[0] ? (rg.hi[0] - first + kWarps - 1) / kWarps : 0;
+    // 2-bit tiles are only 3 KiB: they are fetched in pairs of neighbours (6 KiB per copy, 3 stages),
+    // because the copy engine's cost per request, not HBM, bounds small copies
+    const int n_tiles = rg.hi[0] - rg.lo[0];
+    const int n_pairs = (n_tiles + 1) / 2;
+    const int first = (warp + kWarps - dealt % kWarps) % kWarps;
+    const int n = first < n_pairs ? (n_pairs - first + kWarps - 1) / kWarps : 0;
     if (n > 0) {
-      const uint8_t* stream = slot_ptr(cv, dm, 0, layer, b, h, 0);
+      const uint8_t* stream = slot_ptr(cv, dm, 0, layer, b, h, 0) + static_cast<long long>(rg.lo[0]) * 3072;
+      const bool mine_is_last = (first + (n - 1) * kWarps) == n_pairs - 1;
+      const uint32_t last_bytes = (mine_is_last && (n_tiles & 1)) ? 3072u : 6144u;
       phase_scale<2>(st, true);
       load_q_phase<2>(qb, qc, q_h, g, t4);
-      stream_units<6, 3072, 1>(pp, n, lane,
-          [&](int u, int) { return stream + static_cast<long long>(first + u * kWarps) * 3072; },
-          [&](const uint8_t* tile, int) { process_qtile<2, G4>(tile, st, qc, qb, c_qscore, c_bias, lane); }, my_ring);
+      stream_units<3, 6144, 1>(pp, n, lane,
+          [&](int u, int) { return stream + static_cast<long long>(first + u * kWarps) * 6144; },
+          [&](const uint8_t* tiles, int u) {
+            process_qtile<2, G4>(tiles, st, qc, qb, c_qscore, c_bias, lane);
+            if (u < n - 1 || last_bytes == 6144u) process_qtile<2, G4>(tiles + 3072, st, qc, qb, c_qscore, c_bias, lane);
+          }, my_ring, last_bytes);
       phase_scale<2>(st, false);
     }
-    dealt += rg.hi[0] - rg.lo[0];
+    dealt += n_pairs;
   }
   {
     const int first = rg.lo[1] + (warp + kWarps - dealt % kWarps) % kWarps;
