@@ -12,7 +12,8 @@
 //            (A = 16 tokens x 16 channels of codes, B = folded queries of the GQA group
 //            padded to 8 columns, fp32 accumulate).  The zero-point term is a second MMA
 //            chain with exact fp16 operands (A = z_k, B = q).
-//   softmax  online, base 2, in registers; the 64x offset keeps p*s_v in fp16 range.
+//   softmax  online, base 2, in registers, with a lazily moved reference maximum; weights are
+//            kept <= 64 so that p*s_v stays in fp16 range.
 //   output   out[c][q] = sum_t code[t][c] * (p[t][q] s_v[t][cg]) + sum_t p[t][q] z_v[t][cg]
 //            again with untouched codes as the A operand (A = V^T, 16 channels x 16 tokens:
 //            the value payload stores, per lane, words of 4 tokens of each channel row it
@@ -149,7 +150,11 @@ __device__ __forceinline__ void rescale(State& st, float c0, float c1) {
 }
 
 // Online-softmax update for NV score vectors x[v][4] (d-fragment order: row g q0, row g q1,
-// row g+8 q0, row g+8 q1; already in base-2 units; -inf = masked).  Returns p~ = 64 * p.
+// row g+8 q0, row g+8 q1; already in base-2 units; -inf = masked).  Returns p~ = 2^(6 - kSlack) * p.
+// The reference maximum m is moved lazily: only when some score exceeds it by more than kSlack
+// does the warp reduce the true maximum (three shuffle rounds) and rescale its accumulators;
+// otherwise m stays and the weights are at most 2^6, well inside fp16 either way.
+constexpr float kSlack = 3.0f;
 template <int NV>
 __device__ __forceinline__ void softmax_update(State& st, float x[NV][4]) {
   float mx0 = -INFINITY, mx1 = -INFINITY;
@@ -158,20 +163,20 @@ __device__ __forceinline__ void softmax_update(State& st, float x[NV][4]) {
     mx0 = fmaxf(mx0, fmaxf(x[v][0], x[v][2]));
     mx1 = fmaxf(mx1, fmaxf(x[v][1], x[v][3]));
   }
+  const bool over = (mx0 > st.m[0] + kSlack) || (mx1 > st.m[1] + kSlack);
+  if (__any_sync(0xffffffffu, over)) {
 #pragma unroll
-  for (int o = 4; o <= 16; o <<= 1) {
-    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, o));
-    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, o));
-  }
-  const float n0 = fmaxf(st.m[0], mx0), n1 = fmaxf(st.m[1], mx1);
-  const bool changed = (n0 != st.m[0]) || (n1 != st.m[1]);
-  if (__any_sync(0xffffffffu, changed)) {
+    for (int o = 4; o <= 16; o <<= 1) {
+      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, o));
+      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, o));
+    }
+    const float n0 = fmaxf(st.m[0], mx0), n1 = fmaxf(st.m[1], mx1);
     const float c0 = (st.m[0] == -INFINITY) ? 0.0f : ex2f(st.m[0] - n0);
     const float c1 = (st.m[1] == -INFINITY) ? 0.0f : ex2f(st.m[1] - n1);
     rescale(st, c0, c1);
     st.m[0] = n0; st.m[1] = n1;
   }
-  const float o0 = 6.0f - st.m[0], o1 = 6.0f - st.m[1];
+  const float o0 = (6.0f - kSlack) - st.m[0], o1 = (6.0f - kSlack) - st.m[1];
 #pragma unroll
   for (int v = 0; v < NV; ++v) {
     x[v][0] = ex2f(x[v][0] + o0); x[v][1] = ex2f(x[v][1] + o1);
