@@ -238,7 +238,7 @@ class Job:
         wl = self.wl
         route = 0 if self.forced is not None else 2 * wl.n_groups        # score+vote, finalise
         quant = 2 * wl.n_layers + (wl.n_groups if self.forced is not None else 0)
-        per_decode = 2 + (1 if wl.decode_steps > 1 else 0)                # split-K, combine (+ append)
+        per_decode = 1 + (1 if wl.decode_steps > 1 else 0)                # split-K with fused combine (+ append)
         return route + quant + per_decode * wl.n_layers * wl.decode_steps
 
 
@@ -365,7 +365,7 @@ def run_ours(args):
             "bytes_per_step": {"route": b_route, "quantize_pack": b_quant, "decode_attn": b_dec},
             "gpu_launches": job.launches_per_step() * args.steps,
             "clocks": clocks,
-            "roofline": {"bound": "hbm", "kernel": "decode_mma_kernel (+ decode_combine_kernel)",
+            "roofline": {"bound": "hbm", "kernel": "decode_mma_kernel (split-K partials + combine by the last CTA)",
                          "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
                          "frac": round(achieved / peak, 4), "peak_source": f"of {peak_kind}",
                          "frac_of_8TBs_spec": round(achieved / 8000.0, 4),

@@ -222,7 +222,7 @@ int moqae_decode_attn_workspace(const moqae_config* cfg, int64_t* out_bytes);
  *   q [batch][n_q_heads][128] input dtype; out [batch][n_q_heads][128] float32;
  *   scale <= 0 selects 1/sqrt(128).  An empty cache gives zeros.
  *   workspace: at least moqae_decode_attn_workspace bytes, 16-byte aligned; contents are
- *   scratch (split partials), overwritten by every call.
+ *   scratch (split partials and arrival counters), overwritten by every call.
  */
 int moqae_decode_attn(const moqae_config* cfg, const void* q, int32_t layer,
                       const moqae_cache* cache, float* out, float scale, void* workspace,

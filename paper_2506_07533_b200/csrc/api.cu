@@ -227,8 +227,8 @@ int moqae_decode_attn_workspace(const moqae_config* cfg, int64_t* out_bytes) {
   int rc = check_config(cfg);
   if (rc != MOQAE_OK) return rc;
   if (!out_bytes) return MOQAE_ERR_INVALID_ARG;
-  const int s = moqae::decode_num_splits(dims_of(cfg));
-  *out_bytes = static_cast<int64_t>(cfg->batch) * cfg->n_q_heads * s * (moqae::kHeadDim + 2) * 4;
+  const moqae::Dims dm = dims_of(cfg);
+  *out_bytes = moqae::decode_workspace_bytes(dm, moqae::decode_num_splits(dm));
   return MOQAE_OK;
 }
 
@@ -243,7 +243,7 @@ int moqae_decode_attn(const moqae_config* cfg, const void* q, int32_t layer, con
   if (!aligned16(q) || !aligned16(out) || !aligned16(workspace)) return MOQAE_ERR_MISALIGNED;
   const moqae::Dims dm = dims_of(cfg);
   const int s = moqae::decode_num_splits(dm);
-  const int64_t need = static_cast<int64_t>(cfg->batch) * cfg->n_q_heads * s * (moqae::kHeadDim + 2) * 4;
+  const int64_t need = moqae::decode_workspace_bytes(dm, s);
   if (workspace_bytes < need) return MOQAE_ERR_WORKSPACE_TOO_SMALL;
   if (!(scale > 0.0f)) scale = 0.08838834764831845f;   // 1/sqrt(128)
   cudaError_t e = moqae::launch_decode(dm, cv, q, layer, out, scale, static_cast<float*>(workspace), s,

@@ -494,7 +494,8 @@ __device__ __forceinline__ void load_qraw_rawset(uint32_t (&qr)[16], const uint1
 template <bool BF16, bool G4>
 __global__ void __launch_bounds__(kThreads, 2)
 decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int layer, float scale,
-                  float* __restrict__ ws_o, float* __restrict__ ws_ml, int n_splits) {
+                  float* __restrict__ ws_o, float* __restrict__ ws_ml, int* __restrict__ arrived,
+                  float* __restrict__ out, int n_splits) {
   extern __shared__ __align__(128) uint8_t smem[];
   uint8_t* rings = smem;                                              // kWarps * kRingBytes
   uint16_t* q_in = reinterpret_cast<uint16_t*>(smem + kWarps * kRingBytes);        // [8][128] input dtype
@@ -675,8 +676,32 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
     }
     const long long row = (static_cast<long long>(b) * dm.n_q_heads + h * G + qi) * n_splits + split;
     ws_o[row * kHeadDim + c] = o;
-    // the combine kernel works with natural-log maxima
-    if (c == 0) { ws_ml[row * 2] = m * 0.6931471805599453f; ws_ml[row * 2 + 1] = l; }
+    if (c == 0) { ws_ml[row * 2] = m; ws_ml[row * 2 + 1] = l; }
+  }
+
+  // ---- split combine by the CTA that finishes last for this (sequence, kv head): no second
+  // launch and nobody waits - a counter tells each CTA whether all the others are already done
+  __shared__ int s_last;
+  __threadfence();                       // this CTA's partials are visible device-wide ...
+  __syncthreads();
+  if (threadIdx.x == 0) s_last = (atomicAdd(&arrived[b * dm.n_kv_heads + h], 1) == n_splits - 1) ? 1 : 0;
+  __syncthreads();                       // ... before its arrival is counted
+  if (!s_last) return;
+  __threadfence();
+  for (int i = threadIdx.x; i < G * kHeadDim; i += kThreads) {
+    const int qi = i / kHeadDim, c = i % kHeadDim;
+    const long long row0 = (static_cast<long long>(b) * dm.n_q_heads + h * G + qi) * n_splits;
+    // out = sum_s o_s 2^(m_s - m*) / sum_s l_s 2^(m_s - m*); partials of other CTAs: read through L2
+    float m = -INFINITY;
+    for (int sp = 0; sp < n_splits; ++sp) m = fmaxf(m, __ldcg(ws_ml + (row0 + sp) * 2));
+    float l = 0.0f, o = 0.0f;
+    for (int sp = 0; sp < n_splits; ++sp) {
+      const float ms = __ldcg(ws_ml + (row0 + sp) * 2);
+      const float f = (ms == -INFINITY) ? 0.0f : ex2f(ms - m);
+      l += __ldcg(ws_ml + (row0 + sp) * 2 + 1) * f;
+      o += __ldcg(ws_o + (row0 + sp) * kHeadDim + c) * f;
+    }
+    out[(static_cast<long long>(b) * dm.n_q_heads + h * G + qi) * kHeadDim + c] = l > 0.0f ? o / l : 0.0f;
   }
 }
 
@@ -685,14 +710,14 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
 int decode_mma_ctas_per_sm() { return 2; }
 
 cudaError_t launch_decode_mma(const Dims& dm, const CacheView& cv, const void* q, int layer, float scale,
-                              float* ws_o, float* ws_ml, int n_splits, cudaStream_t st) {
+                              float* ws_o, float* ws_ml, int* arrived, float* out, int n_splits, cudaStream_t st) {
   const size_t smem = static_cast<size_t>(kWarps) * kRingBytes + 2 * kQBytes + kWarps * 6 * 8;
   dim3 grid(n_splits, dm.n_kv_heads, dm.batch);
   const bool g4 = dm.n_q_heads / dm.n_kv_heads <= 4;
   auto launch = [&](auto kernel) -> cudaError_t {
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return e;
-    kernel<<<grid, kThreads, smem, st>>>(dm, cv, static_cast<const uint16_t*>(q), layer, scale, ws_o, ws_ml, n_splits);
+    kernel<<<grid, kThreads, smem, st>>>(dm, cv, static_cast<const uint16_t*>(q), layer, scale, ws_o, ws_ml, arrived, out, n_splits);
     return cudaSuccess;
   };
   cudaError_t e;
