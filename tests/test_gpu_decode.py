@@ -44,7 +44,7 @@ def test_mixed_cache_mha(dtype, from_oracle_cache):
     decode_case(B, T, 4, 4, chunk, dtype, bmap, 40 + dtype, from_oracle_cache)
 
 
-@pytest.mark.parametrize("G", [1, 2, 4, 8])
+@pytest.mark.parametrize("G", [1, 2, 3, 4, 5, 6, 7, 8])
 def test_query_groups(G):
     B, T, chunk, Hkv = 2, 128 * 6 + 5, 128, 2
     rs = np.random.RandomState(G)
@@ -110,3 +110,26 @@ def test_append_then_decode_matches_oracle_with_longer_tail():
         ok, e_abs, e_rel = H.attn_tolerance_ok(out.cpu().numpy(), ref)
         assert ok, (step, e_abs, e_rel)
     assert mq.moqae_poll_status(cache) == 0
+
+
+def test_decode_is_deterministic_and_leaves_neighbours_alone():
+    # same call twice -> identical bits; bytes around `out` are never touched
+    B, T, Hq, Hkv, chunk, dtype = 2, 64 * 5 + 9, 8, 2, 64, 1
+    K, V = H.make_kv(B, T, Hkv, dtype, 95)
+    bmap = np.random.RandomState(95).randint(0, 4, size=(B, T // chunk)).astype(np.uint8)
+    cfg = mq.make_config(n_layers=1, n_q_heads=Hq, n_kv_heads=Hkv, chunk=chunk, dtype=dtype, d_in=64,
+                         max_tokens=T, batch=B)
+    cache = mq.moqae_cache_bind(cfg, [5, 5, 5, 5], zero_pools=True)
+    mq.moqae_quantize_kv(cfg, K.cuda(), V.cuda(), T, 0, cache, forced_map=torch.from_numpy(bmap).cuda())
+    ws = torch.empty(mq.moqae_decode_attn_workspace(cfg), dtype=torch.uint8, device="cuda")
+    q = synth.normal((B, Hq, 128), dtype, 96, "cuda")
+    n = B * Hq * 128
+    buf = torch.full((n + 64,), -7.25, dtype=torch.float32, device="cuda")      # 32 canary floats on either side
+    out = buf[32:32 + n].view(B, Hq, 128)
+    mq.moqae_decode_attn(cfg, q, 0, cache, out, ws)
+    first = out.clone()
+    ws.fill_(0xAB)                                                                # stale scratch must not matter
+    mq.moqae_decode_attn(cfg, q, 0, cache, out, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(first, out)
+    assert (buf[:32] == -7.25).all() and (buf[32 + n:] == -7.25).all()

@@ -118,3 +118,9 @@ def test_routing_sharing_groups_are_independent_tables():
     for g in range(3):
         got = cache.map[g, :, :6].cpu().numpy()
         assert (got == maps[g]).mean() > 0.8 and (got[:, 0] == 3).all()
+
+
+@pytest.mark.parametrize("D", [32, 96, 160, 2080])
+def test_route_input_widths_that_are_not_whole_boxes(D):
+    # the hidden rows arrive in 64-channel boxes: widths below one box and with a ragged last box
+    check_route(2, 64 * 4 + 3, D, 64, 1, True, True, seed=D, w_std=0.1)
