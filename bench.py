@@ -110,7 +110,7 @@ class Job:
 
     N_DISTINCT = 4      # distinct per-layer K/V inputs; layer l reads input l mod 4 (each > L2)
 
-    def __init__(self, wl, device, seed=1234, context=None, force_map=False):
+    def __init__(self, wl, device, seed=1234, context=None, force_map=False, rf=1):
         import torch
 
         from paper_2506_07533_b200 import binding as mq
@@ -120,7 +120,8 @@ class Job:
         B, Hkv, Hq = wl.batch, wl.n_kv_heads, wl.n_q_heads
         self.cfg = mq.make_config(n_layers=wl.n_layers, n_q_heads=Hq, n_kv_heads=Hkv, chunk=wl.chunk,
                                   dtype=wl.dtype, d_in=wl.d_in, max_tokens=T + wl.chunk, batch=B,
-                                  rs_group=wl.rs_group, rf_first_chunk=1, tail_capacity=wl.chunk)
+                                  rs_group=wl.rs_group, rf_first_chunk=rf, tail_capacity=wl.chunk)
+        self.rf = rf
         nd = min(self.N_DISTINCT, wl.n_layers)
         self.kv = [synth.keys_values(B, T, Hkv, 128, wl.dtype, seed + 10 * i, device,
                                      outlier_frac=wl.outlier_frac) for i in range(nd)]
@@ -150,7 +151,8 @@ class Job:
         torch, mq, wl = self.torch, self.mq, self.wl
         C = self.T // wl.chunk
         probe_cfg = mq.make_config(n_layers=1, n_q_heads=wl.n_q_heads, n_kv_heads=wl.n_kv_heads, chunk=wl.chunk,
-                                   dtype=wl.dtype, d_in=wl.d_in, max_tokens=self.T + wl.chunk, batch=wl.batch)
+                                   dtype=wl.dtype, d_in=wl.d_in, max_tokens=self.T + wl.chunk, batch=wl.batch,
+                                   rf_first_chunk=self.rf)
         probe = mq.moqae_cache_bind(probe_cfg, [1, 1, 1, 1], device=self.device)
         target = np.asarray(wl.mix, dtype=np.float64)
         bias = np.zeros(4)
@@ -159,7 +161,7 @@ class Job:
             self.bias.copy_(torch.tensor(bias, dtype=torch.float32))
             mq.moqae_route(probe_cfg, self.hidden[0], self.T, self.W1, self.W2, self.W3, self.bias, 0, probe)
             cnt = probe.count[0].sum(0).cpu().numpy().astype(np.float64)
-            cnt[3] -= wl.batch                      # frozen first chunks are not the router's choice
+            cnt[3] -= wl.batch * self.rf            # frozen first chunks are not the router's choice
             mix = cnt / max(cnt.sum(), 1)
             if np.abs(mix - target).max() <= 0.05:
                 ok = True
@@ -225,7 +227,7 @@ class Job:
         from paper_2506_07533_b200 import workloads as W
         wl, cnt = self.wl, self.counts()
         tail = self.T % wl.chunk
-        route = 0 if self.forced is not None else wl.n_groups * W.route_bytes_per_group(wl, self.T)
+        route = 0 if self.forced is not None else wl.n_groups * W.route_bytes_per_group(wl, self.T, bool(self.rf))
         quant = sum(W.quantize_bytes_per_layer(cnt[l // wl.rs_group], wl, self.T) for l in range(wl.n_layers))
         dec = 0
         for st in range(wl.decode_steps):
@@ -281,9 +283,13 @@ def run_ours(args):
         wl = dataclasses.replace(wl, n_layers=args.layers)
     if args.chunk:
         wl = dataclasses.replace(wl, chunk=args.chunk)
+    if args.batch:
+        wl = dataclasses.replace(wl, batch=args.batch)
+    if args.rs_group:
+        wl = dataclasses.replace(wl, rs_group=args.rs_group)
     if args.mix:
         wl = dataclasses.replace(wl, mix=tuple(float(x) for x in args.mix.split(",")))
-    job = Job(wl, device, seed=1234 + rank, context=args.context, force_map=bool(args.mix))
+    job = Job(wl, device, seed=1234 + rank, context=args.context, force_map=bool(args.mix), rf=0 if args.no_rf else 1)
     torch.cuda.synchronize()
 
     def one_step(ev=None):
@@ -371,7 +377,7 @@ def run_ours(args):
                          "frac_of_8TBs_spec": round(achieved / 8000.0, 4),
                          "bytes_per_launch": int(per_launch_bytes), "ms_per_launch": round(per_launch_ms, 5),
                          "traffic": args.traffic if args.traffic is not None else
-                         (NCU_DECODE_TRAFFIC.get(wl.name) if (args.context is None and args.chunk is None
+                         (NCU_DECODE_TRAFFIC.get(wl.name) if (args.context is None and args.chunk is None and args.batch is None
                                                               and args.mix is None) else None)},
             "roofline_quantize": {"bound": "hbm", "achieved": round(b_quant / (ms_quant * 1e6), 1), "peak": peak,
                                   "unit": "GB/s", "frac": round(b_quant / (ms_quant * 1e6) / peak, 4)},
@@ -535,6 +541,9 @@ def main():
     ap.add_argument("--context", type=int, default=None, help="override the context length (profiling)")
     ap.add_argument("--layers", type=int, default=None, help="override the layer count (profiling)")
     ap.add_argument("--chunk", type=int, default=None, help="override the chunk size (chunk-size sweep)")
+    ap.add_argument("--batch", type=int, default=None, help="override the batch size (context sweeps)")
+    ap.add_argument("--rs-group", type=int, default=None, help="override the routing-sharing group size")
+    ap.add_argument("--no-rf", action="store_true", help="switch routing freezing off (chunk 0 is routed too)")
     ap.add_argument("--mix", default=None,
                     help="four comma-separated shares: skip the router and force a seeded multinomial map "
                          "with this 2/4/8/16-bit mix (e.g. 1,0,0,0 = uniform 2-bit)")
