@@ -527,7 +527,7 @@ def quantize_kv(K_u16: np.ndarray, V_u16: np.ndarray, dtype: int, chunk: int,
     r = T - C * chunk
     tail_k = np.ascontiguousarray(np.transpose(K_u16[:, C * chunk:], (0, 2, 1, 3)))
     tail_v = np.ascontiguousarray(np.transpose(V_u16[:, C * chunk:], (0, 2, 1, 3)))
-    return dict(pools=pools, slot=slot, count=count, capacity=list(capacity),
+    return dict(pools=pools, slot=slot, count=count, capacity=list(capacity), map=np.array(bmap, dtype=np.uint8),
                 tail_k=tail_k, tail_v=tail_v, tail_len=r)
 
 
@@ -622,3 +622,60 @@ def cache_bytes(count: np.ndarray, chunk: int, n_kv_heads: int, tail_len: int) -
             total += int(count[b, w]) * slot_bytes(EXPERT_BITS[w], chunk) * n_kv_heads
         total += tail_len * n_kv_heads * 2 * HEAD_DIM * 2
     return total
+
+
+# ----------------------------------------------------------------------------
+# Prefill attention over the quantised chunks (causal)
+# ----------------------------------------------------------------------------
+def cache_kv_rows_in_order(cache: dict, dtype: int, chunk: int, b: int, h: int):
+    """Cached rows of (sequence b, kv head h) in TOKEN order as float64 K̂, V̂ [T, 128]:
+    chunk c comes from pool map[b, c], slot slot[b, c]; the tail follows."""
+    Ks, Vs = [], []
+    tpc = chunk // TILE_TOKENS
+    C = cache["map"].shape[1]
+    for c in range(C):
+        w = int(cache["map"][b, c])
+        bits = EXPERT_BITS[w]
+        tb = tile_bytes(bits)
+        blob = cache["pools"][w][b, h, int(cache["slot"][b, c])]
+        for j in range(tpc):
+            tile = blob[j * tb:(j + 1) * tb]
+            if bits == 16:
+                Ku, Vu = unpack_raw_tile(tile)
+                Ks.append(to_f64(Ku, dtype))
+                Vs.append(to_f64(Vu, dtype))
+            else:
+                Kh, Vh = dequantize_tile(unpack_tile(tile, bits))
+                Ks.append(Kh)
+                Vs.append(Vh)
+    if cache["tail_len"] > 0:
+        Ks.append(to_f64(cache["tail_k"][b, h, :cache["tail_len"]], dtype))
+        Vs.append(to_f64(cache["tail_v"][b, h, :cache["tail_len"]], dtype))
+    if not Ks:
+        return np.zeros((0, HEAD_DIM)), np.zeros((0, HEAD_DIM))
+    return np.concatenate(Ks, axis=0), np.concatenate(Vs, axis=0)
+
+
+def prefill_attn(q_u16: np.ndarray, dtype: int, cache: dict, chunk: int, scale=None) -> np.ndarray:
+    """Causal attention of every prompt position over the cache built from the same prompt
+    (Section 3.1: the block quantises its chunks, then "proceeds with the formal calculation";
+    Limitations section: keys are dequantised before the product with the query).
+    q_u16 [B, T, H_q, 128] -> float64 out [B, T, H_q, 128]; position t sees the dequantised
+    rows 0..t of kv head h // (H_q / H_kv)."""
+    B, T, Hq, d = q_u16.shape
+    Hkv = cache["pools"][0].shape[1]
+    G = Hq // Hkv
+    if scale is None:
+        scale = 1.0 / np.sqrt(d)
+    q = to_f64(q_u16, dtype)
+    out = np.zeros((B, T, Hq, d))
+    for b in range(B):
+        for h in range(Hkv):
+            K64, V64 = cache_kv_rows_in_order(cache, dtype, chunk, b, h)
+            assert K64.shape[0] == T
+            for g in range(G):
+                s = (q[b, :, h * G + g] @ K64.T) * scale                       # [T, T]
+                s = np.where(np.tri(T, dtype=bool), s, -np.inf)
+                p = np.exp(s - s.max(axis=1, keepdims=True))
+                out[b, :, h * G + g] = (p @ V64) / p.sum(axis=1, keepdims=True)
+    return out
