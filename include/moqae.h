@@ -229,6 +229,22 @@ int moqae_decode_attn(const moqae_config* cfg, const void* q, int32_t layer,
                       int64_t workspace_bytes, void* stream);
 
 /*
+ * Causal attention of the prompt over its own quantised cache (Section 3.1: a block quantises
+ * its chunks, then carries out its attention; Limitations section: keys are dequantised to
+ * 16-bit floats before the product with the query).  For every position t < T and query head h
+ *   out[b][t][h] = softmax(scale * K̂[0..t] q[b][t][h]) V̂[0..t]
+ * over kv head h / (n_q_heads / n_kv_heads), K̂ and V̂ being the cache rows in token order
+ * (chunk c from pool map[c], slot slot[c]; then the 16-bit tail), each rounded to fp16 after
+ * dequantisation; probabilities are rounded to fp16 too, products accumulate in float32.
+ *   q   [batch][T][n_q_heads][128] input dtype;  out [batch][T][n_q_heads][128] float32.
+ *   T must be the number of tokens the cache of `layer` holds for every sequence
+ *   (chunks * chunk + tail_len), i.e. call it after moqae_quantize_kv of the same prompt.
+ *   scale <= 0 selects 1/sqrt(128).
+ */
+int moqae_prefill_attn(const moqae_config* cfg, const void* q, int32_t T, int32_t layer,
+                       const moqae_cache* cache, float* out, float scale, void* stream);
+
+/*
  * (No counterpart in the paper: this entry point exists for deployment reasons only.)
  * moqae_decode_attn for callers that cannot allocate device memory - for example a plug-in
  * inside a server whose device memory is entirely owned by the host application, a control

@@ -25,7 +25,7 @@ ERR_WORKSPACE_TOO_SMALL, ERR_CUDA, ERR_TIMEOUT = -5, -6, -7
 EXPORTS = ["moqae_version", "moqae_last_cuda_error", "moqae_error_string", "moqae_cache_bytes",
            "moqae_cache_bind", "moqae_route", "moqae_quantize_kv", "moqae_append_kv",
            "moqae_decode_attn_workspace", "moqae_decode_attn", "moqae_poll_status",
-           "moqae_decode_attn_static", "moqae_decode_attn_static_max_bytes", "moqae_flush_tail"]
+           "moqae_decode_attn_static", "moqae_decode_attn_static_max_bytes", "moqae_flush_tail", "moqae_prefill_attn"]
 
 
 class MoqaeConfig(C.Structure):
@@ -84,6 +84,8 @@ def lib() -> C.CDLL:
                                       C.POINTER(MoqaeCache), C.c_void_p]
         L.moqae_flush_tail.argtypes = [C.POINTER(MoqaeConfig), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                        C.c_void_p, C.c_int32, C.POINTER(MoqaeCache), C.c_void_p]
+        L.moqae_prefill_attn.argtypes = [C.POINTER(MoqaeConfig), C.c_void_p, C.c_int32, C.c_int32,
+                                         C.POINTER(MoqaeCache), C.c_void_p, C.c_float, C.c_void_p]
         L.moqae_decode_attn_workspace.argtypes = [C.POINTER(MoqaeConfig), C.POINTER(C.c_int64)]
         L.moqae_decode_attn.argtypes = [C.POINTER(MoqaeConfig), C.c_void_p, C.c_int32, C.POINTER(MoqaeCache),
                                         C.c_void_p, C.c_float, C.c_void_p, C.c_int64, C.c_void_p]
@@ -227,6 +229,11 @@ def moqae_append_kv(cfg, k_new, v_new, layer, cache: Cache):
 def moqae_flush_tail(cfg, hidden_tail, W1, W2, W3, bias, layer_group, cache: Cache):
     _check(lib().moqae_flush_tail(C.byref(cfg), _ptr(hidden_tail), _ptr(W1), _ptr(W2), _ptr(W3), _ptr(bias),
                                   int(layer_group), C.byref(cache.view), _stream()), "moqae_flush_tail")
+
+
+def moqae_prefill_attn(cfg, q, T, layer, cache: Cache, out, scale=0.0):
+    _check(lib().moqae_prefill_attn(C.byref(cfg), _ptr(q), int(T), int(layer), C.byref(cache.view), _ptr(out),
+                                    C.c_float(scale), _stream()), "moqae_prefill_attn")
 
 
 def moqae_decode_attn_workspace(cfg) -> int:

@@ -251,6 +251,21 @@ int moqae_decode_attn(const moqae_config* cfg, const void* q, int32_t layer, con
   return e == cudaSuccess ? MOQAE_OK : cuda_fail(e);
 }
 
+int moqae_prefill_attn(const moqae_config* cfg, const void* q, int32_t T, int32_t layer, const moqae_cache* cache,
+                       float* out, float scale, void* stream) {
+  int rc = check_config(cfg);
+  if (rc != MOQAE_OK) return rc;
+  moqae::CacheView cv;
+  rc = check_cache(cache, &cv);
+  if (rc != MOQAE_OK) return rc;
+  if (T < 0 || T > cfg->max_tokens || layer < 0 || layer >= cfg->n_layers) return MOQAE_ERR_INVALID_ARG;
+  if (T > 0 && (!q || !out)) return MOQAE_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(out)) return MOQAE_ERR_MISALIGNED;
+  if (!(scale > 0.0f)) scale = 0.08838834764831845f;   // 1/sqrt(128)
+  cudaError_t e = moqae::launch_prefill_attn(dims_of(cfg), cv, q, T, layer, scale, out, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? MOQAE_OK : cuda_fail(e);
+}
+
 int moqae_poll_status(const moqae_cache* cache, void* stream, int32_t* out_status) {
   if (!cache || !cache->status || !out_status) return MOQAE_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);

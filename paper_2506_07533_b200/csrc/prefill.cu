@@ -1,0 +1,459 @@
+// Causal prefill attention over the quantised chunks (Section 3.1: a block quantises its
+// chunks and then proceeds with its attention; Limitations section: keys are dequantised to
+// 16-bit floats before the product with the query).
+//
+// A dense contraction, so it runs on the 5th-generation tensor cores: one CTA owns 128
+// consecutive query positions of one query head and walks the cache in blocks of 128 tokens
+// (four storage tiles, in token order through the chunk map).  Per block
+//   dequantise   eight warps turn the four packed tiles into fp16 K^ [128 tokens x 128 ch]
+//                (K-major) and V^ [128 x 128] (channel-major) in shared memory, laid out as the
+//                8 x 16-byte core matrices that tcgen05.mma reads without swizzle;
+//   S = Q K^T    8 x tcgen05.mma (M 128, N 128, K 16), fp32 accumulator in tensor memory;
+//   softmax      four warps, one query row per thread, read S with tcgen05.ld, apply the causal
+//                mask, keep the running maximum and sum, write P as fp16 into shared memory;
+//   O_blk = P V^ 8 x tcgen05.mma into a second tensor-memory accumulator, which the same
+//                threads read back and fold into their fp32 output row.
+// Every wait on an mbarrier is bounded; on expiry the CTA records MOQAE_ERR_TIMEOUT, skips the
+// rest of its work and still frees its tensor memory.
+#include <cuda_bf16.h>
+
+#include "common.cuh"
+
+namespace moqae {
+
+namespace {
+
+constexpr int kPThreads = 256;
+constexpr int kQTile = 128;                    // query rows per CTA
+constexpr int kKvBlock = 128;                  // tokens per block (four storage tiles)
+constexpr int kOperandBytes = 128 * 128 * 2;   // one fp16 operand tile
+constexpr int kTmemCols = 256;                 // S: columns 0..127, O block: 128..255
+constexpr long long kWaitLimitP = 1ll << 22;
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ bool mbar_try_wait_p(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
+               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_bounded_p(uint32_t bar, uint32_t parity) {
+  for (long long i = 0; i < kWaitLimitP; ++i)
+    if (mbar_try_wait_p(bar, parity)) return true;
+  return false;
+}
+
+// ---- tcgen05 wrappers -------------------------------------------------------------------
+// Shared-memory matrix descriptor, no swizzle: start address, leading-dimension byte offset
+// (between the two 8-element halves of a K step, or between groups of 8 K rows for an
+// MN-major operand) and stride byte offset (between groups of 8 rows / of 8 MN elements), all
+// in units of 16 bytes; bits 46..47 = 1 is the descriptor version of this architecture.
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  return static_cast<uint64_t>((saddr >> 4) & 0x3fffu) | (static_cast<uint64_t>((lbo_bytes >> 4) & 0x3fffu) << 16) |
+         (static_cast<uint64_t>((sbo_bytes >> 4) & 0x3fffu) << 32) | (1ull << 46);
+}
+// Instruction descriptor of kind::f16: fp32 accumulator, fp16 A and B, M = 128, N = 128;
+// bit 16 set = B is MN-major (its N index is the contiguous one).
+constexpr uint32_t kIdescKK = (1u << 4) | (16u << 17) | (8u << 24);
+constexpr uint32_t kIdescKMN = kIdescKK | (1u << 16);
+
+__device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+               "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+               ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory"); }
+__device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory"); }
+
+// 32 consecutive fp32 columns of this thread's tensor-memory lane
+__device__ __forceinline__ void tmem_ld32(float (&v)[32], uint32_t taddr) {
+  uint32_t r[32];
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+               "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+               "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                 "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                 "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                 "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+               : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// ---- operand tiles in shared memory -------------------------------------------------------
+// K-major operand (Q, K^, P): element (row n, k) of a 128 x 128 fp16 tile.  Core matrix =
+// 8 rows x 8 elements (128 bytes); the 16 core matrices of one 8-element K slab are
+// contiguous (stride 128 B between row groups), K slabs follow each other (2048 B).
+__device__ __forceinline__ int kmajor_unit_offset(int n, int k8) {       // byte offset of the 16-byte unit (n, k8*8..+7)
+  return (k8 * 16 + (n >> 3)) * 128 + (n & 7) * 16;
+}
+// MN-major operand (V^: rows = tokens (K of the MMA), contiguous index = channels): core
+// matrix = 8 tokens x 8 channels; the 16 channel groups of one 8-token slab are contiguous.
+__device__ __forceinline__ int mnmajor_unit_offset(int t, int c8) {      // byte offset of the 16-byte unit (t, c8*8..+7)
+  return ((t >> 3) * 16 + c8) * 128 + (t & 7) * 16;
+}
+
+__device__ __forceinline__ uint32_t pack_h2(float a, float b) {
+  const __half2 h = __floats2half2_rn(a, b);
+  return *reinterpret_cast<const uint32_t*>(&h);
+}
+// eight 16-bit inputs (one uint4) -> eight fp16
+template <bool BF16> __device__ __forceinline__ uint4 to_fp16x8(uint4 v) {
+  if (!BF16) return v;
+  uint4 o;
+  o.x = pack_h2(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xffff0000u));
+  o.y = pack_h2(__uint_as_float(v.y << 16), __uint_as_float(v.y & 0xffff0000u));
+  o.z = pack_h2(__uint_as_float(v.z << 16), __uint_as_float(v.z & 0xffff0000u));
+  o.w = pack_h2(__uint_as_float(v.w << 16), __uint_as_float(v.w & 0xffff0000u));
+  return o;
+}
+__device__ __forceinline__ float h_lo(uint32_t w) { return __low2float(*reinterpret_cast<const __half2*>(&w)); }
+__device__ __forceinline__ float h_hi(uint32_t w) { return __high2float(*reinterpret_cast<const __half2*>(&w)); }
+
+// ---- dequantisation of one 32-token storage tile into the operand tiles --------------------
+// The packed layout is the one the decode kernel's lanes consume (lane = 4g + t4); the same
+// 16-byte units are read here, straight from global memory, and expanded to fp16.
+template <int BITS> __host__ __device__ constexpr int key_reg_channel_lo(int r) {
+  constexpr int n = 32 / BITS;
+  return (r / (n / 2)) * n + ((r % (n / 2)) / (n / 4)) * (n / 4) + r % (n / 4);
+}
+
+template <int BITS>
+__device__ __forceinline__ void dequant_keys(const uint8_t* __restrict__ tile, uint8_t* sK, int sub, int lane) {
+  constexpr int n = 32 / BITS;
+  constexpr uint32_t mask = (1u << BITS) - 1u;
+  const int g = lane >> 2, t4 = lane & 3;
+  float sc[32], zr[32];                    // scale and zero of channels 32*t4 .. +31
+  {
+    const uint4* sp = reinterpret_cast<const uint4*>(tile) + t4;
+    const uint4* zp = reinterpret_cast<const uint4*>(tile + 256) + t4;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const uint4 s4 = __ldg(sp + 4 * i), z4 = __ldg(zp + 4 * i);
+      const uint32_t sw[4] = {s4.x, s4.y, s4.z, s4.w};
+      const uint32_t zw[4] = {z4.x, z4.z, z4.y, z4.w};     // zeros are stored in register order 0, 2, 1, 3
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int cl = key_reg_channel_lo<BITS>(4 * i + j);
+        sc[cl] = h_lo(sw[j]); sc[cl + n / 2] = h_hi(sw[j]);
+        zr[cl] = h_lo(zw[j]); zr[cl + n / 2] = h_hi(zw[j]);
+      }
+    }
+  }
+  const uint8_t* kpay = tile + kMetaBytes;
+#pragma unroll
+  for (int blk = 0; blk < 2; ++blk)
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+      uint32_t w[BITS];
+      if (BITS == 2) {
+        const uint4 v = __ldg(reinterpret_cast<const uint4*>(kpay + (blk * 32 + lane) * 16));
+        w[0] = hh ? v.z : v.x; w[1] = hh ? v.w : v.y;
+      } else if (BITS == 4) {
+        const uint4 v = __ldg(reinterpret_cast<const uint4*>(kpay + ((2 * blk + hh) * 32 + lane) * 16));
+        w[0] = v.x; w[1] = v.y; w[2 % BITS] = v.z; w[3 % BITS] = v.w;
+      } else {
+#pragma unroll
+        for (int j2 = 0; j2 < 2; ++j2) {
+          const uint4 v = __ldg(reinterpret_cast<const uint4*>(kpay + (((2 * blk + hh) * 2 + j2) * 32 + lane) * 16));
+          w[(4 * j2) % BITS] = v.x; w[(4 * j2 + 1) % BITS] = v.y; w[(4 * j2 + 2) % BITS] = v.z; w[(4 * j2 + 3) % BITS] = v.w;
+        }
+      }
+      const int row = 32 * sub + 16 * blk + 8 * hh + g;
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        float v[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const int cc = 8 * u + e;
+          const uint32_t code = (w[(cc * BITS) >> 5] >> ((cc * BITS) & 31)) & mask;
+          v[e] = fmaf(static_cast<float>(code), sc[cc], zr[cc]);
+        }
+        *reinterpret_cast<uint4*>(sK + kmajor_unit_offset(row, 4 * t4 + u)) =
+            make_uint4(pack_h2(v[0], v[1]), pack_h2(v[2], v[3]), pack_h2(v[4], v[5]), pack_h2(v[6], v[7]));
+      }
+    }
+}
+
+template <int BITS>
+__device__ __forceinline__ void dequant_values(const uint8_t* __restrict__ tile, uint8_t* sV, int sub, int lane) {
+  constexpr uint32_t mask = (1u << BITS) - 1u;
+  constexpr int per = 8 / BITS;                                   // channel rows per word
+  const int g = lane >> 2, t4 = lane & 3;
+  const uint8_t* vpay = tile + kMetaBytes + kTileTokens * 16 * BITS;
+#pragma unroll
+  for (int blk = 0; blk < 2; ++blk) {
+    uint32_t sw[4][2], zw[4][2];                                  // [channel group][half]: fp16 pair (e = 0, 1)
+#pragma unroll
+    for (int cp = 0; cp < 2; ++cp) {
+      const uint4 s4 = __ldg(reinterpret_cast<const uint4*>(tile + 512 + ((blk * 2 + cp) * 4 + t4) * 16));
+      sw[2 * cp][0] = s4.x; sw[2 * cp][1] = s4.y; sw[2 * cp + 1][0] = s4.z; sw[2 * cp + 1][1] = s4.w;
+    }
+#pragma unroll
+    for (int cg = 0; cg < 4; ++cg) {
+      const uint2 z2 = __ldg(reinterpret_cast<const uint2*>(tile + 768 + ((blk * 4 + cg) * 4 + t4) * 8));
+      zw[cg][0] = z2.x; zw[cg][1] = z2.y;
+    }
+    uint32_t wv[2 * BITS];
+#pragma unroll
+    for (int u = 0; u < BITS / 2; ++u) {
+      const uint4 v = __ldg(reinterpret_cast<const uint4*>(vpay + ((blk * (BITS / 2) + u) * 32 + lane) * 16));
+      wv[4 * u] = v.x; wv[4 * u + 1] = v.y; wv[4 * u + 2] = v.z; wv[4 * u + 3] = v.w;
+    }
+#pragma unroll
+    for (int cg = 0; cg < 4; ++cg)
+#pragma unroll
+      for (int half = 0; half < 2; ++half)
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const float s = e ? h_hi(sw[cg][half]) : h_lo(sw[cg][half]);
+          const float z = e ? h_hi(zw[cg][half]) : h_lo(zw[cg][half]);
+          float v[4];
+#pragma unroll
+          for (int r4 = 0; r4 < 4; ++r4) {
+            const int R = 4 * cg + r4;
+            const uint32_t code = (wv[R / per] >> (BITS * (R % per) + 8 * half + 16 * e)) & mask;
+            v[r4] = fmaf(static_cast<float>(code), s, z);
+          }
+          const int tok = 32 * sub + 16 * blk + 8 * half + 2 * t4 + e;
+          // channels 32cg + 4g .. +3: half of the 16-byte unit c8 = 4cg + g/2
+          *reinterpret_cast<uint2*>(sV + mnmajor_unit_offset(tok, 4 * cg + (g >> 1)) + (g & 1) * 8) =
+              make_uint2(pack_h2(v[0], v[1]), pack_h2(v[2], v[3]));
+        }
+  }
+}
+
+// 32 rows of 256 bytes in the input dtype -> one operand tile.  SWIZZLED: rows of a 16-bit
+// pool tile (units permuted inside each row); otherwise plain rows (the tail), of which only
+// the first n_valid exist.
+template <bool BF16, bool SWIZZLED, bool IS_V>
+__device__ __forceinline__ void copy_rows(const uint8_t* __restrict__ src, uint8_t* dst, int sub, int n_valid, int lane) {
+#pragma unroll 4
+  for (int i = 0; i < 16; ++i) {
+    const int idx = i * 32 + lane;
+    const int row = idx >> 4, U = idx & 15;
+    const int up = SWIZZLED ? ((U & 8) | ((U ^ row) & 7)) : U;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (row < n_valid) v = to_fp16x8<BF16>(__ldg(reinterpret_cast<const uint4*>(src + row * 256 + up * 16)));
+    const int off = IS_V ? mnmajor_unit_offset(32 * sub + row, U) : kmajor_unit_offset(32 * sub + row, U);
+    *reinterpret_cast<uint4*>(dst + off) = v;
+  }
+}
+
+template <bool BF16>
+__global__ void __launch_bounds__(kPThreads, 1)
+prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T, int layer, float scale_log2,
+                    float* __restrict__ out) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  uint8_t* sQ = smem;
+  uint8_t* sK = smem + kOperandBytes;
+  uint8_t* sV = smem + 2 * kOperandBytes;
+  uint8_t* sP = smem + 3 * kOperandBytes;
+  uint64_t* bar_mem = reinterpret_cast<uint64_t*>(smem + 4 * kOperandBytes);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_mem + 1);
+  const uint32_t bar = smem_addr(bar_mem);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int qt = blockIdx.x, hq = blockIdx.y, b = blockIdx.z;
+  const int H = dm.n_kv_heads, Hq = dm.n_q_heads;
+  const int h = hq / (Hq / H);
+  const int q0 = qt * kQTile;
+
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_addr(tmem_slot)), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+  }
+  if (tid == 0) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;\n" ::"r"(bar) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+  }
+  // the CTA's 128 query rows as the A operand (rows past the prompt are zero)
+  for (int i = tid; i < kQTile * 16; i += kPThreads) {
+    const int row = i >> 4, U = i & 15;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (q0 + row < T)
+      v = to_fp16x8<BF16>(__ldg(reinterpret_cast<const uint4*>(Q + ((static_cast<long long>(b) * T + q0 + row) * Hq + hq) * kHeadDim + 8 * U)));
+    *reinterpret_cast<uint4*>(sQ + kmajor_unit_offset(row, U)) = v;
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  // where the cache of this (layer, sequence, kv head) lives
+  const int group = layer / dm.rs_group;
+  const long long tbl = (static_cast<long long>(group) * dm.batch + b) * dm.max_chunks;
+  const int32_t* cnt = cv.count + (static_cast<long long>(group) * dm.batch + b) * 4;
+  const int n_chunks = min(cnt[0] + cnt[1] + cnt[2] + cnt[3], dm.max_chunks);
+  const int chunk_tokens = n_chunks * dm.chunk;
+  const int tail_len = min(cv.tail_len[layer * dm.batch + b], dm.tail_capacity);
+  const int tpc = dm.chunk / kTileTokens;
+  const long long tail_base = ((static_cast<long long>(layer) * dm.batch + b) * H + h) * dm.tail_capacity;   // rows
+
+  const uint32_t aQ = smem_addr(sQ), aK = smem_addr(sK), aV = smem_addr(sV), aP = smem_addr(sP);
+  const int row = tid & 127;                                  // query row of a softmax thread (warps 0..3)
+  const int qpos = q0 + row;
+  const uint32_t lane_addr = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+  float o[kHeadDim];
+#pragma unroll
+  for (int c = 0; c < kHeadDim; ++c) o[c] = 0.0f;
+  float m = -INFINITY, l = 0.0f, corr = 1.0f;
+  uint32_t phase = 0;
+  bool ok = true;
+
+  for (int kb = 0; kb <= qt; ++kb) {
+    // ---- dequantise: warp w takes storage tile (w & 3) of the block, keys (w < 4) or values
+    {
+      const int sub = warp & 3;
+      const bool is_v = warp >= 4;
+      const int pos0 = kb * kKvBlock + sub * kTileTokens;
+      if (pos0 < chunk_tokens) {
+        const int c = pos0 / dm.chunk, j = (pos0 % dm.chunk) / kTileTokens;
+        const int w = cv.map[tbl + c] & 3;
+        const long long slot = cv.slot[tbl + c];
+        long long cap = 0;
+        const uint8_t* pool = nullptr;
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          if (w == k) { cap = cv.capacity[k]; pool = cv.pool[k]; }
+        const long long tb = tile_bytes_of_expert(w);
+        const uint8_t* tile = pool + ((((static_cast<long long>(layer) * dm.batch + b) * H + h) * cap + min(slot, cap - 1)) * tpc + j) * tb;
+        if (w == 0) { if (is_v) dequant_values<2>(tile, sV, sub, lane); else dequant_keys<2>(tile, sK, sub, lane); }
+        else if (w == 1) { if (is_v) dequant_values<4>(tile, sV, sub, lane); else dequant_keys<4>(tile, sK, sub, lane); }
+        else if (w == 2) { if (is_v) dequant_values<8>(tile, sV, sub, lane); else dequant_keys<8>(tile, sK, sub, lane); }
+        else if (is_v) copy_rows<BF16, true, true>(tile + 8192, sV, sub, 32, lane);
+        else copy_rows<BF16, true, false>(tile, sK, sub, 32, lane);
+      } else {
+        const int ti0 = pos0 - chunk_tokens;
+        const int n_valid = max(0, min(32, tail_len - ti0));
+        const uint8_t* src = reinterpret_cast<const uint8_t*>(is_v ? cv.tail_v : cv.tail_k) + (tail_base + ti0) * 256;
+        if (is_v) copy_rows<BF16, false, true>(src, sV, sub, n_valid, lane);
+        else copy_rows<BF16, false, false>(src, sK, sub, n_valid, lane);
+      }
+    }
+    fence_async_proxy();                   // generic-proxy writes of the operand tiles -> visible to the MMA
+    tc_fence_before();
+    __syncthreads();
+    // ---- S = Q K^T
+    if (tid == 0) {
+      tc_fence_after();
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks)
+        umma_f16(tmem, make_desc(aQ + ks * 4096, 2048, 128), make_desc(aK + ks * 4096, 2048, 128), kIdescKK, ks > 0);
+      umma_commit(bar);
+    }
+    // ---- softmax of the block, one query row per thread
+    if (warp < 4) {
+      if (ok && !mbar_wait_bounded_p(bar, phase)) ok = false;
+      phase ^= 1u;
+      tc_fence_after();
+      float mx = -INFINITY;
+      if (ok) {
+#pragma unroll 1
+        for (int c4 = 0; c4 < 4; ++c4) {
+          float v[32];
+          tmem_ld32(v, lane_addr + 32 * c4);
+#pragma unroll
+          for (int i = 0; i < 32; ++i)
+            if (kb * kKvBlock + 32 * c4 + i <= qpos) mx = fmaxf(mx, v[i] * scale_log2);
+        }
+      }
+      const float m_new = fmaxf(m, mx);
+      corr = (m == -INFINITY) ? 0.0f : exp2f(m - m_new);
+      l *= corr;
+#pragma unroll 1
+      for (int c4 = 0; c4 < 4; ++c4) {
+        float v[32];
+        if (ok) tmem_ld32(v, lane_addr + 32 * c4);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          uint32_t pk[4];
+#pragma unroll
+          for (int e2 = 0; e2 < 4; ++e2) {
+            float p2[2];
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+              const int i = 8 * u + 2 * e2 + e;
+              const bool seen = ok && (kb * kKvBlock + 32 * c4 + i <= qpos) && m_new > -INFINITY;
+              p2[e] = seen ? exp2f(v[i] * scale_log2 - m_new) : 0.0f;
+            }
+            pk[e2] = pack_h2(p2[0], p2[1]);
+            l += h_lo(pk[e2]) + h_hi(pk[e2]);             // the sum uses the weights the MMA will see
+          }
+          *reinterpret_cast<uint4*>(sP + kmajor_unit_offset(row, 4 * c4 + u)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        }
+      }
+      m = m_new;
+      fence_async_proxy();
+      tc_fence_before();
+    }
+    __syncthreads();
+    // ---- O_blk = P V^ (fresh accumulator), folded into the threads' fp32 rows
+    if (tid == 0) {
+      tc_fence_after();
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks)
+        umma_f16(tmem + 128, make_desc(aP + ks * 4096, 2048, 128), make_desc(aV + ks * 4096, 2048, 128), kIdescKMN, ks > 0);
+      umma_commit(bar);
+    }
+    if (warp < 4) {
+      if (ok && !mbar_wait_bounded_p(bar, phase)) ok = false;
+      phase ^= 1u;
+      tc_fence_after();
+      if (ok) {
+#pragma unroll
+        for (int c4 = 0; c4 < 4; ++c4) {
+          float v[32];
+          tmem_ld32(v, lane_addr + 128 + 32 * c4);
+#pragma unroll
+          for (int i = 0; i < 32; ++i) o[32 * c4 + i] = fmaf(o[32 * c4 + i], corr, v[i]);
+        }
+      }
+      tc_fence_before();
+    }
+    __syncthreads();
+  }
+
+  if (warp < 4) {
+    if (!ok && lane == 0) set_status(cv.status, MOQAE_ERR_TIMEOUT, blockIdx.x, warp);
+    if (qpos < T) {
+      const float inv = l > 0.0f ? 1.0f / l : 0.0f;
+      float4* dst = reinterpret_cast<float4*>(out + ((static_cast<long long>(b) * T + qpos) * Hq + hq) * kHeadDim);
+#pragma unroll
+      for (int c = 0; c < kHeadDim; c += 4) dst[c >> 2] = make_float4(o[c] * inv, o[c + 1] * inv, o[c + 2] * inv, o[c + 3] * inv);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(kTmemCols) : "memory");
+}
+
+}  // namespace
+
+cudaError_t launch_prefill_attn(const Dims& dm, const CacheView& cv, const void* q, int T, int layer, float scale,
+                                float* out, cudaStream_t st) {
+  if (T <= 0) return cudaSuccess;
+  const size_t smem = 4 * kOperandBytes + 16;
+  dim3 grid((T + kQTile - 1) / kQTile, dm.n_q_heads, dm.batch);
+  const float scale_log2 = scale * 1.4426950408889634f;
+  cudaError_t e;
+  if (dm.dtype == MOQAE_DTYPE_BF16) {
+    e = cudaFuncSetAttribute(prefill_attn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (e != cudaSuccess) return e;
+    prefill_attn_kernel<true><<<grid, kPThreads, smem, st>>>(dm, cv, static_cast<const uint16_t*>(q), T, layer, scale_log2, out);
+  } else {
+    e = cudaFuncSetAttribute(prefill_attn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (e != cudaSuccess) return e;
+    prefill_attn_kernel<false><<<grid, kPThreads, smem, st>>>(dm, cv, static_cast<const uint16_t*>(q), T, layer, scale_log2, out);
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace moqae
