@@ -390,12 +390,40 @@ def run_ours(args):
                     "note": "host-resident hidden, K, V, q copied in and out read back inside the timed step; "
                             "value = decode-phase bytes / (decode phase incl. q upload and out download)"},
         }
+        if args.prefill_attn:
+            line["prefill_attn"] = measure_prefill_attn(job, torch)
         if not args.no_cpu_baseline and world == 1:
             line["cpu_baseline"] = cpu_baseline(wl, budget_s=args.cpu_seconds)
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
+
+
+def measure_prefill_attn(job, torch, reps=3):
+    """Causal prefill attention of layer 0 over its quantised cache (tensor-core bound): device time of
+    `reps` launches after one warm-up; FLOPs = 2 products x 2 x 128 x (T (T + 1) / 2) per query head."""
+    wl, T = job.wl, job.T
+    q = job.torch.randn(wl.batch, T, wl.n_q_heads, 128, device=job.device, dtype=torch.float32)
+    q = q.to(torch.bfloat16 if wl.dtype == 1 else torch.float16)
+    out = torch.empty((wl.batch, T, wl.n_q_heads, 128), dtype=torch.float32, device=job.device)
+    job.mq.moqae_prefill_attn(job.cfg, q, T, 0, job.cache, out)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    ev[0].record()
+    for _ in range(reps):
+        job.mq.moqae_prefill_attn(job.cfg, q, T, 0, job.cache, out)
+    ev[1].record()
+    torch.cuda.synchronize()
+    ms = ev[0].elapsed_time(ev[1]) / reps
+    flops = 4.0 * 128 * (T * (T + 1) / 2) * wl.n_q_heads * wl.batch
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            peak, src = float(json.load(f)["bf16_tflops"]), "of measured"
+    except Exception:
+        peak, src = 1590.0, "of fallback"
+    tf = flops / (ms * 1e9)
+    return {"ms": round(ms, 3), "tflops": round(tf, 1), "bound": "tensor", "peak": peak, "frac": round(tf / peak, 4),
+            "peak_source": src, "flops": flops, "status": job.mq.moqae_poll_status(job.cache)}
 
 
 def measure_e2e(job, args, torch):
@@ -543,6 +571,8 @@ def main():
     ap.add_argument("--chunk", type=int, default=None, help="override the chunk size (chunk-size sweep)")
     ap.add_argument("--batch", type=int, default=None, help="override the batch size (context sweeps)")
     ap.add_argument("--rs-group", type=int, default=None, help="override the routing-sharing group size")
+    ap.add_argument("--prefill-attn", action="store_true",
+                    help="also time the causal prefill attention of layer 0 over its quantised cache")
     ap.add_argument("--no-rf", action="store_true", help="switch routing freezing off (chunk 0 is routed too)")
     ap.add_argument("--mix", default=None,
                     help="four comma-separated shares: skip the router and force a seeded multinomial map "
