@@ -2,19 +2,22 @@
 // chunks and then proceeds with its attention; Limitations section: keys are dequantised to
 // 16-bit floats before the product with the query).
 //
-// A dense contraction, so it runs on the 5th-generation tensor cores: one CTA owns 128
-// consecutive query positions of one query head and walks the cache in blocks of 128 tokens
-// (four storage tiles, in token order through the chunk map).  Per block
-//   dequantise   eight warps turn the four packed tiles into fp16 K^ [128 tokens x 128 ch]
+// A dense contraction, so it runs on the 5th-generation tensor cores: one CTA owns 256
+// consecutive query positions (two tiles of 128) of one query head and walks the cache in
+// blocks of 128 tokens (four storage tiles, in token order through the chunk map).  Per block
+//   dequantise   four warps turn the four packed tiles into fp16 K^ [128 tokens x 128 ch]
 //                (K-major) and V^ [128 x 128] (channel-major) in shared memory, laid out as the
-//                8 x 16-byte core matrices that tcgen05.mma reads without swizzle;
-//   S = Q K^T    8 x tcgen05.mma (M 128, N 128, K 16), fp32 accumulator in tensor memory;
-//   softmax      four warps, one query row per thread, read S with tcgen05.ld, apply the causal
-//                mask, keep the running maximum and sum, write P as fp16 into shared memory;
-//   O_blk = P V^ 8 x tcgen05.mma into a second tensor-memory accumulator, which the same
-//                threads read back and fold into their fp32 output row.
-// Every wait on an mbarrier is bounded; on expiry the CTA records MOQAE_ERR_TIMEOUT, skips the
-// rest of its work and still frees its tensor memory.
+//                8 x 16-byte core matrices that tcgen05.mma reads without swizzle; K^ of the
+//                next block is produced while the softmax of this one runs;
+//   S_i = Q_i K^T  8 x tcgen05.mma (M 128, N 128, K 16) per query tile, fp32 in tensor memory;
+//   softmax      eight warps, one query row per thread, read S_i with tcgen05.ld, apply the
+//                causal mask, keep a lazily moved reference maximum and the running sum, write
+//                P_i as fp16 into shared memory;
+//   O_i += P_i V^  8 x tcgen05.mma accumulating in tensor memory across blocks (rescaled in place
+//                on the rare blocks where the reference maximum moves).
+// The three roles (softmax, dequantise, MMA issue) run concurrently and meet on mbarriers only.
+// Every wait is bounded; on expiry the CTA records MOQAE_ERR_TIMEOUT, every role stops and the
+// tensor memory is still freed.
 #include <cuda_bf16.h>
 
 #include "common.cuh"
@@ -23,11 +26,9 @@ namespace moqae {
 
 namespace {
 
-constexpr int kPThreads = 256;
 constexpr int kQTile = 128;                    // query rows per CTA
 constexpr int kKvBlock = 128;                  // tokens per block (four storage tiles)
 constexpr int kOperandBytes = 128 * 128 * 2;   // one fp16 operand tile
-constexpr int kTmemCols = 256;                 // S: columns 0..127, O block: 128..255
 constexpr long long kWaitLimitP = 1ll << 22;
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) {
@@ -39,12 +40,6 @@ __device__ __forceinline__ bool mbar_try_wait_p(uint32_t bar, uint32_t parity) {
                : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-__device__ __forceinline__ bool mbar_wait_bounded_p(uint32_t bar, uint32_t parity) {
-  for (long long i = 0; i < kWaitLimitP; ++i)
-    if (mbar_try_wait_p(bar, parity)) return true;
-  return false;
-}
-
 // ---- tcgen05 wrappers -------------------------------------------------------------------
 // Shared-memory matrix descriptor, no swizzle: start address, leading-dimension byte offset
 // (between the two 8-element halves of a K step, or between groups of 8 K rows for an
@@ -247,192 +242,294 @@ __device__ __forceinline__ void copy_rows(const uint8_t* __restrict__ src, uint8
   }
 }
 
+// ---- the kernel ----------------------------------------------------------------------------
+// Roles (13 warps): warps 0..3 and 4..7 are the softmax threads of the CTA's two query tiles
+// (one row each, tensor-memory lane = tid % 128); warps 8..11 dequantise (one storage tile
+// each: keys of block kb, then values of block kb); warp 12 issues the MMAs.  They meet
+// only on mbarriers:
+//   kfull / vfull     K^ / V^ of a block are in shared memory            (4 dequant warps)
+//   sfull[i]          S_i = Q_i K^T is in tensor memory                  (tcgen05.commit)
+//   pfull[i]          P_i is in shared memory and S_i has been read      (4 softmax warps)
+//   ofull[i]          O_i += P_i V^ is done                              (tcgen05.commit)
+// K^ is free again when sfull[1] completes, V^ when ofull[1] completes.  Every barrier
+// completes once per block, so completion number kb is awaited with parity kb & 1.
+constexpr int kSoftmaxWarps = 8, kDequantWarps = 4;
+constexpr int kP2Threads = (kSoftmaxWarps + kDequantWarps + 1) * 32;
+constexpr int kTmemCols2 = 512;                // S_0, S_1, O_0, O_1: 128 columns each
+constexpr float kRescaleSlack = 8.0f;          // base-2 units: weights stay below 2^8
+
+enum { BAR_KFULL = 0, BAR_VFULL, BAR_SFULL0, BAR_SFULL1, BAR_PFULL0, BAR_PFULL1, BAR_OFULL0, BAR_OFULL1, BAR_COUNT };
+
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+               "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+               "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};\n"
+               ::"r"(taddr),
+                 "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])), "r"(__float_as_uint(v[3])),
+                 "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])), "r"(__float_as_uint(v[7])),
+                 "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])), "r"(__float_as_uint(v[11])),
+                 "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15])),
+                 "r"(__float_as_uint(v[16])), "r"(__float_as_uint(v[17])), "r"(__float_as_uint(v[18])), "r"(__float_as_uint(v[19])),
+                 "r"(__float_as_uint(v[20])), "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])), "r"(__float_as_uint(v[23])),
+                 "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])), "r"(__float_as_uint(v[26])), "r"(__float_as_uint(v[27])),
+                 "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31]))
+               : "memory");
+  asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory");
+}
+
+// Where the cache of one (layer, sequence, kv head) lives, and how to reach a 32-token tile of it.
+struct KvSource {
+  const CacheView* cv;
+  const Dims* dm;
+  long long tbl, tail_base;
+  int layer, b, h, chunk_tokens, tail_len, tpc;
+};
+
 template <bool BF16>
-__global__ void __launch_bounds__(kPThreads, 1)
+__device__ __forceinline__ void dequant_subtile(const KvSource& ks, int pos0, int sub, bool is_v, uint8_t* dst, int lane) {
+  const CacheView& cv = *ks.cv;
+  const Dims& dm = *ks.dm;
+  if (pos0 < ks.chunk_tokens) {
+    const int c = pos0 / dm.chunk, j = (pos0 % dm.chunk) / kTileTokens;
+    const int w = cv.map[ks.tbl + c] & 3;
+    const long long slot = cv.slot[ks.tbl + c];
+    long long cap = 0;
+    const uint8_t* pool = nullptr;
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+      if (w == k) { cap = cv.capacity[k]; pool = cv.pool[k]; }
+    const long long tb = tile_bytes_of_expert(w);
+    const long long s = slot < 0 ? 0 : (slot < cap ? slot : cap - 1);          // never leave the pool
+    const uint8_t* tile = pool + ((((static_cast<long long>(ks.layer) * dm.batch + ks.b) * dm.n_kv_heads + ks.h) * cap + s) * ks.tpc + j) * tb;
+    if (w == 0) { if (is_v) dequant_values<2>(tile, dst, sub, lane); else dequant_keys<2>(tile, dst, sub, lane); }
+    else if (w == 1) { if (is_v) dequant_values<4>(tile, dst, sub, lane); else dequant_keys<4>(tile, dst, sub, lane); }
+    else if (w == 2) { if (is_v) dequant_values<8>(tile, dst, sub, lane); else dequant_keys<8>(tile, dst, sub, lane); }
+    else if (is_v) copy_rows<BF16, true, true>(tile + 8192, dst, sub, 32, lane);
+    else copy_rows<BF16, true, false>(tile, dst, sub, 32, lane);
+  } else {
+    const int ti0 = pos0 - ks.chunk_tokens;
+    const int n_valid = max(0, min(32, ks.tail_len - ti0));
+    const uint8_t* src = reinterpret_cast<const uint8_t*>(is_v ? cv.tail_v : cv.tail_k) + (ks.tail_base + ti0) * 256;
+    if (is_v) copy_rows<BF16, false, true>(src, dst, sub, n_valid, lane);
+    else copy_rows<BF16, false, false>(src, dst, sub, n_valid, lane);
+  }
+}
+
+template <bool BF16>
+__global__ void __launch_bounds__(kP2Threads, 1)
 prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T, int layer, float scale_log2,
                     float* __restrict__ out) {
   extern __shared__ __align__(128) uint8_t smem[];
-  uint8_t* sQ = smem;
-  uint8_t* sK = smem + kOperandBytes;
-  uint8_t* sV = smem + 2 * kOperandBytes;
-  uint8_t* sP = smem + 3 * kOperandBytes;
-  uint64_t* bar_mem = reinterpret_cast<uint64_t*>(smem + 4 * kOperandBytes);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_mem + 1);
-  const uint32_t bar = smem_addr(bar_mem);
+  uint8_t* sQ = smem;                               // two query tiles
+  uint8_t* sK = smem + 2 * kOperandBytes;
+  uint8_t* sV = smem + 3 * kOperandBytes;
+  uint8_t* sP = smem + 4 * kOperandBytes;           // two probability tiles
+  uint64_t* bar_mem = reinterpret_cast<uint64_t*>(smem + 6 * kOperandBytes);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_mem + BAR_COUNT);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  const uint32_t bar0 = smem_addr(bar_mem);
+  auto bar = [&](int i) { return bar0 + 8u * i; };
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int qt = blockIdx.x, hq = blockIdx.y, b = blockIdx.z;
+  const int pair = blockIdx.x, hq = blockIdx.y, b = blockIdx.z;
   const int H = dm.n_kv_heads, Hq = dm.n_q_heads;
   const int h = hq / (Hq / H);
-  const int q0 = qt * kQTile;
+  const int n_blocks = min(2 * pair + 2, (T + kKvBlock - 1) / kKvBlock);
 
-  if (warp == 0) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_addr(tmem_slot)), "r"(kTmemCols) : "memory");
+  if (warp == kSoftmaxWarps + kDequantWarps) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_addr(tmem_slot)), "r"(kTmemCols2) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
   }
   if (tid == 0) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;\n" ::"r"(bar) : "memory");
+    for (int i = 0; i < BAR_COUNT; ++i) {
+      const int count = (i == BAR_KFULL || i == BAR_VFULL) ? kDequantWarps : (i == BAR_PFULL0 || i == BAR_PFULL1) ? 4 : 1;
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar(i)), "r"(count) : "memory");
+    }
+    *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
   }
-  // the CTA's 128 query rows as the A operand (rows past the prompt are zero)
-  for (int i = tid; i < kQTile * 16; i += kPThreads) {
-    const int row = i >> 4, U = i & 15;
+  // the CTA's 2 x 128 query rows as A operands (rows past the prompt are zero)
+  for (int i = tid; i < 2 * kQTile * 16; i += kP2Threads) {
+    const int row = i >> 4, U = i & 15;             // row 0..255
+    const int pos = 2 * pair * kQTile + row;
     uint4 v = make_uint4(0u, 0u, 0u, 0u);
-    if (q0 + row < T)
-      v = to_fp16x8<BF16>(__ldg(reinterpret_cast<const uint4*>(Q + ((static_cast<long long>(b) * T + q0 + row) * Hq + hq) * kHeadDim + 8 * U)));
-    *reinterpret_cast<uint4*>(sQ + kmajor_unit_offset(row, U)) = v;
+    if (pos < T)
+      v = to_fp16x8<BF16>(__ldg(reinterpret_cast<const uint4*>(Q + ((static_cast<long long>(b) * T + pos) * Hq + hq) * kHeadDim + 8 * U)));
+    *reinterpret_cast<uint4*>(sQ + (row >> 7) * kOperandBytes + kmajor_unit_offset(row & 127, U)) = v;
   }
+  fence_async_proxy();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
 
-  // where the cache of this (layer, sequence, kv head) lives
-  const int group = layer / dm.rs_group;
-  const long long tbl = (static_cast<long long>(group) * dm.batch + b) * dm.max_chunks;
-  const int32_t* cnt = cv.count + (static_cast<long long>(group) * dm.batch + b) * 4;
-  const int n_chunks = min(cnt[0] + cnt[1] + cnt[2] + cnt[3], dm.max_chunks);
-  const int chunk_tokens = n_chunks * dm.chunk;
-  const int tail_len = min(cv.tail_len[layer * dm.batch + b], dm.tail_capacity);
-  const int tpc = dm.chunk / kTileTokens;
-  const long long tail_base = ((static_cast<long long>(layer) * dm.batch + b) * H + h) * dm.tail_capacity;   // rows
-
-  const uint32_t aQ = smem_addr(sQ), aK = smem_addr(sK), aV = smem_addr(sV), aP = smem_addr(sP);
-  const int row = tid & 127;                                  // query row of a softmax thread (warps 0..3)
-  const int qpos = q0 + row;
-  const uint32_t lane_addr = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
-  float o[kHeadDim];
-#pragma unroll
-  for (int c = 0; c < kHeadDim; ++c) o[c] = 0.0f;
-  float m = -INFINITY, l = 0.0f, corr = 1.0f;
-  uint32_t phase = 0;
-  bool ok = true;
-
-  for (int kb = 0; kb <= qt; ++kb) {
-    // ---- dequantise: warp w takes storage tile (w & 3) of the block, keys (w < 4) or values
-    {
-      const int sub = warp & 3;
-      const bool is_v = warp >= 4;
-      const int pos0 = kb * kKvBlock + sub * kTileTokens;
-      if (pos0 < chunk_tokens) {
-        const int c = pos0 / dm.chunk, j = (pos0 % dm.chunk) / kTileTokens;
-        const int w = cv.map[tbl + c] & 3;
-        const long long slot = cv.slot[tbl + c];
-        long long cap = 0;
-        const uint8_t* pool = nullptr;
-#pragma unroll
-        for (int k = 0; k < 4; ++k)
-          if (w == k) { cap = cv.capacity[k]; pool = cv.pool[k]; }
-        const long long tb = tile_bytes_of_expert(w);
-        const uint8_t* tile = pool + ((((static_cast<long long>(layer) * dm.batch + b) * H + h) * cap + min(slot, cap - 1)) * tpc + j) * tb;
-        if (w == 0) { if (is_v) dequant_values<2>(tile, sV, sub, lane); else dequant_keys<2>(tile, sK, sub, lane); }
-        else if (w == 1) { if (is_v) dequant_values<4>(tile, sV, sub, lane); else dequant_keys<4>(tile, sK, sub, lane); }
-        else if (w == 2) { if (is_v) dequant_values<8>(tile, sV, sub, lane); else dequant_keys<8>(tile, sK, sub, lane); }
-        else if (is_v) copy_rows<BF16, true, true>(tile + 8192, sV, sub, 32, lane);
-        else copy_rows<BF16, true, false>(tile, sK, sub, 32, lane);
-      } else {
-        const int ti0 = pos0 - chunk_tokens;
-        const int n_valid = max(0, min(32, tail_len - ti0));
-        const uint8_t* src = reinterpret_cast<const uint8_t*>(is_v ? cv.tail_v : cv.tail_k) + (tail_base + ti0) * 256;
-        if (is_v) copy_rows<BF16, false, true>(src, sV, sub, n_valid, lane);
-        else copy_rows<BF16, false, false>(src, sK, sub, n_valid, lane);
-      }
+  // bounded wait that also gives up when another role has given up
+  auto wait = [&](int which, int completion) -> bool {
+    const uint32_t a = bar(which), parity = static_cast<uint32_t>(completion) & 1u;
+    for (long long it = 0; it < kWaitLimitP; ++it) {
+      if (mbar_try_wait_p(a, parity)) return true;
+      if ((it & 1023) == 1023 && *abort_flag) return false;
     }
-    fence_async_proxy();                   // generic-proxy writes of the operand tiles -> visible to the MMA
-    tc_fence_before();
-    __syncthreads();
-    // ---- S = Q K^T
-    if (tid == 0) {
-      tc_fence_after();
-#pragma unroll
-      for (int ks = 0; ks < 8; ++ks)
-        umma_f16(tmem, make_desc(aQ + ks * 4096, 2048, 128), make_desc(aK + ks * 4096, 2048, 128), kIdescKK, ks > 0);
-      umma_commit(bar);
-    }
-    // ---- softmax of the block, one query row per thread
-    if (warp < 4) {
-      if (ok && !mbar_wait_bounded_p(bar, phase)) ok = false;
-      phase ^= 1u;
+    *abort_flag = 1;
+    return false;
+  };
+
+  if (warp < kSoftmaxWarps) {
+    // ================= softmax: one query row per thread =================
+    const int i = warp >> 2;                        // query tile of this warp
+    const int row = tid & 127;
+    const int qpos = (2 * pair + i) * kQTile + row;
+    const uint32_t lane_addr = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+    const uint32_t s_addr = lane_addr + 128 * i, o_addr = lane_addr + 256 + 128 * i;
+    uint8_t* sPi = sP + i * kOperandBytes;
+    float m_ref = -INFINITY, l = 0.0f;
+    bool ok = true;
+    for (int kb = 0; kb < n_blocks && ok; ++kb) {
+      ok = __all_sync(0xffffffffu, wait(BAR_SFULL0 + i, kb));
+      if (!ok) break;
       tc_fence_after();
       float mx = -INFINITY;
-      if (ok) {
-#pragma unroll 1
-        for (int c4 = 0; c4 < 4; ++c4) {
-          float v[32];
-          tmem_ld32(v, lane_addr + 32 * c4);
-#pragma unroll
-          for (int i = 0; i < 32; ++i)
-            if (kb * kKvBlock + 32 * c4 + i <= qpos) mx = fmaxf(mx, v[i] * scale_log2);
-        }
-      }
-      const float m_new = fmaxf(m, mx);
-      corr = (m == -INFINITY) ? 0.0f : exp2f(m - m_new);
-      l *= corr;
 #pragma unroll 1
       for (int c4 = 0; c4 < 4; ++c4) {
         float v[32];
-        if (ok) tmem_ld32(v, lane_addr + 32 * c4);
+        tmem_ld32(v, s_addr + 32 * c4);
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          uint32_t pk[4];
+        for (int e = 0; e < 32; ++e)
+          if (kb * kKvBlock + 32 * c4 + e <= qpos) mx = fmaxf(mx, v[e] * scale_log2);
+      }
+      // the reference maximum moves lazily: only when some row of the warp exceeds it by kRescaleSlack
+      const bool move = __any_sync(0xffffffffu, mx > m_ref + kRescaleSlack);
+      const float m_new = move ? fmaxf(m_ref, mx) : m_ref;
+      uint32_t pk[64];
+      float l_blk = 0.0f;
 #pragma unroll
-          for (int e2 = 0; e2 < 4; ++e2) {
-            float p2[2];
+      for (int c4 = 0; c4 < 4; ++c4) {
+        float v[32];
+        tmem_ld32(v, s_addr + 32 * c4);
 #pragma unroll
-            for (int e = 0; e < 2; ++e) {
-              const int i = 8 * u + 2 * e2 + e;
-              const bool seen = ok && (kb * kKvBlock + 32 * c4 + i <= qpos) && m_new > -INFINITY;
-              p2[e] = seen ? exp2f(v[i] * scale_log2 - m_new) : 0.0f;
-            }
-            pk[e2] = pack_h2(p2[0], p2[1]);
-            l += h_lo(pk[e2]) + h_hi(pk[e2]);             // the sum uses the weights the MMA will see
+        for (int e2 = 0; e2 < 16; ++e2) {
+          float p2[2];
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            const int col = 32 * c4 + 2 * e2 + e;
+            const bool seen = (kb * kKvBlock + col <= qpos) && m_new > -INFINITY;
+            p2[e] = seen ? exp2f(v[2 * e2 + e] * scale_log2 - m_new) : 0.0f;
           }
-          *reinterpret_cast<uint4*>(sP + kmajor_unit_offset(row, 4 * c4 + u)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+          pk[16 * c4 + e2] = pack_h2(p2[0], p2[1]);
+          l_blk += h_lo(pk[16 * c4 + e2]) + h_hi(pk[16 * c4 + e2]);    // the sum uses the weights the MMA will see
         }
       }
-      m = m_new;
+      if (kb > 0) {                                  // P_i and O_i are busy until the previous block's PV is done
+        ok = __all_sync(0xffffffffu, wait(BAR_OFULL0 + i, kb - 1));
+        if (!ok) break;
+        tc_fence_after();
+        if (move) {
+          const float corr = (m_ref == -INFINITY) ? 0.0f : exp2f(m_ref - m_new);
+#pragma unroll 1
+          for (int c4 = 0; c4 < 4; ++c4) {
+            float v[32];
+            tmem_ld32(v, o_addr + 32 * c4);
+#pragma unroll
+            for (int e = 0; e < 32; ++e) v[e] *= corr;
+            tmem_st32(o_addr + 32 * c4, v);
+          }
+          l *= corr;
+        }
+      }
+      m_ref = m_new;
+      l += l_blk;
+#pragma unroll
+      for (int u = 0; u < 16; ++u)
+        *reinterpret_cast<uint4*>(sPi + kmajor_unit_offset(row, u)) = make_uint4(pk[4 * u], pk[4 * u + 1], pk[4 * u + 2], pk[4 * u + 3]);
       fence_async_proxy();
       tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(BAR_PFULL0 + i));
     }
-    __syncthreads();
-    // ---- O_blk = P V^ (fresh accumulator), folded into the threads' fp32 rows
-    if (tid == 0) {
+    if (ok && n_blocks > 0) ok = __all_sync(0xffffffffu, wait(BAR_OFULL0 + i, n_blocks - 1));
+    if (ok) {
       tc_fence_after();
+      const float inv = l > 0.0f ? 1.0f / l : 0.0f;
+#pragma unroll 1
+      for (int c4 = 0; c4 < 4; ++c4) {
+        float v[32];
+        tmem_ld32(v, o_addr + 32 * c4);
+        if (qpos < T) {
+          float4* dst = reinterpret_cast<float4*>(out + ((static_cast<long long>(b) * T + qpos) * Hq + hq) * kHeadDim + 32 * c4);
 #pragma unroll
-      for (int ks = 0; ks < 8; ++ks)
-        umma_f16(tmem + 128, make_desc(aP + ks * 4096, 2048, 128), make_desc(aV + ks * 4096, 2048, 128), kIdescKMN, ks > 0);
-      umma_commit(bar);
-    }
-    if (warp < 4) {
-      if (ok && !mbar_wait_bounded_p(bar, phase)) ok = false;
-      phase ^= 1u;
-      tc_fence_after();
-      if (ok) {
-#pragma unroll
-        for (int c4 = 0; c4 < 4; ++c4) {
-          float v[32];
-          tmem_ld32(v, lane_addr + 128 + 32 * c4);
-#pragma unroll
-          for (int i = 0; i < 32; ++i) o[32 * c4 + i] = fmaf(o[32 * c4 + i], corr, v[i]);
+          for (int e = 0; e < 32; e += 4) dst[e >> 2] = make_float4(v[e] * inv, v[e + 1] * inv, v[e + 2] * inv, v[e + 3] * inv);
         }
       }
-      tc_fence_before();
+    } else if (lane == 0) {
+      set_status(cv.status, MOQAE_ERR_TIMEOUT, blockIdx.x, warp);
     }
-    __syncthreads();
-  }
-
-  if (warp < 4) {
-    if (!ok && lane == 0) set_status(cv.status, MOQAE_ERR_TIMEOUT, blockIdx.x, warp);
-    if (qpos < T) {
-      const float inv = l > 0.0f ? 1.0f / l : 0.0f;
-      float4* dst = reinterpret_cast<float4*>(out + ((static_cast<long long>(b) * T + qpos) * Hq + hq) * kHeadDim);
+  } else if (warp < kSoftmaxWarps + kDequantWarps) {
+    // ================= dequantise: storage tile `sub` of every block, keys then values =================
+    const int sub = warp - kSoftmaxWarps;
+    KvSource ks;
+    ks.cv = &cv; ks.dm = &dm; ks.layer = layer; ks.b = b; ks.h = h;
+    const int group = layer / dm.rs_group;
+    ks.tbl = (static_cast<long long>(group) * dm.batch + b) * dm.max_chunks;
+    const int32_t* cnt = cv.count + (static_cast<long long>(group) * dm.batch + b) * 4;
+    ks.chunk_tokens = min(cnt[0] + cnt[1] + cnt[2] + cnt[3], dm.max_chunks) * dm.chunk;
+    ks.tail_len = min(cv.tail_len[layer * dm.batch + b], dm.tail_capacity);
+    ks.tpc = dm.chunk / kTileTokens;
+    ks.tail_base = ((static_cast<long long>(layer) * dm.batch + b) * H + h) * dm.tail_capacity;
+    for (int kb = 0; kb < n_blocks; ++kb) {
+      const int pos0 = kb * kKvBlock + sub * kTileTokens;
+      if (kb > 0 && !wait(BAR_SFULL1, kb - 1)) break;          // K^ is free once both S products of the last block are done
+      dequant_subtile<BF16>(ks, pos0, sub, false, sK, lane);
+      fence_async_proxy();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(BAR_KFULL));
+      if (kb > 0 && !wait(BAR_OFULL1, kb - 1)) break;          // V^ is free once both PV products are done
+      dequant_subtile<BF16>(ks, pos0, sub, true, sV, lane);
+      fence_async_proxy();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(BAR_VFULL));
+    }
+  } else {
+    // ================= MMA issue (one thread) =================
+    const uint32_t aQ = smem_addr(sQ), aK = smem_addr(sK), aV = smem_addr(sV), aP = smem_addr(sP);
+    bool ok = true;
+    for (int kb = 0; kb < n_blocks && ok; ++kb) {
+      ok = wait(BAR_KFULL, kb);
+      for (int i = 0; i < 2 && ok; ++i) {
+        if (kb > 0) ok = wait(BAR_PFULL0 + i, kb - 1);         // S_i of the last block has been read
+        if (!ok) break;
+        tc_fence_after();
+        if (lane == 0) {
 #pragma unroll
-      for (int c = 0; c < kHeadDim; c += 4) dst[c >> 2] = make_float4(o[c] * inv, o[c + 1] * inv, o[c + 2] * inv, o[c + 3] * inv);
+          for (int k = 0; k < 8; ++k)
+            umma_f16(tmem + 128 * i, make_desc(aQ + i * kOperandBytes + k * 4096, 2048, 128), make_desc(aK + k * 4096, 2048, 128),
+                     kIdescKK, k > 0);
+          umma_commit(bar(BAR_SFULL0 + i));
+        }
+        __syncwarp();
+      }
+      if (ok) ok = wait(BAR_VFULL, kb);
+      for (int i = 0; i < 2 && ok; ++i) {
+        ok = wait(BAR_PFULL0 + i, kb);
+        if (!ok) break;
+        tc_fence_after();
+        if (lane == 0) {
+#pragma unroll
+          for (int k = 0; k < 8; ++k)
+            umma_f16(tmem + 256 + 128 * i, make_desc(aP + i * kOperandBytes + k * 4096, 2048, 128), make_desc(aV + k * 4096, 2048, 128),
+                     kIdescKMN, (kb > 0 || k > 0) ? 1u : 0u);
+          umma_commit(bar(BAR_OFULL0 + i));
+        }
+        __syncwarp();
+      }
     }
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(kTmemCols) : "memory");
+  if (warp == kSoftmaxWarps + kDequantWarps)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(kTmemCols2) : "memory");
 }
 
 }  // namespace
@@ -440,18 +537,18 @@ prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T
 cudaError_t launch_prefill_attn(const Dims& dm, const CacheView& cv, const void* q, int T, int layer, float scale,
                                 float* out, cudaStream_t st) {
   if (T <= 0) return cudaSuccess;
-  const size_t smem = 4 * kOperandBytes + 16;
-  dim3 grid((T + kQTile - 1) / kQTile, dm.n_q_heads, dm.batch);
+  const size_t smem = 6 * kOperandBytes + BAR_COUNT * 8 + 16;
+  dim3 grid((T + 2 * kQTile - 1) / (2 * kQTile), dm.n_q_heads, dm.batch);
   const float scale_log2 = scale * 1.4426950408889634f;
   cudaError_t e;
   if (dm.dtype == MOQAE_DTYPE_BF16) {
     e = cudaFuncSetAttribute(prefill_attn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return e;
-    prefill_attn_kernel<true><<<grid, kPThreads, smem, st>>>(dm, cv, static_cast<const uint16_t*>(q), T, layer, scale_log2, out);
+    prefill_attn_kernel<true><<<grid, kP2Threads, smem, st>>>(dm, cv, static_cast<const uint16_t*>(q), T, layer, scale_log2, out);
   } else {
     e = cudaFuncSetAttribute(prefill_attn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return e;
-    prefill_attn_kernel<false><<<grid, kPThreads, smem, st>>>(dm, cv, static_cast<const uint16_t*>(q), T, layer, scale_log2, out);
+    prefill_attn_kernel<false><<<grid, kP2Threads, smem, st>>>(dm, cv, static_cast<const uint16_t*>(q), T, layer, scale_log2, out);
   }
   return cudaGetLastError();
 }
