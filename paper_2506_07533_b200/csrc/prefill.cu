@@ -243,17 +243,17 @@ __device__ __forceinline__ void copy_rows(const uint8_t* __restrict__ src, uint8
 }
 
 // ---- the kernel ----------------------------------------------------------------------------
-// Roles (13 warps): warps 0..3 and 4..7 are the softmax threads of the CTA's two query tiles
-// (one row each, tensor-memory lane = tid % 128); warps 8..11 dequantise (one storage tile
-// each: keys of block kb, then values of block kb); warp 12 issues the MMAs.  They meet
+// Roles (17 warps): warps 0..3 and 4..7 are the softmax threads of the CTA's two query tiles
+// (one row each, tensor-memory lane = tid % 128); warps 8..11 dequantise the keys and warps
+// 12..15 the values of every block (one storage tile each); warp 16 issues the MMAs.  They meet
 // only on mbarriers:
-//   kfull / vfull     K^ / V^ of a block are in shared memory            (4 dequant warps)
+//   kfull / vfull     K^ / V^ of a block are in shared memory            (4 of the dequant warps)
 //   sfull[i]          S_i = Q_i K^T is in tensor memory                  (tcgen05.commit)
 //   pfull[i]          P_i is in shared memory and S_i has been read      (4 softmax warps)
 //   ofull[i]          O_i += P_i V^ is done                              (tcgen05.commit)
 // K^ is free again when sfull[1] completes, V^ when ofull[1] completes.  Every barrier
 // completes once per block, so completion number kb is awaited with parity kb & 1.
-constexpr int kSoftmaxWarps = 8, kDequantWarps = 4;
+constexpr int kSoftmaxWarps = 8, kDequantWarps = 8;   // dequant: 4 warps for keys, 4 for values
 constexpr int kP2Threads = (kSoftmaxWarps + kDequantWarps + 1) * 32;
 constexpr int kTmemCols2 = 512;                // S_0, S_1, O_0, O_1: 128 columns each
 constexpr float kRescaleSlack = 8.0f;          // base-2 units: weights stay below 2^8
@@ -345,7 +345,7 @@ prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T
   }
   if (tid == 0) {
     for (int i = 0; i < BAR_COUNT; ++i) {
-      const int count = (i == BAR_KFULL || i == BAR_VFULL) ? kDequantWarps : (i == BAR_PFULL0 || i == BAR_PFULL1) ? 4 : 1;
+      const int count = (i == BAR_KFULL || i == BAR_VFULL) ? kDequantWarps / 2 : (i == BAR_PFULL0 || i == BAR_PFULL1) ? 4 : 1;
       asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar(i)), "r"(count) : "memory");
     }
     *abort_flag = 0;
@@ -403,25 +403,6 @@ prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T
       // the reference maximum moves lazily: only when some row of the warp exceeds it by kRescaleSlack
       const bool move = __any_sync(0xffffffffu, mx > m_ref + kRescaleSlack);
       const float m_new = move ? fmaxf(m_ref, mx) : m_ref;
-      uint32_t pk[64];
-      float l_blk = 0.0f;
-#pragma unroll
-      for (int c4 = 0; c4 < 4; ++c4) {
-        float v[32];
-        tmem_ld32(v, s_addr + 32 * c4);
-#pragma unroll
-        for (int e2 = 0; e2 < 16; ++e2) {
-          float p2[2];
-#pragma unroll
-          for (int e = 0; e < 2; ++e) {
-            const int col = 32 * c4 + 2 * e2 + e;
-            const bool seen = (kb * kKvBlock + col <= qpos) && m_new > -INFINITY;
-            p2[e] = seen ? exp2f(v[2 * e2 + e] * scale_log2 - m_new) : 0.0f;
-          }
-          pk[16 * c4 + e2] = pack_h2(p2[0], p2[1]);
-          l_blk += h_lo(pk[16 * c4 + e2]) + h_hi(pk[16 * c4 + e2]);    // the sum uses the weights the MMA will see
-        }
-      }
       if (kb > 0) {                                  // P_i and O_i are busy until the previous block's PV is done
         ok = __all_sync(0xffffffffu, wait(BAR_OFULL0 + i, kb - 1));
         if (!ok) break;
@@ -440,10 +421,27 @@ prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T
         }
       }
       m_ref = m_new;
-      l += l_blk;
+#pragma unroll 1
+      for (int c4 = 0; c4 < 4; ++c4) {
+        float v[32];
+        tmem_ld32(v, s_addr + 32 * c4);
+        uint32_t pk[16];
 #pragma unroll
-      for (int u = 0; u < 16; ++u)
-        *reinterpret_cast<uint4*>(sPi + kmajor_unit_offset(row, u)) = make_uint4(pk[4 * u], pk[4 * u + 1], pk[4 * u + 2], pk[4 * u + 3]);
+        for (int e2 = 0; e2 < 16; ++e2) {
+          float p2[2];
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            const int col = 32 * c4 + 2 * e2 + e;
+            const bool seen = (kb * kKvBlock + col <= qpos) && m_new > -INFINITY;
+            p2[e] = seen ? exp2f(v[2 * e2 + e] * scale_log2 - m_new) : 0.0f;
+          }
+          pk[e2] = pack_h2(p2[0], p2[1]);
+          l += h_lo(pk[e2]) + h_hi(pk[e2]);            // the sum uses the weights the MMA will see
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+          *reinterpret_cast<uint4*>(sPi + kmajor_unit_offset(row, 4 * c4 + u)) = make_uint4(pk[4 * u], pk[4 * u + 1], pk[4 * u + 2], pk[4 * u + 3]);
+      }
       fence_async_proxy();
       tc_fence_before();
       __syncwarp();
@@ -468,7 +466,8 @@ prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T
     }
   } else if (warp < kSoftmaxWarps + kDequantWarps) {
     // ================= dequantise: storage tile `sub` of every block, keys then values =================
-    const int sub = warp - kSoftmaxWarps;
+    const int sub = (warp - kSoftmaxWarps) & 3;
+    const bool is_v = (warp - kSoftmaxWarps) >= 4;
     KvSource ks;
     ks.cv = &cv; ks.dm = &dm; ks.layer = layer; ks.b = b; ks.h = h;
     const int group = layer / dm.rs_group;
@@ -480,16 +479,12 @@ prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T
     ks.tail_base = ((static_cast<long long>(layer) * dm.batch + b) * H + h) * dm.tail_capacity;
     for (int kb = 0; kb < n_blocks; ++kb) {
       const int pos0 = kb * kKvBlock + sub * kTileTokens;
-      if (kb > 0 && !wait(BAR_SFULL1, kb - 1)) break;          // K^ is free once both S products of the last block are done
-      dequant_subtile<BF16>(ks, pos0, sub, false, sK, lane);
+      // K^ is free once both S products of the last block are done, V^ once both PV products are
+      if (kb > 0 && !wait(is_v ? BAR_OFULL1 : BAR_SFULL1, kb - 1)) break;
+      dequant_subtile<BF16>(ks, pos0, sub, is_v, is_v ? sV : sK, lane);
       fence_async_proxy();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar(BAR_KFULL));
-      if (kb > 0 && !wait(BAR_OFULL1, kb - 1)) break;          // V^ is free once both PV products are done
-      dequant_subtile<BF16>(ks, pos0, sub, true, sV, lane);
-      fence_async_proxy();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(BAR_VFULL));
+      if (lane == 0) mbar_arrive(bar(is_v ? BAR_VFULL : BAR_KFULL));
     }
   } else {
     // ================= MMA issue (one thread) =================
