@@ -109,6 +109,11 @@ template <bool BF16> __device__ __forceinline__ uint4 to_fp16x8(uint4 v) {
   o.w = pack_h2(__uint_as_float(v.w << 16), __uint_as_float(v.w & 0xffff0000u));
   return o;
 }
+__device__ __forceinline__ float ex2_approx(float x) {
+  float r;
+  asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(r) : "f"(x));
+  return r;
+}
 __device__ __forceinline__ float h_lo(uint32_t w) { return __low2float(*reinterpret_cast<const __half2*>(&w)); }
 __device__ __forceinline__ float h_hi(uint32_t w) { return __high2float(*reinterpret_cast<const __half2*>(&w)); }
 
@@ -391,24 +396,63 @@ prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T
       ok = __all_sync(0xffffffffu, wait(BAR_SFULL0 + i, kb));
       if (!ok) break;
       tc_fence_after();
-      float mx = -INFINITY;
-#pragma unroll 1
-      for (int c4 = 0; c4 < 4; ++c4) {
-        float v[32];
-        tmem_ld32(v, s_addr + 32 * c4);
-#pragma unroll
-        for (int e = 0; e < 32; ++e)
-          if (kb * kKvBlock + 32 * c4 + e <= qpos) mx = fmaxf(mx, v[e] * scale_log2);
-      }
-      // the reference maximum moves lazily: only when some row of the warp exceeds it by kRescaleSlack
-      const bool move = __any_sync(0xffffffffu, mx > m_ref + kRescaleSlack);
-      const float m_new = move ? fmaxf(m_ref, mx) : m_ref;
       if (kb > 0) {                                  // P_i and O_i are busy until the previous block's PV is done
         ok = __all_sync(0xffffffffu, wait(BAR_OFULL0 + i, kb - 1));
         if (!ok) break;
         tc_fence_after();
-        if (move) {
-          const float corr = (m_ref == -INFINITY) ? 0.0f : exp2f(m_ref - m_new);
+      }
+      // Blocks left of the diagonal are fully visible; only the last one or two need the mask.
+      const bool diag = kb >= 2 * pair + i;
+      const int rel = qpos - kb * kKvBlock;          // columns 0..rel of this block are visible
+      // One pass over S_i: weights against the reference maximum `mref` into P_i, their sum, and
+      // the largest score seen.
+      auto emit = [&](float mref, float& sum, float& mx) {
+        sum = 0.0f;
+        mx = -INFINITY;
+#pragma unroll 1
+        for (int c4 = 0; c4 < 4; ++c4) {
+          float v[32];
+          tmem_ld32(v, s_addr + 32 * c4);
+          uint32_t pk[16];
+#pragma unroll
+          for (int e2 = 0; e2 < 16; ++e2) {
+            float x0 = v[2 * e2] * scale_log2, x1 = v[2 * e2 + 1] * scale_log2;
+            if (diag) {
+              if (32 * c4 + 2 * e2 > rel) x0 = -INFINITY;
+              if (32 * c4 + 2 * e2 + 1 > rel) x1 = -INFINITY;
+            }
+            mx = fmaxf(mx, fmaxf(x0, x1));
+            const float p0 = ex2_approx(x0 - mref), p1 = ex2_approx(x1 - mref);
+            sum += p0 + p1;
+            pk[e2] = pack_h2(p0, p1);
+          }
+#pragma unroll
+          for (int u = 0; u < 4; ++u)
+            *reinterpret_cast<uint4*>(sPi + kmajor_unit_offset(row, 4 * c4 + u)) = make_uint4(pk[4 * u], pk[4 * u + 1], pk[4 * u + 2], pk[4 * u + 3]);
+        }
+      };
+      float sum, mx;
+      bool move = (kb == 0);                         // the first block has no reference yet
+      if (!move) {
+        // optimistic single pass against the current reference; it stands unless some row of the
+        // warp found a score more than kRescaleSlack above its reference
+        emit(m_ref, sum, mx);
+        move = __any_sync(0xffffffffu, mx > m_ref + kRescaleSlack);
+      } else {
+        mx = -INFINITY;
+#pragma unroll 1
+        for (int c4 = 0; c4 < 4; ++c4) {
+          float v[32];
+          tmem_ld32(v, s_addr + 32 * c4);
+#pragma unroll
+          for (int e = 0; e < 32; ++e)
+            if (!diag || 32 * c4 + e <= rel) mx = fmaxf(mx, v[e] * scale_log2);
+        }
+      }
+      if (move) {
+        const float m_new = fmaxf(m_ref, mx);
+        if (kb > 0) {
+          const float corr = (m_ref == -INFINITY) ? 0.0f : ex2_approx(m_ref - m_new);
 #pragma unroll 1
           for (int c4 = 0; c4 < 4; ++c4) {
             float v[32];
@@ -419,29 +463,11 @@ prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T
           }
           l *= corr;
         }
+        m_ref = m_new;
+        float mx2;
+        emit(m_ref, sum, mx2);
       }
-      m_ref = m_new;
-#pragma unroll 1
-      for (int c4 = 0; c4 < 4; ++c4) {
-        float v[32];
-        tmem_ld32(v, s_addr + 32 * c4);
-        uint32_t pk[16];
-#pragma unroll
-        for (int e2 = 0; e2 < 16; ++e2) {
-          float p2[2];
-#pragma unroll
-          for (int e = 0; e < 2; ++e) {
-            const int col = 32 * c4 + 2 * e2 + e;
-            const bool seen = (kb * kKvBlock + col <= qpos) && m_new > -INFINITY;
-            p2[e] = seen ? exp2f(v[2 * e2 + e] * scale_log2 - m_new) : 0.0f;
-          }
-          pk[e2] = pack_h2(p2[0], p2[1]);
-          l += h_lo(pk[e2]) + h_hi(pk[e2]);            // the sum uses the weights the MMA will see
-        }
-#pragma unroll
-        for (int u = 0; u < 4; ++u)
-          *reinterpret_cast<uint4*>(sPi + kmajor_unit_offset(row, 4 * c4 + u)) = make_uint4(pk[4 * u], pk[4 * u + 1], pk[4 * u + 2], pk[4 * u + 3]);
-      }
+      l += sum;
       fence_async_proxy();
       tc_fence_before();
       __syncwarp();
