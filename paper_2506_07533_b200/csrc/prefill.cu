@@ -114,8 +114,6 @@ __device__ __forceinline__ float ex2_approx(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(r) : "f"(x));
   return r;
 }
-__device__ __forceinline__ float h_lo(uint32_t w) { return __low2float(*reinterpret_cast<const __half2*>(&w)); }
-__device__ __forceinline__ float h_hi(uint32_t w) { return __high2float(*reinterpret_cast<const __half2*>(&w)); }
 
 // ---- dequantisation of one 32-token storage tile into the operand tiles --------------------
 // The packed layout is the one the decode kernel's lanes consume (lane = 4g + t4); the same
@@ -125,26 +123,36 @@ template <int BITS> __host__ __device__ constexpr int key_reg_channel_lo(int r) 
   return (r / (n / 2)) * n + ((r % (n / 2)) / (n / 4)) * (n / 4) + r % (n / 4);
 }
 
+// Two codes that sit at the same bit position `pos` of the two half-words of `w` -> (code_lo,
+// code_hi) as fp16: shifting them to bit 0 and OR-ing 0x6400 gives 1024 + code exactly.
+template <int BITS> __device__ __forceinline__ uint32_t codes_to_half2(uint32_t w, int pos) {
+  constexpr uint32_t mask = ((1u << BITS) - 1u) * 0x00010001u;
+  uint32_t x = ((w >> pos) & mask) | 0x64006400u, r;
+  asm("sub.rn.f16x2 %0, %1, %2;\n" : "=r"(r) : "r"(x), "r"(0x64006400u));
+  return r;
+}
+__device__ __forceinline__ uint32_t hfma2_u32(uint32_t a, uint32_t b, uint32_t c) {
+  uint32_t r;
+  asm("fma.rn.f16x2 %0, %1, %2, %3;\n" : "=r"(r) : "r"(a), "r"(b), "r"(c));
+  return r;
+}
+
+// Keys.  A payload word masked at one code position carries the codes of channels c and
+// c + n/2 (n = codes per word); the scale and zero arrays hold exactly those pairs, so one
+// packed FMA dequantises two channels: K^ = RN(code * scale + zero) in fp16.
 template <int BITS>
 __device__ __forceinline__ void dequant_keys(const uint8_t* __restrict__ tile, uint8_t* sK, int sub, int lane) {
-  constexpr int n = 32 / BITS;
-  constexpr uint32_t mask = (1u << BITS) - 1u;
+  constexpr int n = 32 / BITS, regs = n / 2, direct = n / 4;
   const int g = lane >> 2, t4 = lane & 3;
-  float sc[32], zr[32];                    // scale and zero of channels 32*t4 .. +31
+  uint32_t sc[16], zr[16];                 // register r: (lo, hi) = channels cl(r), cl(r) + n/2 of quarter t4
   {
     const uint4* sp = reinterpret_cast<const uint4*>(tile) + t4;
     const uint4* zp = reinterpret_cast<const uint4*>(tile + 256) + t4;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const uint4 s4 = __ldg(sp + 4 * i), z4 = __ldg(zp + 4 * i);
-      const uint32_t sw[4] = {s4.x, s4.y, s4.z, s4.w};
-      const uint32_t zw[4] = {z4.x, z4.z, z4.y, z4.w};     // zeros are stored in register order 0, 2, 1, 3
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const int cl = key_reg_channel_lo<BITS>(4 * i + j);
-        sc[cl] = h_lo(sw[j]); sc[cl + n / 2] = h_hi(sw[j]);
-        zr[cl] = h_lo(zw[j]); zr[cl + n / 2] = h_hi(zw[j]);
-      }
+      sc[4 * i] = s4.x; sc[4 * i + 1] = s4.y; sc[4 * i + 2] = s4.z; sc[4 * i + 3] = s4.w;
+      zr[4 * i] = z4.x; zr[4 * i + 1] = z4.z; zr[4 * i + 2] = z4.y; zr[4 * i + 3] = z4.w;   // stored in order 0, 2, 1, 3
     }
   }
   const uint8_t* kpay = tile + kMetaBytes;
@@ -166,25 +174,38 @@ __device__ __forceinline__ void dequant_keys(const uint8_t* __restrict__ tile, u
           w[(4 * j2) % BITS] = v.x; w[(4 * j2 + 1) % BITS] = v.y; w[(4 * j2 + 2) % BITS] = v.z; w[(4 * j2 + 3) % BITS] = v.w;
         }
       }
+      // value pair of register r: channels (cl, cl + n/2); val[c] collects them by channel pair
+      uint32_t byreg[16];
+#pragma unroll
+      for (int r = 0; r < 16; ++r) {
+        const int j = r / regs, s = (r % regs) / direct, m = r % direct;
+        byreg[r] = hfma2_u32(codes_to_half2<BITS>(w[j], 8 * s + BITS * m), sc[r], zr[r]);
+      }
+      // channels cc and cc + 1 (cc even) of the piece: low or high halves of two neighbouring registers
       const int row = 32 * sub + 16 * blk + 8 * hh + g;
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
-        float v[8];
+        uint32_t o[4];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          const int cc = 8 * u + e;
-          const uint32_t code = (w[(cc * BITS) >> 5] >> ((cc * BITS) & 31)) & mask;
-          v[e] = fmaf(static_cast<float>(code), sc[cc], zr[cc]);
+        for (int e2 = 0; e2 < 4; ++e2) {
+          const int cc = 8 * u + 2 * e2;                      // even channel of the pair
+          const int j = cc / n, i = cc % n;                   // word, position inside the word
+          const bool hi = i >= n / 2;
+          const int i2 = i % (n / 2);
+          const int ra = j * regs + (i2 / direct) * direct + i2 % direct;         // register of channel cc
+          const int i3 = (i + 1) % (n / 2);
+          const int rb = j * regs + (i3 / direct) * direct + i3 % direct;         // register of channel cc + 1
+          o[e2] = __byte_perm(byreg[ra], byreg[rb], hi ? 0x7632 : 0x5410);
         }
-        *reinterpret_cast<uint4*>(sK + kmajor_unit_offset(row, 4 * t4 + u)) =
-            make_uint4(pack_h2(v[0], v[1]), pack_h2(v[2], v[3]), pack_h2(v[4], v[5]), pack_h2(v[6], v[7]));
+        *reinterpret_cast<uint4*>(sK + kmajor_unit_offset(row, 4 * t4 + u)) = make_uint4(o[0], o[1], o[2], o[3]);
       }
     }
 }
 
+// Values.  A payload word masked at one slot carries the codes of tokens e = 0, 1 of one
+// channel row; the scale and zero arrays hold those token pairs per channel group.
 template <int BITS>
 __device__ __forceinline__ void dequant_values(const uint8_t* __restrict__ tile, uint8_t* sV, int sub, int lane) {
-  constexpr uint32_t mask = (1u << BITS) - 1u;
   constexpr int per = 8 / BITS;                                   // channel rows per word
   const int g = lane >> 2, t4 = lane & 3;
   const uint8_t* vpay = tile + kMetaBytes + kTileTokens * 16 * BITS;
@@ -210,23 +231,20 @@ __device__ __forceinline__ void dequant_values(const uint8_t* __restrict__ tile,
 #pragma unroll
     for (int cg = 0; cg < 4; ++cg)
 #pragma unroll
-      for (int half = 0; half < 2; ++half)
+      for (int half = 0; half < 2; ++half) {
+        uint32_t v[4];                                             // channel rows r4 = 0..3: (token e = 0, token e = 1)
 #pragma unroll
-        for (int e = 0; e < 2; ++e) {
-          const float s = e ? h_hi(sw[cg][half]) : h_lo(sw[cg][half]);
-          const float z = e ? h_hi(zw[cg][half]) : h_lo(zw[cg][half]);
-          float v[4];
-#pragma unroll
-          for (int r4 = 0; r4 < 4; ++r4) {
-            const int R = 4 * cg + r4;
-            const uint32_t code = (wv[R / per] >> (BITS * (R % per) + 8 * half + 16 * e)) & mask;
-            v[r4] = fmaf(static_cast<float>(code), s, z);
-          }
-          const int tok = 32 * sub + 16 * blk + 8 * half + 2 * t4 + e;
-          // channels 32cg + 4g .. +3: half of the 16-byte unit c8 = 4cg + g/2
-          *reinterpret_cast<uint2*>(sV + mnmajor_unit_offset(tok, 4 * cg + (g >> 1)) + (g & 1) * 8) =
-              make_uint2(pack_h2(v[0], v[1]), pack_h2(v[2], v[3]));
+        for (int r4 = 0; r4 < 4; ++r4) {
+          const int R = 4 * cg + r4;
+          v[r4] = hfma2_u32(codes_to_half2<BITS>(wv[R / per], BITS * (R % per) + 8 * half), sw[cg][half], zw[cg][half]);
         }
+        const int tok = 32 * sub + 16 * blk + 8 * half + 2 * t4;
+        // channels 32cg + 4g .. +3: half of the 16-byte unit c8 = 4cg + g/2, one store per token
+        *reinterpret_cast<uint2*>(sV + mnmajor_unit_offset(tok, 4 * cg + (g >> 1)) + (g & 1) * 8) =
+            make_uint2(__byte_perm(v[0], v[1], 0x5410), __byte_perm(v[2], v[3], 0x5410));
+        *reinterpret_cast<uint2*>(sV + mnmajor_unit_offset(tok + 1, 4 * cg + (g >> 1)) + (g & 1) * 8) =
+            make_uint2(__byte_perm(v[0], v[1], 0x7632), __byte_perm(v[2], v[3], 0x7632));
+      }
   }
 }
 
