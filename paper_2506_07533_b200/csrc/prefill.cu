@@ -28,16 +28,18 @@ namespace {
 
 constexpr int kQTile = 128;                    // query rows per CTA
 constexpr int kKvBlock = 128;                  // tokens per block (four storage tiles)
-constexpr int kOperandBytes = 128 * 128 * 2;   // one fp16 operand tile
-constexpr long long kWaitLimitP = 1ll << 22;
+constexpr long long kWaitCycles = 1ll << 31;    // about a second: no wait of a healthy launch comes near
+constexpr uint32_t kSuspendNs = 20000;         // how long one try_wait may keep the warp parked
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
+// One try_wait with a suspend-time hint: the warp is parked by the hardware until the phase
+// completes or the hint runs out, so a waiting role issues almost nothing.
 __device__ __forceinline__ bool mbar_try_wait_p(uint32_t bar, uint32_t parity) {
   uint32_t ok;
-  asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
-               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\nselp.u32 %0, 1, 0, p;\n}\n"
+               : "=r"(ok) : "r"(bar), "r"(parity), "r"(kSuspendNs) : "memory");
   return ok != 0;
 }
 // ---- tcgen05 wrappers -------------------------------------------------------------------
@@ -51,13 +53,25 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes
 }
 // Instruction descriptor of kind::f16: fp32 accumulator, fp16 A and B, M = 128, N = 128;
 // bit 16 set = B is MN-major (its N index is the contiguous one).
-constexpr uint32_t kIdescKK = (1u << 4) | (16u << 17) | (8u << 24);
-constexpr uint32_t kIdescKMN = kIdescKK | (1u << 16);
+constexpr uint32_t kIdescS = (1u << 4) | (16u << 17) | (8u << 24);
+constexpr uint32_t kIdescPV = kIdescS | (1u << 16);
 
-__device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
-               "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
-               ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+// D (tensor memory) = / += A B with the A operand read from tensor memory: row = lane, 16-bit
+// elements packed two per 32-bit column (element 2j in the low half of column j), 8 columns per
+// K step of 16.  The B descriptor arrives as its two words so that the issuing thread only adds
+// a block offset to the low one (start address field; it never carries out of its 14 bits).
+__device__ __forceinline__ void umma_f16_ta(uint32_t tmem_d, uint32_t tmem_a, uint32_t bdesc_lo, uint32_t bdesc_hi, uint32_t idesc,
+                                            uint32_t accumulate) {
+  asm volatile("{\n.reg .pred p;\n.reg .b64 bd;\nsetp.ne.b32 p, %5, 0;\nmov.b64 bd, {%2, %3};\n"
+               "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], bd, %4, p;\n}\n"
+               ::"r"(tmem_d), "r"(tmem_a), "r"(bdesc_lo), "r"(bdesc_hi), "r"(idesc), "r"(accumulate) : "memory");
+}
+// The same with both operands in shared memory.
+__device__ __forceinline__ void umma_f16_ss(uint32_t tmem_d, uint32_t adesc_lo, uint32_t adesc_hi, uint32_t bdesc_lo, uint32_t bdesc_hi,
+                                            uint32_t idesc, uint32_t accumulate) {
+  asm volatile("{\n.reg .pred p;\n.reg .b64 ad, bd;\nsetp.ne.b32 p, %6, 0;\nmov.b64 ad, {%1, %2};\nmov.b64 bd, {%3, %4};\n"
+               "tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %5, p;\n}\n"
+               ::"r"(tmem_d), "r"(adesc_lo), "r"(adesc_hi), "r"(bdesc_lo), "r"(bdesc_hi), "r"(idesc), "r"(accumulate) : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar) : "memory");
@@ -83,11 +97,12 @@ __device__ __forceinline__ void tmem_ld32(float (&v)[32], uint32_t taddr) {
 }
 
 // ---- operand tiles in shared memory -------------------------------------------------------
-// K-major operand (Q, K^, P): element (row n, k) of a 128 x 128 fp16 tile.  Core matrix =
-// 8 rows x 8 elements (128 bytes); the 16 core matrices of one 8-element K slab are
-// contiguous (stride 128 B between row groups), K slabs follow each other (2048 B).
+// K-major operand (Q; K^ with the 128 token rows of a block): element (row n, k) of a
+// ROWS x 128 fp16 tile.  Core matrix = 8 rows x 8 elements (128 bytes); the ROWS/8 core matrices
+// of one 8-element K slab are contiguous (128 B between row groups), K slabs follow each other.
+template <int ROWS>
 __device__ __forceinline__ int kmajor_unit_offset(int n, int k8) {       // byte offset of the 16-byte unit (n, k8*8..+7)
-  return (k8 * 16 + (n >> 3)) * 128 + (n & 7) * 16;
+  return (k8 * (ROWS / 8) + (n >> 3)) * 128 + (n & 7) * 16;
 }
 // MN-major operand (V^: rows = tokens (K of the MMA), contiguous index = channels): core
 // matrix = 8 tokens x 8 channels; the 16 channel groups of one 8-token slab are contiguous.
@@ -156,7 +171,7 @@ __device__ __forceinline__ void dequant_keys(const uint8_t* __restrict__ tile, u
     }
   }
   const uint8_t* kpay = tile + kMetaBytes;
-#pragma unroll
+#pragma unroll 1
   for (int blk = 0; blk < 2; ++blk)
 #pragma unroll
     for (int hh = 0; hh < 2; ++hh) {
@@ -197,7 +212,7 @@ __device__ __forceinline__ void dequant_keys(const uint8_t* __restrict__ tile, u
           const int rb = j * regs + (i3 / direct) * direct + i3 % direct;         // register of channel cc + 1
           o[e2] = __byte_perm(byreg[ra], byreg[rb], hi ? 0x7632 : 0x5410);
         }
-        *reinterpret_cast<uint4*>(sK + kmajor_unit_offset(row, 4 * t4 + u)) = make_uint4(o[0], o[1], o[2], o[3]);
+        *reinterpret_cast<uint4*>(sK + kmajor_unit_offset<128>(row, 4 * t4 + u)) = make_uint4(o[0], o[1], o[2], o[3]);
       }
     }
 }
@@ -209,7 +224,7 @@ __device__ __forceinline__ void dequant_values(const uint8_t* __restrict__ tile,
   constexpr int per = 8 / BITS;                                   // channel rows per word
   const int g = lane >> 2, t4 = lane & 3;
   const uint8_t* vpay = tile + kMetaBytes + kTileTokens * 16 * BITS;
-#pragma unroll
+#pragma unroll 1
   for (int blk = 0; blk < 2; ++blk) {
     uint32_t sw[4][2], zw[4][2];                                  // [channel group][half]: fp16 pair (e = 0, 1)
 #pragma unroll
@@ -260,7 +275,7 @@ __device__ __forceinline__ void copy_rows(const uint8_t* __restrict__ src, uint8
     const int up = SWIZZLED ? ((U & 8) | ((U ^ row) & 7)) : U;
     uint4 v = make_uint4(0u, 0u, 0u, 0u);
     if (row < n_valid) v = to_fp16x8<BF16>(__ldg(reinterpret_cast<const uint4*>(src + row * 256 + up * 16)));
-    const int off = IS_V ? mnmajor_unit_offset(32 * sub + row, U) : kmajor_unit_offset(32 * sub + row, U);
+    const int off = IS_V ? mnmajor_unit_offset(32 * sub + row, U) : kmajor_unit_offset<128>(32 * sub + row, U);
     *reinterpret_cast<uint4*>(dst + off) = v;
   }
 }
@@ -268,39 +283,79 @@ __device__ __forceinline__ void copy_rows(const uint8_t* __restrict__ src, uint8
 // ---- the kernel ----------------------------------------------------------------------------
 // Roles (17 warps): warps 0..3 and 4..7 are the softmax threads of the CTA's two query tiles
 // (one row each, tensor-memory lane = tid % 128); warps 8..11 dequantise the keys and warps
-// 12..15 the values of every block (one storage tile each); warp 16 issues the MMAs.  They meet
-// only on mbarriers:
-//   kfull / vfull     K^ / V^ of a block are in shared memory            (4 of the dequant warps)
-//   sfull[i]          S_i = Q_i K^T is in tensor memory                  (tcgen05.commit)
-//   pfull[i]          P_i is in shared memory and S_i has been read      (4 softmax warps)
-//   ofull[i]          O_i += P_i V^ is done                              (tcgen05.commit)
-// K^ is free again when sfull[1] completes, V^ when ofull[1] completes.  Every barrier
-// completes once per block, so completion number kb is awaited with parity kb & 1.
+// 12..15 the values of every block (one storage tile each); warp 16 issues the MMAs.  Shared
+// memory holds the two query tiles and kStages blocks of K^ and of V^; the probabilities are an
+// A operand read from tensor memory.  Tensor memory (512 columns):
+//   S_i   128 columns at 128 i        scores (fp32) of the current block; P_i (packed fp16, 64
+//                                     columns) overwrites its first half chunk by chunk as the
+//                                     scores are read
+//   O_i   128 columns at 256 + 128 i
+// Every product is M 128 x N 128 x K 16, the shape at which the tensor pipe runs at its peak
+// when fed by one issuing thread.  The two tiles alternate: while the softmax threads of one
+// work on S_i, the pipe runs O += P V^ and the next S of the other.  The roles meet only on
+// mbarriers:
+//   kfull[st] / vfull[st]   K^ / V^ of a block are in stage st               (4 dequant warps)
+//   kfree[st] / vfree[st]   the products that read stage st are done         (tcgen05.commit)
+//   sfull[i]                S_i = Q_i K^T is in tensor memory                (tcgen05.commit)
+//   pfull[i]                P_i is in tensor memory                          (4 softmax warps)
+//   ofull[i]                the last O_i += P_i V^ is done                   (tcgen05.commit, once)
+// Stage barriers complete once per kStages blocks, tile barriers once per block, and every
+// waiter follows its barrier completion by completion, so waiting on the parity of the
+// completion index is exact.  The MMAs of one thread execute in issue order: S_i of block
+// kb + 1 is issued after O_i += P_i V^ of block kb, so it may overwrite P_i, and its completion
+// tells the softmax threads that O_i is at rest (they rescale it in place when the reference
+// maximum moves).
 constexpr int kSoftmaxWarps = 8, kDequantWarps = 8;   // dequant: 4 warps for keys, 4 for values
 constexpr int kP2Threads = (kSoftmaxWarps + kDequantWarps + 1) * 32;
-constexpr int kTmemCols2 = 512;                // S_0, S_1, O_0, O_1: 128 columns each
+constexpr int kTmemCols2 = 512;
 constexpr float kRescaleSlack = 8.0f;          // base-2 units: weights stay below 2^8
+constexpr int kStages = 2;
+constexpr int kStageBytes = kKvBlock * 128 * 2;  // one K^ / V^ stage
+constexpr int kQTileBytes = kQTile * 128 * 2;
 
-enum { BAR_KFULL = 0, BAR_VFULL, BAR_SFULL0, BAR_SFULL1, BAR_PFULL0, BAR_PFULL1, BAR_OFULL0, BAR_OFULL1, BAR_COUNT };
+enum { BAR_KFULL = 0, BAR_VFULL = kStages, BAR_KFREE = 2 * kStages, BAR_VFREE = 3 * kStages,
+       BAR_SFULL = 4 * kStages, BAR_PFULL = 4 * kStages + 2, BAR_OFULL = 4 * kStages + 4, BAR_COUNT = 4 * kStages + 6 };
 
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) {
+// 32 consecutive 32-bit columns of this thread's tensor-memory lane
+__device__ __forceinline__ void tmem_st32u(uint32_t taddr, const uint32_t (&v)[32]) {
   asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
                "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
                "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};\n"
                ::"r"(taddr),
-                 "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])), "r"(__float_as_uint(v[3])),
-                 "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])), "r"(__float_as_uint(v[7])),
-                 "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])), "r"(__float_as_uint(v[11])),
-                 "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15])),
-                 "r"(__float_as_uint(v[16])), "r"(__float_as_uint(v[17])), "r"(__float_as_uint(v[18])), "r"(__float_as_uint(v[19])),
-                 "r"(__float_as_uint(v[20])), "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])), "r"(__float_as_uint(v[23])),
-                 "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])), "r"(__float_as_uint(v[26])), "r"(__float_as_uint(v[27])),
-                 "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31]))
+                 "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+                 "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]),
+                 "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]),
+                 "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
                : "memory");
   asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) {
+  uint32_t r[32];
+#pragma unroll
+  for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(v[i]);
+  tmem_st32u(taddr, r);
+}
+
+// 16 consecutive 32-bit columns; the store is not waited for here (tmem_st_wait)
+__device__ __forceinline__ void tmem_st16u_nowait(uint32_t taddr, const uint32_t (&v)[16]) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+               "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};\n"
+               ::"r"(taddr),
+                 "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+                 "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+               : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory"); }
+__device__ __forceinline__ void tmem_ld16u(uint32_t (&r)[16], uint32_t taddr) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+               "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];\n"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                 "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+               : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
 }
 
 // Where the cache of one (layer, sequence, kv head) lives, and how to reach a 32-token tile of it.
@@ -347,20 +402,22 @@ prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T
                     float* __restrict__ out) {
   extern __shared__ __align__(128) uint8_t smem[];
   uint8_t* sQ = smem;                               // two query tiles
-  uint8_t* sK = smem + 2 * kOperandBytes;
-  uint8_t* sV = smem + 3 * kOperandBytes;
-  uint8_t* sP = smem + 4 * kOperandBytes;           // two probability tiles
-  uint64_t* bar_mem = reinterpret_cast<uint64_t*>(smem + 6 * kOperandBytes);
+  uint8_t* sK = sQ + 2 * kQTileBytes;               // kStages blocks
+  uint8_t* sV = sK + kStages * kStageBytes;         // kStages blocks
+  uint64_t* bar_mem = reinterpret_cast<uint64_t*>(sV + kStages * kStageBytes);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_mem + BAR_COUNT);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const uint32_t bar0 = smem_addr(bar_mem);
   auto bar = [&](int i) { return bar0 + 8u * i; };
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int pair = blockIdx.x, hq = blockIdx.y, b = blockIdx.z;
+  const int pair = gridDim.x - 1 - blockIdx.x;      // longest rows of blocks first
+  const int hq = blockIdx.y, b = blockIdx.z;
   const int H = dm.n_kv_heads, Hq = dm.n_q_heads;
   const int h = hq / (Hq / H);
-  const int n_blocks = min(2 * pair + 2, (T + kKvBlock - 1) / kKvBlock);
+  // blocks that tile i can see: up to the one holding its last row's own position
+  const int nb_all = (T + kKvBlock - 1) / kKvBlock;
+  const int nb0 = min(2 * pair + 1, nb_all), nb1 = min(2 * pair + 2, nb_all);
 
   if (warp == kSoftmaxWarps + kDequantWarps) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_addr(tmem_slot)), "r"(kTmemCols2) : "memory");
@@ -368,7 +425,7 @@ prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T
   }
   if (tid == 0) {
     for (int i = 0; i < BAR_COUNT; ++i) {
-      const int count = (i == BAR_KFULL || i == BAR_VFULL) ? kDequantWarps / 2 : (i == BAR_PFULL0 || i == BAR_PFULL1) ? 4 : 1;
+      const int count = (i < BAR_KFREE || (i >= BAR_PFULL && i < BAR_OFULL)) ? 4 : 1;
       asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar(i)), "r"(count) : "memory");
     }
     *abort_flag = 0;
@@ -381,7 +438,7 @@ prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T
     uint4 v = make_uint4(0u, 0u, 0u, 0u);
     if (pos < T)
       v = to_fp16x8<BF16>(__ldg(reinterpret_cast<const uint4*>(Q + ((static_cast<long long>(b) * T + pos) * Hq + hq) * kHeadDim + 8 * U)));
-    *reinterpret_cast<uint4*>(sQ + (row >> 7) * kOperandBytes + kmajor_unit_offset(row & 127, U)) = v;
+    *reinterpret_cast<uint4*>(sQ + (row >> 7) * kQTileBytes + kmajor_unit_offset<128>(row & 127, U)) = v;
   }
   fence_async_proxy();
   tc_fence_before();
@@ -392,106 +449,97 @@ prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T
   // bounded wait that also gives up when another role has given up
   auto wait = [&](int which, int completion) -> bool {
     const uint32_t a = bar(which), parity = static_cast<uint32_t>(completion) & 1u;
-    for (long long it = 0; it < kWaitLimitP; ++it) {
+    if (mbar_try_wait_p(a, parity)) return true;
+    const long long t0 = clock64();
+    while (!*abort_flag) {
       if (mbar_try_wait_p(a, parity)) return true;
-      if ((it & 1023) == 1023 && *abort_flag) return false;
+      if (clock64() - t0 > kWaitCycles) *abort_flag = 1;
     }
-    *abort_flag = 1;
     return false;
   };
 
   if (warp < kSoftmaxWarps) {
     // ================= softmax: one query row per thread =================
     const int i = warp >> 2;                        // query tile of this warp
+    const int nb = i ? nb1 : nb0;
     const int row = tid & 127;
     const int qpos = (2 * pair + i) * kQTile + row;
     const uint32_t lane_addr = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
     const uint32_t s_addr = lane_addr + 128 * i, o_addr = lane_addr + 256 + 128 * i;
-    uint8_t* sPi = sP + i * kOperandBytes;
+    // The reference maximum m_ref is an integer (base-2 units), so that a move of it rescales
+    // what is already stored by an exact power of two.
     float m_ref = -INFINITY, l = 0.0f;
     bool ok = true;
-    for (int kb = 0; kb < n_blocks && ok; ++kb) {
-      ok = __all_sync(0xffffffffu, wait(BAR_SFULL0 + i, kb));
+    for (int kb = 0; kb < nb && ok; ++kb) {
+      ok = __all_sync(0xffffffffu, wait(BAR_SFULL + i, kb));
       if (!ok) break;
       tc_fence_after();
-      if (kb > 0) {                                  // P_i and O_i are busy until the previous block's PV is done
-        ok = __all_sync(0xffffffffu, wait(BAR_OFULL0 + i, kb - 1));
-        if (!ok) break;
-        tc_fence_after();
-      }
-      // Blocks left of the diagonal are fully visible; only the last one or two need the mask.
+      // Blocks left of the diagonal are fully visible; only the last one needs the mask.
       const bool diag = kb >= 2 * pair + i;
       const int rel = qpos - kb * kKvBlock;          // columns 0..rel of this block are visible
-      // One pass over S_i: weights against the reference maximum `mref` into P_i, their sum, and
-      // the largest score seen.
-      auto emit = [&](float mref, float& sum, float& mx) {
-        sum = 0.0f;
-        mx = -INFINITY;
+      float sum = 0.0f;
 #pragma unroll 1
-        for (int c4 = 0; c4 < 4; ++c4) {
-          float v[32];
-          tmem_ld32(v, s_addr + 32 * c4);
-          uint32_t pk[16];
-#pragma unroll
-          for (int e2 = 0; e2 < 16; ++e2) {
-            float x0 = v[2 * e2] * scale_log2, x1 = v[2 * e2 + 1] * scale_log2;
-            if (diag) {
-              if (32 * c4 + 2 * e2 > rel) x0 = -INFINITY;
-              if (32 * c4 + 2 * e2 + 1 > rel) x1 = -INFINITY;
-            }
-            mx = fmaxf(mx, fmaxf(x0, x1));
-            const float p0 = ex2_approx(x0 - mref), p1 = ex2_approx(x1 - mref);
-            sum += p0 + p1;
-            pk[e2] = pack_h2(p0, p1);
-          }
-#pragma unroll
-          for (int u = 0; u < 4; ++u)
-            *reinterpret_cast<uint4*>(sPi + kmajor_unit_offset(row, 4 * c4 + u)) = make_uint4(pk[4 * u], pk[4 * u + 1], pk[4 * u + 2], pk[4 * u + 3]);
-        }
-      };
-      float sum, mx;
-      bool move = (kb == 0);                         // the first block has no reference yet
-      if (!move) {
-        // optimistic single pass against the current reference; it stands unless some row of the
-        // warp found a score more than kRescaleSlack above its reference
-        emit(m_ref, sum, mx);
-        move = __any_sync(0xffffffffu, mx > m_ref + kRescaleSlack);
-      } else {
-        mx = -INFINITY;
-#pragma unroll 1
-        for (int c4 = 0; c4 < 4; ++c4) {
-          float v[32];
-          tmem_ld32(v, s_addr + 32 * c4);
+      for (int c4 = 0; c4 < kKvBlock / 32; ++c4) {
+        float v[32];
+        tmem_ld32(v, s_addr + 32 * c4);
+        if (diag) {
 #pragma unroll
           for (int e = 0; e < 32; ++e)
-            if (!diag || 32 * c4 + e <= rel) mx = fmaxf(mx, v[e] * scale_log2);
+            if (32 * c4 + e > rel) v[e] = -INFINITY;
         }
-      }
-      if (move) {
-        const float m_new = fmaxf(m_ref, mx);
-        if (kb > 0) {
-          const float corr = (m_ref == -INFINITY) ? 0.0f : ex2_approx(m_ref - m_new);
-#pragma unroll 1
-          for (int c4 = 0; c4 < 4; ++c4) {
-            float v[32];
-            tmem_ld32(v, o_addr + 32 * c4);
+        float mx = v[0];
 #pragma unroll
-            for (int e = 0; e < 32; ++e) v[e] *= corr;
-            tmem_st32(o_addr + 32 * c4, v);
+        for (int e = 1; e < 32; ++e) mx = fmaxf(mx, v[e]);
+        mx *= scale_log2;                            // scale_log2 > 0
+        if (__any_sync(0xffffffffu, mx > m_ref + kRescaleSlack)) {
+          // Rare: some row of the warp found a score far above its reference.  Move the reference
+          // and rescale what was accumulated against the old one: O_i (at rest: S_i of this block
+          // was issued after the last O_i += P_i V^), the running sums, and the chunks of P_i already
+          // written for this block.
+          const float m_new = fmaxf(m_ref, ceilf(mx));
+          const float corr = (m_ref == -INFINITY) ? 0.0f : ex2_approx(m_ref - m_new);
+          if (kb > 0) {
+#pragma unroll 1
+            for (int o4 = 0; o4 < 4; ++o4) {
+              float o[32];
+              tmem_ld32(o, o_addr + 32 * o4);
+#pragma unroll
+              for (int e = 0; e < 32; ++e) o[e] *= corr;
+              tmem_st32(o_addr + 32 * o4, o);
+            }
+          }
+          tmem_st_wait();
+#pragma unroll 1
+          for (int p4 = 0; p4 < c4; ++p4) {
+            uint32_t pw[16];
+            tmem_ld16u(pw, s_addr + 16 * p4);
+#pragma unroll
+            for (int e = 0; e < 16; ++e) {
+              const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&pw[e]));
+              pw[e] = pack_h2(f.x * corr, f.y * corr);
+            }
+            tmem_st16u_nowait(s_addr + 16 * p4, pw);
           }
           l *= corr;
+          sum *= corr;
+          m_ref = m_new;
         }
-        m_ref = m_new;
-        float mx2;
-        emit(m_ref, sum, mx2);
+        uint32_t pk[16];
+#pragma unroll
+        for (int e2 = 0; e2 < 16; ++e2) {
+          const float p0 = ex2_approx(fmaf(v[2 * e2], scale_log2, -m_ref)), p1 = ex2_approx(fmaf(v[2 * e2 + 1], scale_log2, -m_ref));
+          sum += p0 + p1;
+          pk[e2] = pack_h2(p0, p1);
+        }
+        tmem_st16u_nowait(s_addr + 16 * c4, pk);     // columns already read: 16 (c4 + 1) <= 32 (c4 + 1)
       }
       l += sum;
-      fence_async_proxy();
+      tmem_st_wait();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar(BAR_PFULL0 + i));
+      if (lane == 0) mbar_arrive(bar(BAR_PFULL + i));
     }
-    if (ok && n_blocks > 0) ok = __all_sync(0xffffffffu, wait(BAR_OFULL0 + i, n_blocks - 1));
+    if (ok && nb > 0) ok = __all_sync(0xffffffffu, wait(BAR_OFULL + i, 0));
     if (ok) {
       tc_fence_after();
       const float inv = l > 0.0f ? 1.0f / l : 0.0f;
@@ -509,9 +557,10 @@ prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T
       set_status(cv.status, MOQAE_ERR_TIMEOUT, blockIdx.x, warp);
     }
   } else if (warp < kSoftmaxWarps + kDequantWarps) {
-    // ================= dequantise: storage tile `sub` of every block, keys then values =================
-    const int sub = (warp - kSoftmaxWarps) & 3;
-    const bool is_v = (warp - kSoftmaxWarps) >= 4;
+    // ================= dequantise: storage tile `sub` of every block =================
+    const int dw = warp - kSoftmaxWarps;
+    const bool is_v = dw >= 4;
+    const int sub = dw & 3;
     KvSource ks;
     ks.cv = &cv; ks.dm = &dm; ks.layer = layer; ks.b = b; ks.h = h;
     const int group = layer / dm.rs_group;
@@ -521,47 +570,69 @@ prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T
     ks.tail_len = min(cv.tail_len[layer * dm.batch + b], dm.tail_capacity);
     ks.tpc = dm.chunk / kTileTokens;
     ks.tail_base = ((static_cast<long long>(layer) * dm.batch + b) * H + h) * dm.tail_capacity;
-    for (int kb = 0; kb < n_blocks; ++kb) {
+    for (int kb = 0; kb < nb1; ++kb) {
+      const int st = kb % kStages;
       const int pos0 = kb * kKvBlock + sub * kTileTokens;
-      // K^ is free once both S products of the last block are done, V^ once both PV products are
-      if (kb > 0 && !wait(is_v ? BAR_OFULL1 : BAR_SFULL1, kb - 1)) break;
-      dequant_subtile<BF16>(ks, pos0, sub, is_v, is_v ? sV : sK, lane);
+      // the stage is free once the products that read it kStages blocks back are done
+      if (kb >= kStages && !wait((is_v ? BAR_VFREE : BAR_KFREE) + st, kb / kStages - 1)) break;
+      dequant_subtile<BF16>(ks, pos0, sub, is_v, (is_v ? sV : sK) + st * kStageBytes, lane);
       fence_async_proxy();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar(is_v ? BAR_VFULL : BAR_KFULL));
+      if (lane == 0) mbar_arrive(bar((is_v ? BAR_VFULL : BAR_KFULL) + st));
     }
   } else {
     // ================= MMA issue (one thread) =================
-    const uint32_t aQ = smem_addr(sQ), aK = smem_addr(sK), aV = smem_addr(sV), aP = smem_addr(sP);
-    bool ok = true;
-    for (int kb = 0; kb < n_blocks && ok; ++kb) {
-      ok = wait(BAR_KFULL, kb);
-      for (int i = 0; i < 2 && ok; ++i) {
-        if (kb > 0) ok = wait(BAR_PFULL0 + i, kb - 1);         // S_i of the last block has been read
-        if (!ok) break;
-        tc_fence_after();
-        if (lane == 0) {
+    // descriptors of stage 0, K step 0; a stage adds kStageBytes / 16 to the low word, a K step
+    // (two 2 KiB slabs of 8 channels or 8 tokens) 256
+    const uint64_t qd = make_desc(smem_addr(sQ), 2048, 128), kd = make_desc(smem_addr(sK), 2048, 128), vd = make_desc(smem_addr(sV), 2048, 128);
+    const uint32_t qd_lo = static_cast<uint32_t>(qd), qd_hi = static_cast<uint32_t>(qd >> 32);
+    const uint32_t kd_lo = static_cast<uint32_t>(kd), kd_hi = static_cast<uint32_t>(kd >> 32);
+    const uint32_t vd_lo = static_cast<uint32_t>(vd), vd_hi = static_cast<uint32_t>(vd >> 32);
+    // S_i = Q_i K^[st]^T: K = 128 channels in 8 steps of 16; the last product that reads K^[st]
+    // (tile 1) also frees the stage
+    auto issue_s = [&](int i, int kb) {
+      const int st = kb % kStages;
+      if (lane == 0) {
+        const uint32_t a_lo = qd_lo + i * (kQTileBytes >> 4), b_lo = kd_lo + st * (kStageBytes >> 4), d = tmem + 128 * i;
 #pragma unroll
-          for (int k = 0; k < 8; ++k)
-            umma_f16(tmem + 128 * i, make_desc(aQ + i * kOperandBytes + k * 4096, 2048, 128), make_desc(aK + k * 4096, 2048, 128),
-                     kIdescKK, k > 0);
-          umma_commit(bar(BAR_SFULL0 + i));
-        }
-        __syncwarp();
+        for (int k = 0; k < 8; ++k) umma_f16_ss(d, a_lo + 256 * k, qd_hi, b_lo + 256 * k, kd_hi, kIdescS, k > 0);
+        umma_commit(bar(BAR_SFULL + i));
+        if (i == 1) umma_commit(bar(BAR_KFREE + st));
       }
-      if (ok) ok = wait(BAR_VFULL, kb);
+      __syncwarp();
+    };
+    // O_i += P_i V^[st]: K = 128 tokens in 8 steps of 16
+    auto issue_pv = [&](int i, int kb, bool last) {
+      const int st = kb % kStages;
+      if (lane == 0) {
+        const uint32_t lo = vd_lo + st * (kStageBytes >> 4), d = tmem + 256 + 128 * i, a = tmem + 128 * i;
+        umma_f16_ta(d, a, lo, vd_hi, kIdescPV, kb > 0);
+#pragma unroll
+        for (int k = 1; k < 8; ++k) umma_f16_ta(d, a + 8 * k, lo + 256 * k, vd_hi, kIdescPV, 1u);
+        if (i == 1) umma_commit(bar(BAR_VFREE + st));
+        if (last) umma_commit(bar(BAR_OFULL + i));
+      }
+      __syncwarp();
+    };
+    bool ok = wait(BAR_KFULL, 0);
+    if (ok) {
+      tc_fence_after();
+      issue_s(0, 0);
+      issue_s(1, 0);
+    }
+    // Block kb, tile by tile: O_i += P_i V^ as soon as P_i is there, then at once S_i of the next
+    // block; the other tile's products run while this tile's softmax threads work on it.
+    for (int kb = 0; kb < nb1 && ok; ++kb) {
+      ok = wait(BAR_VFULL + kb % kStages, kb / kStages);
+      if (ok && kb + 1 < nb1) ok = wait(BAR_KFULL + (kb + 1) % kStages, (kb + 1) / kStages);
       for (int i = 0; i < 2 && ok; ++i) {
-        ok = wait(BAR_PFULL0 + i, kb);
+        const int nb = i ? nb1 : nb0;
+        if (kb >= nb) continue;
+        ok = wait(BAR_PFULL + i, kb);
         if (!ok) break;
         tc_fence_after();
-        if (lane == 0) {
-#pragma unroll
-          for (int k = 0; k < 8; ++k)
-            umma_f16(tmem + 256 + 128 * i, make_desc(aP + i * kOperandBytes + k * 4096, 2048, 128), make_desc(aV + k * 4096, 2048, 128),
-                     kIdescKMN, (kb > 0 || k > 0) ? 1u : 0u);
-          umma_commit(bar(BAR_OFULL0 + i));
-        }
-        __syncwarp();
+        issue_pv(i, kb, kb + 1 == nb);
+        if (kb + 1 < nb) issue_s(i, kb + 1);
       }
     }
   }
@@ -576,7 +647,7 @@ prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T
 cudaError_t launch_prefill_attn(const Dims& dm, const CacheView& cv, const void* q, int T, int layer, float scale,
                                 float* out, cudaStream_t st) {
   if (T <= 0) return cudaSuccess;
-  const size_t smem = 6 * kOperandBytes + BAR_COUNT * 8 + 16;
+  const size_t smem = 2 * kQTileBytes + 2 * kStages * kStageBytes + BAR_COUNT * 8 + 16;
   dim3 grid((T + 2 * kQTile - 1) / (2 * kQTile), dm.n_q_heads, dm.batch);
   const float scale_log2 = scale * 1.4426950408889634f;
   cudaError_t e;

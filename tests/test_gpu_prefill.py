@@ -1,7 +1,9 @@
 """GPU parity: moqae_prefill_attn (causal attention of the prompt over its quantised cache) against
-the oracle on the same packed cache.  The kernel rounds the dequantised rows and the softmax
-weights to fp16 before its tensor-core products, so the bound is the fp16 rounding of V̂ and P:
-|err| <= 4e-3 and, per (sequence, position, head) row, max|err| / max|ref| <= 1e-2."""
+the oracle on the same packed cache.  The kernel rounds three things to fp16 before its
+tensor-core products: the dequantised keys (which perturbs the scores), the softmax weights P
+and the dequantised values.  Each rounding is at most 2^-11 relative, and a row whose softmax
+is dominated by one token passes them on undamped, so the bound is
+|err| <= 3 * 2^-11 * max|V| and, per (sequence, position, head) row, max|err| / max|ref| <= 1e-2."""
 import numpy as np
 import pytest
 import torch
@@ -31,7 +33,8 @@ def prefill_case(B, T, Hq, Hkv, chunk, dtype, bmap, seed):
     assert mq.moqae_poll_status(cache) == 0
     got = out.cpu().numpy().astype(np.float64)
     assert np.isfinite(got).all()
-    ok, e_abs, e_rel = H.attn_tolerance_ok(got.reshape(1, -1, 128), ref.reshape(1, -1, 128), abs_tol=4e-3, rel_tol=1e-2)
+    abs_tol = 3 * 2.0 ** -11 * float(V.float().abs().max())
+    ok, e_abs, e_rel = H.attn_tolerance_ok(got.reshape(1, -1, 128), ref.reshape(1, -1, 128), abs_tol=abs_tol, rel_tol=1e-2)
     assert ok, (e_abs, e_rel)
     return e_abs, e_rel
 
