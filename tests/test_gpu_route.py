@@ -12,9 +12,9 @@ pytestmark = pytest.mark.gpu
 TAU = 1e-4      # a token whose top-2 logits differ by less than TAU * max|P| may flip in float32
 
 
-def check_route(B, T, D, chunk, dtype, gated, rf, seed, bias=None, w_std=0.02):
+def check_route(B, T, D, chunk, dtype, gated, rf, seed, bias=None, w_std=0.02, weights=None, abs_margin=None):
     hid = synth.hidden_states(B, T, D, chunk, dtype, seed, "cpu")
-    W1, W2, W3, b0 = synth.router_weights(D, 4, dtype, seed + 1, "cpu", std=w_std, gated=gated)
+    W1, W2, W3, b0 = weights or synth.router_weights(D, 4, dtype, seed + 1, "cpu", std=w_std, gated=gated)
     if bias is not None:
         b0 = torch.tensor(bias, dtype=torch.float32)
     ref = O.route(synth.to_u16(hid), dtype, chunk, synth.to_u16(W1),
@@ -36,7 +36,8 @@ def check_route(B, T, D, chunk, dtype, gated, rf, seed, bias=None, w_std=0.02):
     for b in range(B):
         for c in range(C):
             sl = slice(c * chunk, (c + 1) * chunk)
-            frag = np.where(ref["margin"][b, sl] < TAU * np.maximum(ref["pmax"][b, sl], 1e-30))[0]
+            thr = abs_margin if abs_margin is not None else TAU * np.maximum(ref["pmax"][b, sl], 1e-30)
+            frag = np.where(ref["margin"][b, sl] < thr)[0]
             diff = got_votes[b, c].astype(np.int64) - ref["votes"][b, c]
             assert diff.sum() == 0
             assert np.abs(diff).sum() // 2 <= len(frag), (b, c, diff, len(frag))
@@ -124,3 +125,23 @@ def test_routing_sharing_groups_are_independent_tables():
 def test_route_input_widths_that_are_not_whole_boxes(D):
     # the hidden rows arrive in 64-channel boxes: widths below one box and with a ragged last box
     check_route(2, 64 * 4 + 3, D, 64, 1, True, True, seed=D, w_std=0.1)
+
+
+def test_three_expert_set_through_a_masked_logit():
+    # the {2, 4, 16}-bit expert set of the ablation: zero weights and an unreachable bias for the
+    # 8-bit expert; the GPU router must never choose it and must match the oracle elsewhere
+    D, chunk, dtype = 256, 64, 1
+    W1, W2, W3, b = synth.router_weights(D, 3, dtype, 91, "cpu", std=0.1)
+    keep = [0, 1, 3]
+    W1_4 = torch.zeros(D, 4, dtype=W1.dtype); W1_4[:, keep] = W1
+    W2_4 = torch.zeros(D, 4, dtype=W2.dtype); W2_4[:, keep] = W2
+    W3_4 = torch.zeros(4, 4)
+    for i, ki in enumerate(keep):
+        for j, kj in enumerate(keep):
+            W3_4[ki, kj] = W3[i, j]
+    b_4 = torch.full((4,), -3.0e38); b_4[keep] = b
+    # the masked logit would blow up a tolerance relative to max|P|: near-ties are judged against
+    # the size of the live logits (a few units) instead
+    n_frag, n_chunks, m = check_route(2, chunk * 12 + 9, D, chunk, dtype, True, True, seed=90,
+                                      weights=(W1_4, W2_4, W3_4, b_4), abs_margin=1e-3)
+    assert not (m == 2).any() and len(np.unique(m)) > 1 and n_frag < n_chunks // 2

@@ -126,3 +126,30 @@ def test_reachable_winners():
     assert O.reachable_winners(v, [], []) == {0}
     assert O.reachable_winners(v, [0], [1]) == {0, 1}
     assert O.reachable_winners(np.array([9, 1, 0, 0]), [0], [1]) == {0}
+
+
+def _embed_three_experts(W1, W2, W3, bias):
+    """A {2, 4, 16}-bit router written as the four-expert one: the 8-bit expert gets zero weights
+    and a logit no token can choose."""
+    keep = [0, 1, 3]
+    W1_4 = np.zeros((W1.shape[0], 4), W1.dtype); W1_4[:, keep] = W1
+    W2_4 = np.zeros((W2.shape[0], 4), W2.dtype); W2_4[:, keep] = W2
+    W3_4 = np.zeros((4, 4), np.float32); W3_4[np.ix_(keep, keep)] = W3
+    b_4 = np.full(4, -3.0e38, np.float32); b_4[keep] = bias
+    return W1_4, W2_4, W3_4, b_4
+
+
+def test_three_expert_set_is_the_four_expert_router_with_one_logit_masked():
+    # the ablation with M = 3 experts {2, 4, 16 bits} (Section 4.4): its router, run with M = 3 in
+    # the oracle, chooses exactly what the M = 4 router chooses when the 8-bit expert is masked
+    rs = RS(11)
+    B, T, D, N = 2, 32 * 9 + 5, 24, 32
+    hid = f16bits(rs.randn(B, T, D))
+    W1, W2 = f16bits(rs.randn(D, 3) * 0.5), f16bits(rs.randn(D, 3) * 0.5)
+    W3, bias = rs.randn(3, 3).astype(np.float32), (rs.randn(3) * 0.1).astype(np.float32)
+    r3 = O.route(hid, 0, N, W1, W2, W3, bias, rf_first_chunk=True)
+    r4 = O.route(hid, 0, N, *_embed_three_experts(W1, W2, W3, bias), rf_first_chunk=True)
+    widths = np.array([0, 1, 3], np.uint8)              # expert index of the 3-set -> index of the 4-set
+    assert (widths[r3["map"]] == r4["map"]).all()
+    assert (r4["votes"][:, :, [0, 1, 3]] == r3["votes"]).all() and (r4["votes"][:, :, 2] == 0).all()
+    assert (r4["map"][:, 0] == 3).all() and len(np.unique(r4["map"])) > 1
