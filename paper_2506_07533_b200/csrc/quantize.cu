@@ -26,7 +26,8 @@ constexpr int kInBytes = 8192;                 // 32 rows x 256 B
 constexpr int kOutBytes = 9216;                // largest quantised tile
 constexpr int kPrmBytes = 1024;                // value groups: [32 tokens][4 groups] (zero, 1/scale)
 constexpr int kWarpSmem = 2 * kInBytes + kOutBytes + kPrmBytes;
-constexpr long long kWaitLimit = 1ll << 22;
+constexpr long long kWaitCycles = 1ll << 30;  // a bounded wait gives up after this many SM cycles
+constexpr uint32_t kSuspendNs = 20000;         // how long one try_wait may keep the warp parked
 constexpr float kMagic = 12582912.0f;          // 1.5 * 2^23
 constexpr int kSkipTile = 0xfe;                // width marker: nothing to do for this tile
 
@@ -57,15 +58,21 @@ __device__ __forceinline__ void bulk_store_wait_all() {
 __device__ __forceinline__ void fence_async_smem() {
   asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
 }
+// One try_wait with a suspend-time hint: the hardware parks the warp until the phase completes
+// or the hint runs out, so a waiting warp takes no issue slots from the working ones.
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
-  asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
-               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\nselp.u32 %0, 1, 0, p;\n}\n"
+               : "=r"(ok) : "r"(bar), "r"(parity), "r"(kSuspendNs) : "memory");
   return ok != 0;
 }
+// Bounded by elapsed SM cycles (about half a second), not by the number of attempts.
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
-  for (long long i = 0; i < kWaitLimit; ++i)
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  do {
     if (mbar_try_wait(bar, parity)) return true;
+  } while (clock64() - t0 < kWaitCycles);
   return false;
 }
 
