@@ -240,9 +240,18 @@ int moqae_decode_attn(const moqae_config* cfg, const void* q, int32_t layer,
  *   T must be the number of tokens the cache of `layer` holds for every sequence
  *   (chunks * chunk + tail_len), i.e. call it after moqae_quantize_kv of the same prompt.
  *   scale <= 0 selects 1/sqrt(128).
+ *   workspace: NULL, or caller-owned device scratch of at least moqae_prefill_attn_workspace()
+ *   bytes (2 * batch * n_kv_heads * round_up(T, 128) * 256), 16-byte aligned.  With a workspace the
+ *   layer's cache is expanded once into fp16 rows there and every CTA fetches its blocks from it
+ *   (faster: without it each CTA expands the packed tiles it walks over again, but no extra
+ *   memory is needed).  Both ways compute the same quantity; the workspace holds nothing the
+ *   caller needs afterwards.  Errors: MOQAE_ERR_WORKSPACE_TOO_SMALL, MOQAE_ERR_MISALIGNED,
+ *   MOQAE_ERR_INVALID_ARG (T outside [0, max_tokens], bad layer, missing pointers).
  */
+int moqae_prefill_attn_workspace(const moqae_config* cfg, int32_t T, int64_t* bytes);
 int moqae_prefill_attn(const moqae_config* cfg, const void* q, int32_t T, int32_t layer,
-                       const moqae_cache* cache, float* out, float scale, void* stream);
+                       const moqae_cache* cache, float* out, float scale, void* workspace,
+                       int64_t workspace_bytes, void* stream);
 
 /*
  * (No counterpart in the paper: this entry point exists for deployment reasons only.)

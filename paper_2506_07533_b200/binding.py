@@ -25,7 +25,7 @@ ERR_WORKSPACE_TOO_SMALL, ERR_CUDA, ERR_TIMEOUT = -5, -6, -7
 EXPORTS = ["moqae_version", "moqae_last_cuda_error", "moqae_error_string", "moqae_cache_bytes",
            "moqae_cache_bind", "moqae_route", "moqae_quantize_kv", "moqae_append_kv",
            "moqae_decode_attn_workspace", "moqae_decode_attn", "moqae_poll_status",
-           "moqae_decode_attn_static", "moqae_decode_attn_static_max_bytes", "moqae_flush_tail", "moqae_prefill_attn"]
+           "moqae_decode_attn_static", "moqae_decode_attn_static_max_bytes", "moqae_flush_tail", "moqae_prefill_attn", "moqae_prefill_attn_workspace"]
 
 
 class MoqaeConfig(C.Structure):
@@ -85,7 +85,8 @@ def lib() -> C.CDLL:
         L.moqae_flush_tail.argtypes = [C.POINTER(MoqaeConfig), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                        C.c_void_p, C.c_int32, C.POINTER(MoqaeCache), C.c_void_p]
         L.moqae_prefill_attn.argtypes = [C.POINTER(MoqaeConfig), C.c_void_p, C.c_int32, C.c_int32,
-                                         C.POINTER(MoqaeCache), C.c_void_p, C.c_float, C.c_void_p]
+                                         C.POINTER(MoqaeCache), C.c_void_p, C.c_float, C.c_void_p, C.c_int64, C.c_void_p]
+        L.moqae_prefill_attn_workspace.argtypes = [C.POINTER(MoqaeConfig), C.c_int32, C.POINTER(C.c_int64)]
         L.moqae_decode_attn_workspace.argtypes = [C.POINTER(MoqaeConfig), C.POINTER(C.c_int64)]
         L.moqae_decode_attn.argtypes = [C.POINTER(MoqaeConfig), C.c_void_p, C.c_int32, C.POINTER(MoqaeCache),
                                         C.c_void_p, C.c_float, C.c_void_p, C.c_int64, C.c_void_p]
@@ -231,9 +232,16 @@ def moqae_flush_tail(cfg, hidden_tail, W1, W2, W3, bias, layer_group, cache: Cac
                                   int(layer_group), C.byref(cache.view), _stream()), "moqae_flush_tail")
 
 
-def moqae_prefill_attn(cfg, q, T, layer, cache: Cache, out, scale=0.0):
+def moqae_prefill_attn_workspace(cfg, T) -> int:
+    out = C.c_int64(0)
+    _check(lib().moqae_prefill_attn_workspace(C.byref(cfg), int(T), C.byref(out)), "moqae_prefill_attn_workspace")
+    return int(out.value)
+
+
+def moqae_prefill_attn(cfg, q, T, layer, cache: Cache, out, scale=0.0, workspace=None):
+    nbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     _check(lib().moqae_prefill_attn(C.byref(cfg), _ptr(q), int(T), int(layer), C.byref(cache.view), _ptr(out),
-                                    C.c_float(scale), _stream()), "moqae_prefill_attn")
+                                    C.c_float(scale), _ptr(workspace), C.c_int64(nbytes), _stream()), "moqae_prefill_attn")
 
 
 def moqae_decode_attn_workspace(cfg) -> int:

@@ -251,8 +251,16 @@ int moqae_decode_attn(const moqae_config* cfg, const void* q, int32_t layer, con
   return e == cudaSuccess ? MOQAE_OK : cuda_fail(e);
 }
 
+int moqae_prefill_attn_workspace(const moqae_config* cfg, int32_t T, int64_t* bytes) {
+  int rc = check_config(cfg);
+  if (rc != MOQAE_OK) return rc;
+  if (!bytes || T < 0 || T > cfg->max_tokens) return MOQAE_ERR_INVALID_ARG;
+  *bytes = moqae::prefill_workspace_bytes(dims_of(cfg), T);
+  return MOQAE_OK;
+}
+
 int moqae_prefill_attn(const moqae_config* cfg, const void* q, int32_t T, int32_t layer, const moqae_cache* cache,
-                       float* out, float scale, void* stream) {
+                       float* out, float scale, void* workspace, int64_t workspace_bytes, void* stream) {
   int rc = check_config(cfg);
   if (rc != MOQAE_OK) return rc;
   moqae::CacheView cv;
@@ -260,9 +268,10 @@ int moqae_prefill_attn(const moqae_config* cfg, const void* q, int32_t T, int32_
   if (rc != MOQAE_OK) return rc;
   if (T < 0 || T > cfg->max_tokens || layer < 0 || layer >= cfg->n_layers) return MOQAE_ERR_INVALID_ARG;
   if (T > 0 && (!q || !out)) return MOQAE_ERR_INVALID_ARG;
-  if (!aligned16(q) || !aligned16(out)) return MOQAE_ERR_MISALIGNED;
+  if (!aligned16(q) || !aligned16(out) || !aligned16(workspace)) return MOQAE_ERR_MISALIGNED;
+  if (workspace && workspace_bytes < moqae::prefill_workspace_bytes(dims_of(cfg), T)) return MOQAE_ERR_WORKSPACE_TOO_SMALL;
   if (!(scale > 0.0f)) scale = 0.08838834764831845f;   // 1/sqrt(128)
-  cudaError_t e = moqae::launch_prefill_attn(dims_of(cfg), cv, q, T, layer, scale, out, static_cast<cudaStream_t>(stream));
+  cudaError_t e = moqae::launch_prefill_attn(dims_of(cfg), cv, q, T, layer, scale, out, workspace, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? MOQAE_OK : cuda_fail(e);
 }
 

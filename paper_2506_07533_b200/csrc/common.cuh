@@ -82,7 +82,8 @@ cudaError_t launch_append(const Dims& dm, const CacheView& cv, const void* k_new
 int decode_num_splits(const Dims& dm);
 int decode_mma_ctas_per_sm();
 cudaError_t launch_prefill_attn(const Dims& dm, const CacheView& cv, const void* q, int T, int layer, float scale,
-                                float* out, cudaStream_t st);
+                                float* out, void* workspace, cudaStream_t st);
+long long prefill_workspace_bytes(const Dims& dm, int T);
 long long decode_workspace_bytes(const Dims& dm, int n_splits);
 cudaError_t launch_decode_mma(const Dims& dm, const CacheView& cv, const void* q, int layer, float scale,
                               float* ws_o, float* ws_ml, int* arrived, float* out, int n_splits, cudaStream_t st);

@@ -18,6 +18,9 @@
 // The three roles (softmax, dequantise, MMA issue) run concurrently and meet on mbarriers only.
 // Every wait is bounded; on expiry the CTA records MOQAE_ERR_TIMEOUT, every role stops and the
 // tensor memory is still freed.
+#include <cstring>
+
+#include <cuda.h>
 #include <cuda_bf16.h>
 
 #include "common.cuh"
@@ -110,6 +113,13 @@ __device__ __forceinline__ int mnmajor_unit_offset(int t, int c8) {      // byte
   return ((t >> 3) * 16 + c8) * 128 + (t & 7) * 16;
 }
 
+// Where the dequantising code puts the 16-byte unit (token row t of the block, channels
+// 8 c8 .. 8 c8 + 7): into the operand tile in shared memory, or (ROWS = true) into plain rows of
+// 256 bytes in global memory.
+template <bool ROWS, bool IS_V> __device__ __forceinline__ int dst_unit_offset(int t, int c8) {
+  return ROWS ? t * 256 + c8 * 16 : (IS_V ? mnmajor_unit_offset(t, c8) : kmajor_unit_offset<128>(t, c8));
+}
+
 __device__ __forceinline__ uint32_t pack_h2(float a, float b) {
   const __half2 h = __floats2half2_rn(a, b);
   return *reinterpret_cast<const uint32_t*>(&h);
@@ -155,7 +165,7 @@ __device__ __forceinline__ uint32_t hfma2_u32(uint32_t a, uint32_t b, uint32_t c
 // Keys.  A payload word masked at one code position carries the codes of channels c and
 // c + n/2 (n = codes per word); the scale and zero arrays hold exactly those pairs, so one
 // packed FMA dequantises two channels: K^ = RN(code * scale + zero) in fp16.
-template <int BITS>
+template <int BITS, bool ROWS>
 __device__ __forceinline__ void dequant_keys(const uint8_t* __restrict__ tile, uint8_t* sK, int sub, int lane) {
   constexpr int n = 32 / BITS, regs = n / 2, direct = n / 4;
   const int g = lane >> 2, t4 = lane & 3;
@@ -212,14 +222,14 @@ __device__ __forceinline__ void dequant_keys(const uint8_t* __restrict__ tile, u
           const int rb = j * regs + (i3 / direct) * direct + i3 % direct;         // register of channel cc + 1
           o[e2] = __byte_perm(byreg[ra], byreg[rb], hi ? 0x7632 : 0x5410);
         }
-        *reinterpret_cast<uint4*>(sK + kmajor_unit_offset<128>(row, 4 * t4 + u)) = make_uint4(o[0], o[1], o[2], o[3]);
+        *reinterpret_cast<uint4*>(sK + dst_unit_offset<ROWS, false>(row, 4 * t4 + u)) = make_uint4(o[0], o[1], o[2], o[3]);
       }
     }
 }
 
 // Values.  A payload word masked at one slot carries the codes of tokens e = 0, 1 of one
 // channel row; the scale and zero arrays hold those token pairs per channel group.
-template <int BITS>
+template <int BITS, bool ROWS>
 __device__ __forceinline__ void dequant_values(const uint8_t* __restrict__ tile, uint8_t* sV, int sub, int lane) {
   constexpr int per = 8 / BITS;                                   // channel rows per word
   const int g = lane >> 2, t4 = lane & 3;
@@ -255,9 +265,9 @@ __device__ __forceinline__ void dequant_values(const uint8_t* __restrict__ tile,
         }
         const int tok = 32 * sub + 16 * blk + 8 * half + 2 * t4;
         // channels 32cg + 4g .. +3: half of the 16-byte unit c8 = 4cg + g/2, one store per token
-        *reinterpret_cast<uint2*>(sV + mnmajor_unit_offset(tok, 4 * cg + (g >> 1)) + (g & 1) * 8) =
+        *reinterpret_cast<uint2*>(sV + dst_unit_offset<ROWS, true>(tok, 4 * cg + (g >> 1)) + (g & 1) * 8) =
             make_uint2(__byte_perm(v[0], v[1], 0x5410), __byte_perm(v[2], v[3], 0x5410));
-        *reinterpret_cast<uint2*>(sV + mnmajor_unit_offset(tok + 1, 4 * cg + (g >> 1)) + (g & 1) * 8) =
+        *reinterpret_cast<uint2*>(sV + dst_unit_offset<ROWS, true>(tok + 1, 4 * cg + (g >> 1)) + (g & 1) * 8) =
             make_uint2(__byte_perm(v[0], v[1], 0x7632), __byte_perm(v[2], v[3], 0x7632));
       }
   }
@@ -266,7 +276,7 @@ __device__ __forceinline__ void dequant_values(const uint8_t* __restrict__ tile,
 // 32 rows of 256 bytes in the input dtype -> one operand tile.  SWIZZLED: rows of a 16-bit
 // pool tile (units permuted inside each row); otherwise plain rows (the tail), of which only
 // the first n_valid exist.
-template <bool BF16, bool SWIZZLED, bool IS_V>
+template <bool BF16, bool SWIZZLED, bool IS_V, bool ROWS>
 __device__ __forceinline__ void copy_rows(const uint8_t* __restrict__ src, uint8_t* dst, int sub, int n_valid, int lane) {
 #pragma unroll 4
   for (int i = 0; i < 16; ++i) {
@@ -275,7 +285,7 @@ __device__ __forceinline__ void copy_rows(const uint8_t* __restrict__ src, uint8
     const int up = SWIZZLED ? ((U & 8) | ((U ^ row) & 7)) : U;
     uint4 v = make_uint4(0u, 0u, 0u, 0u);
     if (row < n_valid) v = to_fp16x8<BF16>(__ldg(reinterpret_cast<const uint4*>(src + row * 256 + up * 16)));
-    const int off = IS_V ? mnmajor_unit_offset(32 * sub + row, U) : kmajor_unit_offset<128>(32 * sub + row, U);
+    const int off = dst_unit_offset<ROWS, IS_V>(32 * sub + row, U);
     *reinterpret_cast<uint4*>(dst + off) = v;
   }
 }
@@ -366,7 +376,20 @@ struct KvSource {
   int layer, b, h, chunk_tokens, tail_len, tpc;
 };
 
-template <bool BF16>
+__device__ __forceinline__ KvSource kv_source(const CacheView& cv, const Dims& dm, int layer, int b, int h) {
+  KvSource ks;
+  ks.cv = &cv; ks.dm = &dm; ks.layer = layer; ks.b = b; ks.h = h;
+  const int group = layer / dm.rs_group;
+  ks.tbl = (static_cast<long long>(group) * dm.batch + b) * dm.max_chunks;
+  const int32_t* cnt = cv.count + (static_cast<long long>(group) * dm.batch + b) * 4;
+  ks.chunk_tokens = min(cnt[0] + cnt[1] + cnt[2] + cnt[3], dm.max_chunks) * dm.chunk;
+  ks.tail_len = min(cv.tail_len[layer * dm.batch + b], dm.tail_capacity);
+  ks.tpc = dm.chunk / kTileTokens;
+  ks.tail_base = ((static_cast<long long>(layer) * dm.batch + b) * dm.n_kv_heads + h) * dm.tail_capacity;
+  return ks;
+}
+
+template <bool BF16, bool ROWS>
 __device__ __forceinline__ void dequant_subtile(const KvSource& ks, int pos0, int sub, bool is_v, uint8_t* dst, int lane) {
   const CacheView& cv = *ks.cv;
   const Dims& dm = *ks.dm;
@@ -382,25 +405,60 @@ __device__ __forceinline__ void dequant_subtile(const KvSource& ks, int pos0, in
     const long long tb = tile_bytes_of_expert(w);
     const long long s = slot < 0 ? 0 : (slot < cap ? slot : cap - 1);          // never leave the pool
     const uint8_t* tile = pool + ((((static_cast<long long>(ks.layer) * dm.batch + ks.b) * dm.n_kv_heads + ks.h) * cap + s) * ks.tpc + j) * tb;
-    if (w == 0) { if (is_v) dequant_values<2>(tile, dst, sub, lane); else dequant_keys<2>(tile, dst, sub, lane); }
-    else if (w == 1) { if (is_v) dequant_values<4>(tile, dst, sub, lane); else dequant_keys<4>(tile, dst, sub, lane); }
-    else if (w == 2) { if (is_v) dequant_values<8>(tile, dst, sub, lane); else dequant_keys<8>(tile, dst, sub, lane); }
-    else if (is_v) copy_rows<BF16, true, true>(tile + 8192, dst, sub, 32, lane);
-    else copy_rows<BF16, true, false>(tile, dst, sub, 32, lane);
+    if (w == 0) { if (is_v) dequant_values<2, ROWS>(tile, dst, sub, lane); else dequant_keys<2, ROWS>(tile, dst, sub, lane); }
+    else if (w == 1) { if (is_v) dequant_values<4, ROWS>(tile, dst, sub, lane); else dequant_keys<4, ROWS>(tile, dst, sub, lane); }
+    else if (w == 2) { if (is_v) dequant_values<8, ROWS>(tile, dst, sub, lane); else dequant_keys<8, ROWS>(tile, dst, sub, lane); }
+    else if (is_v) copy_rows<BF16, true, true, ROWS>(tile + 8192, dst, sub, 32, lane);
+    else copy_rows<BF16, true, false, ROWS>(tile, dst, sub, 32, lane);
   } else {
     const int ti0 = pos0 - ks.chunk_tokens;
     const int n_valid = max(0, min(32, ks.tail_len - ti0));
     const uint8_t* src = reinterpret_cast<const uint8_t*>(is_v ? cv.tail_v : cv.tail_k) + (ks.tail_base + ti0) * 256;
-    if (is_v) copy_rows<BF16, false, true>(src, dst, sub, n_valid, lane);
-    else copy_rows<BF16, false, false>(src, dst, sub, n_valid, lane);
+    if (is_v) copy_rows<BF16, false, true, ROWS>(src, dst, sub, n_valid, lane);
+    else copy_rows<BF16, false, false, ROWS>(src, dst, sub, n_valid, lane);
   }
 }
 
+// ---- dequantise once: the cache of one layer as fp16 rows -----------------------------------
+// K^ and V^ of (sequence b, kv head h) as [t_pad][128] fp16 rows in a caller-provided scratch,
+// t_pad = the prompt length rounded up to whole blocks; rows past the cached tokens are zero.
+// One CTA per 32-token storage tile: warp 0 expands the keys, warp 1 the values.  With this
+// pass in front, the attention kernel below fetches ready-made operand tiles with TMA instead of
+// expanding every tile again in each of the T / 256 CTAs that walk over it.
 template <bool BF16>
+__global__ void __launch_bounds__(64) prefill_dequant_kernel(Dims dm, CacheView cv, int layer, int t_pad, uint8_t* __restrict__ kd,
+                                                             uint8_t* __restrict__ vd) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int pos0 = blockIdx.x * kTileTokens, h = blockIdx.y, b = blockIdx.z;
+  const KvSource ks = kv_source(cv, dm, layer, b, h);
+  uint8_t* dst = (warp ? vd : kd) + ((static_cast<long long>(b) * dm.n_kv_heads + h) * t_pad + pos0) * 256;
+  dequant_subtile<BF16, true>(ks, pos0, 0, warp != 0, dst, lane);
+}
+
+// tiled TMA load of the box whose corner is (x = channel, y = row) into a 128-byte swizzled tile
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];\n"
+               ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
+}
+// Descriptors of the 128-byte swizzled layouts TMA writes (bits 61..63 = 2).  K-major (K^: one
+// row of 64 channels = 128 bytes, 1 KiB between groups of 8 token rows; the leading offset is not
+// used) and MN-major (V^: 64 channels contiguous, 128 bytes between the 8 tokens of a group,
+// leading offset = distance between the two 64-channel halves, stride offset = 1 KiB between
+// groups of 8 tokens).
+__device__ __forceinline__ uint64_t make_desc_sw128(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  return make_desc(saddr, lbo_bytes, sbo_bytes) | (2ull << 61);
+}
+
+template <bool BF16, bool PRE>
 __global__ void __launch_bounds__(kP2Threads, 1)
 prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T, int layer, float scale_log2,
-                    float* __restrict__ out) {
-  extern __shared__ __align__(128) uint8_t smem[];
+                    float* __restrict__ out, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+                    int t_pad) {
+  extern __shared__ __align__(128) uint8_t smem_raw[];
+  uint8_t* smem = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);   // swizzled tiles want 1 KiB alignment
   uint8_t* sQ = smem;                               // two query tiles
   uint8_t* sK = sQ + 2 * kQTileBytes;               // kStages blocks
   uint8_t* sV = sK + kStages * kStageBytes;         // kStages blocks
@@ -425,7 +483,8 @@ prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T
   }
   if (tid == 0) {
     for (int i = 0; i < BAR_COUNT; ++i) {
-      const int count = (i < BAR_KFREE || (i >= BAR_PFULL && i < BAR_OFULL)) ? 4 : 1;
+      // kfull / vfull: four dequantising warps, or the one thread that starts the TMA copies
+      const int count = i < BAR_KFREE ? (PRE ? 1 : 4) : ((i >= BAR_PFULL && i < BAR_OFULL) ? 4 : 1);
       asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar(i)), "r"(count) : "memory");
     }
     *abort_flag = 0;
@@ -556,26 +615,35 @@ prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T
     } else if (lane == 0) {
       set_status(cv.status, MOQAE_ERR_TIMEOUT, blockIdx.x, warp);
     }
+  } else if (PRE && warp < kSoftmaxWarps + kDequantWarps) {
+    // ================= fetch: K^ (warp 8) and V^ (warp 12) blocks from the fp16 scratch by TMA =================
+    const int dw = warp - kSoftmaxWarps;
+    if ((dw == 0 || dw == 4) && lane == 0) {
+      const bool is_v = dw == 4;
+      const CUtensorMap* map = is_v ? &map_v : &map_k;
+      const int row0 = (b * H + h) * t_pad;
+      for (int kb = 0; kb < nb1; ++kb) {
+        const int st = kb % kStages;
+        if (kb >= kStages && !wait((is_v ? BAR_VFREE : BAR_KFREE) + st, kb / kStages - 1)) break;
+        const uint32_t full = bar((is_v ? BAR_VFULL : BAR_KFULL) + st);
+        const uint32_t dst = smem_addr((is_v ? sV : sK) + st * kStageBytes);
+        mbar_expect_tx(full, kStageBytes);
+        tma_load_2d(dst, map, 0, row0 + kb * kKvBlock, full);                    // channels 0..63
+        tma_load_2d(dst + kStageBytes / 2, map, 64, row0 + kb * kKvBlock, full);  // channels 64..127
+      }
+    }
   } else if (warp < kSoftmaxWarps + kDequantWarps) {
     // ================= dequantise: storage tile `sub` of every block =================
     const int dw = warp - kSoftmaxWarps;
     const bool is_v = dw >= 4;
     const int sub = dw & 3;
-    KvSource ks;
-    ks.cv = &cv; ks.dm = &dm; ks.layer = layer; ks.b = b; ks.h = h;
-    const int group = layer / dm.rs_group;
-    ks.tbl = (static_cast<long long>(group) * dm.batch + b) * dm.max_chunks;
-    const int32_t* cnt = cv.count + (static_cast<long long>(group) * dm.batch + b) * 4;
-    ks.chunk_tokens = min(cnt[0] + cnt[1] + cnt[2] + cnt[3], dm.max_chunks) * dm.chunk;
-    ks.tail_len = min(cv.tail_len[layer * dm.batch + b], dm.tail_capacity);
-    ks.tpc = dm.chunk / kTileTokens;
-    ks.tail_base = ((static_cast<long long>(layer) * dm.batch + b) * H + h) * dm.tail_capacity;
+    const KvSource ks = kv_source(cv, dm, layer, b, h);
     for (int kb = 0; kb < nb1; ++kb) {
       const int st = kb % kStages;
       const int pos0 = kb * kKvBlock + sub * kTileTokens;
       // the stage is free once the products that read it kStages blocks back are done
       if (kb >= kStages && !wait((is_v ? BAR_VFREE : BAR_KFREE) + st, kb / kStages - 1)) break;
-      dequant_subtile<BF16>(ks, pos0, sub, is_v, (is_v ? sV : sK) + st * kStageBytes, lane);
+      dequant_subtile<BF16, false>(ks, pos0, sub, is_v, (is_v ? sV : sK) + st * kStageBytes, lane);
       fence_async_proxy();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar((is_v ? BAR_VFULL : BAR_KFULL) + st));
@@ -584,7 +652,9 @@ prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T
     // ================= MMA issue (one thread) =================
     // descriptors of stage 0, K step 0; a stage adds kStageBytes / 16 to the low word, a K step
     // (two 2 KiB slabs of 8 channels or 8 tokens) 256
-    const uint64_t qd = make_desc(smem_addr(sQ), 2048, 128), kd = make_desc(smem_addr(sK), 2048, 128), vd = make_desc(smem_addr(sV), 2048, 128);
+    const uint64_t qd = make_desc(smem_addr(sQ), 2048, 128);
+    const uint64_t kd = PRE ? make_desc_sw128(smem_addr(sK), 16, 1024) : make_desc(smem_addr(sK), 2048, 128);
+    const uint64_t vd = PRE ? make_desc_sw128(smem_addr(sV), kStageBytes / 2, 1024) : make_desc(smem_addr(sV), 2048, 128);
     const uint32_t qd_lo = static_cast<uint32_t>(qd), qd_hi = static_cast<uint32_t>(qd >> 32);
     const uint32_t kd_lo = static_cast<uint32_t>(kd), kd_hi = static_cast<uint32_t>(kd >> 32);
     const uint32_t vd_lo = static_cast<uint32_t>(vd), vd_hi = static_cast<uint32_t>(vd >> 32);
@@ -595,7 +665,8 @@ prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T
       if (lane == 0) {
         const uint32_t a_lo = qd_lo + i * (kQTileBytes >> 4), b_lo = kd_lo + st * (kStageBytes >> 4), d = tmem + 128 * i;
 #pragma unroll
-        for (int k = 0; k < 8; ++k) umma_f16_ss(d, a_lo + 256 * k, qd_hi, b_lo + 256 * k, kd_hi, kIdescS, k > 0);
+        for (int k = 0; k < 8; ++k)   // K step of the swizzled K^: 32 bytes inside the row, 16 KiB to the second half of the channels
+          umma_f16_ss(d, a_lo + 256 * k, qd_hi, b_lo + (PRE ? (k >> 2) * 1024 + (k & 3) * 2 : 256 * k), kd_hi, kIdescS, k > 0);
         umma_commit(bar(BAR_SFULL + i));
         if (i == 1) umma_commit(bar(BAR_KFREE + st));
       }
@@ -608,7 +679,8 @@ prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T
         const uint32_t lo = vd_lo + st * (kStageBytes >> 4), d = tmem + 256 + 128 * i, a = tmem + 128 * i;
         umma_f16_ta(d, a, lo, vd_hi, kIdescPV, kb > 0);
 #pragma unroll
-        for (int k = 1; k < 8; ++k) umma_f16_ta(d, a + 8 * k, lo + 256 * k, vd_hi, kIdescPV, 1u);
+        for (int k = 1; k < 8; ++k)   // K step of the swizzled V^: 16 token rows of 128 bytes
+          umma_f16_ta(d, a + 8 * k, lo + (PRE ? 128 : 256) * k, vd_hi, kIdescPV, 1u);
         if (i == 1) umma_commit(bar(BAR_VFREE + st));
         if (last) umma_commit(bar(BAR_OFULL + i));
       }
@@ -644,23 +716,73 @@ prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T
 
 }  // namespace
 
-cudaError_t launch_prefill_attn(const Dims& dm, const CacheView& cv, const void* q, int T, int layer, float scale,
-                                float* out, cudaStream_t st) {
-  if (T <= 0) return cudaSuccess;
-  const size_t smem = 2 * kQTileBytes + 2 * kStages * kStageBytes + BAR_COUNT * 8 + 16;
+// cuTensorMapEncodeTiled through the runtime's driver entry-point lookup (no link against libcuda)
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// [rows][128] fp16 rows, boxes of 64 channels x 128 rows, 128-byte swizzle
+static bool make_block_map(CUtensorMap* m, const void* base, long long rows) {
+  static EncodeTiledFn enc = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess)
+      p = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
+  if (!enc) return false;
+  const cuuint64_t gdim[2] = {kHeadDim, static_cast<cuuint64_t>(rows)};
+  const cuuint64_t gstride[1] = {kHeadDim * 2};
+  const cuuint32_t box[2] = {64, kKvBlock};
+  const cuuint32_t estr[2] = {1, 1};
+  return enc(m, CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, const_cast<void*>(base), gdim, gstride, box, estr,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+static int padded_tokens(int T) { return (T + kKvBlock - 1) / kKvBlock * kKvBlock; }
+
+long long prefill_workspace_bytes(const Dims& dm, int T) {
+  return 2ll * dm.batch * dm.n_kv_heads * padded_tokens(T) * kHeadDim * 2;
+}
+
+template <bool BF16, bool PRE>
+static cudaError_t launch_attn(const Dims& dm, const CacheView& cv, const void* q, int T, int layer, float scale, float* out,
+                               const CUtensorMap& mk, const CUtensorMap& mv, int t_pad, cudaStream_t st) {
+  const size_t smem = 1024 + 2 * kQTileBytes + 2 * kStages * kStageBytes + BAR_COUNT * 8 + 16;
   dim3 grid((T + 2 * kQTile - 1) / (2 * kQTile), dm.n_q_heads, dm.batch);
-  const float scale_log2 = scale * 1.4426950408889634f;
-  cudaError_t e;
-  if (dm.dtype == MOQAE_DTYPE_BF16) {
-    e = cudaFuncSetAttribute(prefill_attn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-    if (e != cudaSuccess) return e;
-    prefill_attn_kernel<true><<<grid, kP2Threads, smem, st>>>(dm, cv, static_cast<const uint16_t*>(q), T, layer, scale_log2, out);
-  } else {
-    e = cudaFuncSetAttribute(prefill_attn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-    if (e != cudaSuccess) return e;
-    prefill_attn_kernel<false><<<grid, kP2Threads, smem, st>>>(dm, cv, static_cast<const uint16_t*>(q), T, layer, scale_log2, out);
-  }
+  cudaError_t e = cudaFuncSetAttribute(prefill_attn_kernel<BF16, PRE>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  if (e != cudaSuccess) return e;
+  prefill_attn_kernel<BF16, PRE><<<grid, kP2Threads, smem, st>>>(dm, cv, static_cast<const uint16_t*>(q), T, layer,
+                                                                 scale * 1.4426950408889634f, out, mk, mv, t_pad);
   return cudaGetLastError();
+}
+
+// workspace == nullptr: every CTA expands the packed tiles itself (no extra memory).  Otherwise the
+// layer is expanded once into the workspace (prefill_workspace_bytes) and fetched from there.
+cudaError_t launch_prefill_attn(const Dims& dm, const CacheView& cv, const void* q, int T, int layer, float scale,
+                                float* out, void* workspace, cudaStream_t st) {
+  if (T <= 0) return cudaSuccess;
+  const bool bf16 = dm.dtype == MOQAE_DTYPE_BF16;
+  CUtensorMap mk, mv;
+  memset(&mk, 0, sizeof(mk));
+  memset(&mv, 0, sizeof(mv));
+  if (!workspace)
+    return bf16 ? launch_attn<true, false>(dm, cv, q, T, layer, scale, out, mk, mv, 0, st)
+                : launch_attn<false, false>(dm, cv, q, T, layer, scale, out, mk, mv, 0, st);
+  const int t_pad = padded_tokens(T);
+  uint8_t* kd = static_cast<uint8_t*>(workspace);
+  uint8_t* vd = kd + prefill_workspace_bytes(dm, T) / 2;
+  const long long rows = static_cast<long long>(dm.batch) * dm.n_kv_heads * t_pad;
+  if (!make_block_map(&mk, kd, rows) || !make_block_map(&mv, vd, rows)) return cudaErrorNotSupported;
+  dim3 dgrid(t_pad / kTileTokens, dm.n_kv_heads, dm.batch);
+  if (bf16) prefill_dequant_kernel<true><<<dgrid, 64, 0, st>>>(dm, cv, layer, t_pad, kd, vd);
+  else prefill_dequant_kernel<false><<<dgrid, 64, 0, st>>>(dm, cv, layer, t_pad, kd, vd);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  return bf16 ? launch_attn<true, true>(dm, cv, q, T, layer, scale, out, mk, mv, t_pad, st)
+              : launch_attn<false, true>(dm, cv, q, T, layer, scale, out, mk, mv, t_pad, st);
 }
 
 }  // namespace moqae

@@ -27,15 +27,19 @@ def prefill_case(B, T, Hq, Hkv, chunk, dtype, bmap, seed):
     cache = mq.moqae_cache_bind(cfg, cap, zero_pools=True)
     fm = torch.from_numpy(bmap).cuda() if bmap.size else None
     mq.moqae_quantize_kv(cfg, K.cuda(), V.cuda(), T, 1, cache, forced_map=fm)
-    out = torch.full((B, T, Hq, 128), float("nan"), dtype=torch.float32, device="cuda")
-    mq.moqae_prefill_attn(cfg, q.cuda(), T, 1, cache, out)
-    torch.cuda.synchronize()
-    assert mq.moqae_poll_status(cache) == 0
-    got = out.cpu().numpy().astype(np.float64)
-    assert np.isfinite(got).all()
     abs_tol = 3 * 2.0 ** -11 * float(V.float().abs().max())
-    ok, e_abs, e_rel = H.attn_tolerance_ok(got.reshape(1, -1, 128), ref.reshape(1, -1, 128), abs_tol=abs_tol, rel_tol=1e-2)
-    assert ok, (e_abs, e_rel)
+    # both ways of feeding the products: every CTA expanding the packed tiles itself (no
+    # workspace), and the layer expanded once into an fp16 workspace that the CTAs fetch from
+    ws = torch.full((mq.moqae_prefill_attn_workspace(cfg, T),), 0xFF, dtype=torch.uint8, device="cuda")
+    for workspace in (None, ws):
+        out = torch.full((B, T, Hq, 128), float("nan"), dtype=torch.float32, device="cuda")
+        mq.moqae_prefill_attn(cfg, q.cuda(), T, 1, cache, out, workspace=workspace)
+        torch.cuda.synchronize()
+        assert mq.moqae_poll_status(cache) == 0
+        got = out.cpu().numpy().astype(np.float64)
+        assert np.isfinite(got).all()
+        ok, e_abs, e_rel = H.attn_tolerance_ok(got.reshape(1, -1, 128), ref.reshape(1, -1, 128), abs_tol=abs_tol, rel_tol=1e-2)
+        assert ok, (workspace is not None, e_abs, e_rel)
     return e_abs, e_rel
 
 
@@ -56,3 +60,15 @@ def test_short_prompts():
     prefill_case(1, 7, 2, 1, 32, 0, np.zeros((1, 0), np.uint8), 720)          # tail only
     prefill_case(1, 128, 1, 1, 128, 1, np.array([[1]], np.uint8), 721)        # exactly one block
     prefill_case(2, 129, 2, 2, 64, 1, np.array([[3, 0], [2, 1]], np.uint8), 722)
+
+
+def test_workspace_size_and_rejection():
+    cfg = mq.make_config(n_layers=1, n_q_heads=4, n_kv_heads=2, chunk=64, dtype=1, d_in=64, max_tokens=300, batch=3)
+    assert mq.moqae_prefill_attn_workspace(cfg, 300) == 2 * 3 * 2 * 384 * 256      # 300 tokens -> 3 blocks of 128
+    assert mq.moqae_prefill_attn_workspace(cfg, 0) == 0
+    cache = mq.moqae_cache_bind(cfg, [1, 1, 1, 1], zero_pools=True)
+    q = torch.zeros(3, 300, 4, 128, dtype=torch.bfloat16, device="cuda")
+    out = torch.zeros(3, 300, 4, 128, dtype=torch.float32, device="cuda")
+    small = torch.zeros(1024, dtype=torch.uint8, device="cuda")
+    with pytest.raises(RuntimeError):
+        mq.moqae_prefill_attn(cfg, q, 300, 0, cache, out, workspace=small)
