@@ -15,6 +15,7 @@ from __future__ import annotations
 
 import argparse
 import dataclasses
+import datetime
 import json
 import os
 import subprocess
@@ -48,8 +49,10 @@ def read_peaks():
 
 
 class ClockSampler:
-    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
-    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+    """nvidia-smi clock / throttle-reason samples taken while the timed region runs.  The tool
+    needs a few hundred ms to produce its first line, so it is started before the warm-up and only
+    the samples whose time stamps fall between begin() and end() are used."""
+    Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
          "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
@@ -57,6 +60,13 @@ class ClockSampler:
         self.gpu = gpu_index
         self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
         self.p = None
+        self.t_begin = self.t_end = None
+
+    def begin(self):
+        self.t_begin = datetime.datetime.now()
+
+    def end(self):
+        self.t_end = datetime.datetime.now()
 
     def start(self):
         try:
@@ -84,6 +94,9 @@ class ClockSampler:
             if len(parts) < 9:
                 continue
             try:
+                when = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f")
+                if self.t_begin and self.t_end and not (self.t_begin <= when <= self.t_end):
+                    continue
                 sm.append(float(parts[1]))
                 mx.append(float(parts[2]))
             except ValueError:
@@ -96,8 +109,7 @@ class ClockSampler:
         except OSError:
             pass
         if sm:
-            busy = sorted(sm)[len(sm) // 2:]          # upper half: samples taken under load
-            out = {"sm_mhz": float(np.median(busy)), "sm_max_mhz": float(max(mx)),
+            out = {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)),
                    "reasons": sorted(reasons), "samples": len(sm)}
         return out
 
@@ -305,6 +317,8 @@ def run_ours(args):
         if ev:
             ev[3].record()
 
+    sampler = ClockSampler(local)
+    sampler.start()
     for _ in range(args.warmup):
         one_step()
     torch.cuda.synchronize()
@@ -313,12 +327,11 @@ def run_ours(args):
         raise RuntimeError(f"device status {status} after warm-up")
     b_route, b_quant, b_dec = job.bytes_per_step()
 
-    sampler = ClockSampler(local)
     events = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
-    sampler.start()
+    sampler.begin()
     t0 = torch.cuda.Event(enable_timing=True)
     t1 = torch.cuda.Event(enable_timing=True)
     t0.record()
@@ -326,6 +339,7 @@ def run_ours(args):
         one_step(events[s])
     t1.record()
     torch.cuda.synchronize()
+    sampler.end()
     if world > 1:
         dist.barrier()
     clocks = sampler.stop()
