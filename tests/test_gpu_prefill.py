@@ -56,6 +56,14 @@ def test_mixed_map_gqa_ragged(dtype):
     prefill_case(B, T, 4, 2, chunk, dtype, bmap, 710 + dtype)
 
 
+def test_longer_prompt_many_blocks_wide_gqa():
+    # 9 blocks of 128 tokens (every operand stage is reused several times, five CTAs per head of
+    # different lengths), 8 query heads on 2 kv heads, chunk 128, a tail of 77 tokens
+    B, T, chunk = 1, 128 * 8 + 77, 128
+    bmap = np.random.RandomState(9).randint(0, 4, size=(B, T // chunk)).astype(np.uint8)
+    prefill_case(B, T, 8, 2, chunk, 1, bmap, 730)
+
+
 def test_short_prompts():
     prefill_case(1, 7, 2, 1, 32, 0, np.zeros((1, 0), np.uint8), 720)          # tail only
     prefill_case(1, 128, 1, 1, 128, 1, np.array([[1]], np.uint8), 721)        # exactly one block
