@@ -318,7 +318,7 @@ __device__ __forceinline__ void copy_rows(const uint8_t* __restrict__ src, uint8
 constexpr int kSoftmaxWarps = 8, kDequantWarps = 8;   // dequant: 4 warps for keys, 4 for values
 constexpr int kP2Threads = (kSoftmaxWarps + kDequantWarps + 1) * 32;
 constexpr int kTmemCols2 = 512;
-constexpr float kRescaleSlack = 8.0f;          // base-2 units: weights stay below 2^8
+constexpr float kSumLimit = 16384.0f;          // a chunk whose weights sum to less cannot overflow fp16 (65504)
 constexpr int kStages = 2;
 constexpr int kStageBytes = kKvBlock * 128 * 2;  // one K^ / V^ stage
 constexpr int kQTileBytes = kQTile * 128 * 2;
@@ -546,15 +546,32 @@ prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T
           for (int e = 0; e < 32; ++e)
             if (32 * c4 + e > rel) v[e] = -INFINITY;
         }
-        float mx = v[0];
+        // Weights against the current reference, with no look at the scores' maximum first: as
+        // long as the chunk's sum stays below kSumLimit no weight can overflow fp16, and the
+        // reference may lag the true maximum.
+        uint32_t pk[16];
+        float csum;
+        auto weights = [&]() {
+          float part[2] = {0.0f, 0.0f};
 #pragma unroll
-        for (int e = 1; e < 32; ++e) mx = fmaxf(mx, v[e]);
-        mx *= scale_log2;                            // scale_log2 > 0
-        if (__any_sync(0xffffffffu, mx > m_ref + kRescaleSlack)) {
-          // Rare: some row of the warp found a score far above its reference.  Move the reference
+          for (int e2 = 0; e2 < 16; ++e2) {
+            const float p0 = ex2_approx(fmaf(v[2 * e2], scale_log2, -m_ref)), p1 = ex2_approx(fmaf(v[2 * e2 + 1], scale_log2, -m_ref));
+            part[e2 & 1] += p0 + p1;
+            pk[e2] = pack_h2(p0, p1);
+          }
+          csum = part[0] + part[1];
+        };
+        weights();
+        if (__any_sync(0xffffffffu, !(csum < kSumLimit))) {
+          // Rare (always on the very first chunk, where the reference is still -inf): some row of
+          // the warp met scores far above its reference.  Move the reference to the chunk's maximum
           // and rescale what was accumulated against the old one: O_i (at rest: S_i of this block
           // was issued after the last O_i += P_i V^), the running sums, and the chunks of P_i already
-          // written for this block.
+          // written for this block; then form this chunk's weights again.
+          float mx = v[0];
+#pragma unroll
+          for (int e = 1; e < 32; ++e) mx = fmaxf(mx, v[e]);
+          mx *= scale_log2;                          // scale_log2 > 0
           const float m_new = fmaxf(m_ref, ceilf(mx));
           const float corr = (m_ref == -INFINITY) ? 0.0f : ex2_approx(m_ref - m_new);
           if (kb > 0) {
@@ -582,14 +599,9 @@ prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T
           l *= corr;
           sum *= corr;
           m_ref = m_new;
+          weights();
         }
-        uint32_t pk[16];
-#pragma unroll
-        for (int e2 = 0; e2 < 16; ++e2) {
-          const float p0 = ex2_approx(fmaf(v[2 * e2], scale_log2, -m_ref)), p1 = ex2_approx(fmaf(v[2 * e2 + 1], scale_log2, -m_ref));
-          sum += p0 + p1;
-          pk[e2] = pack_h2(p0, p1);
-        }
+        sum += csum;
         tmem_st16u_nowait(s_addr + 16 * c4, pk);     // columns already read: 16 (c4 + 1) <= 32 (c4 + 1)
       }
       l += sum;
