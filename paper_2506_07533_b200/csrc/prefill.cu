@@ -139,6 +139,25 @@ __device__ __forceinline__ float ex2_approx(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(r) : "f"(x));
   return r;
 }
+// packed fp32 pairs: one instruction for two lanes of arithmetic
+__device__ __forceinline__ uint64_t pack_f2(float a, float b) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};\n" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ void unpack_f2(uint64_t v, float& a, float& b) {
+  asm("mov.b64 {%0, %1}, %2;\n" : "=f"(a), "=f"(b) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma_f2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;\n" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add_f2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;\n" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
 
 // ---- dequantisation of one 32-token storage tile into the operand tiles --------------------
 // The packed layout is the one the decode kernel's lanes consume (lane = 4g + t4); the same
@@ -552,14 +571,19 @@ prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T
         uint32_t pk[16];
         float csum;
         auto weights = [&]() {
-          float part[2] = {0.0f, 0.0f};
+          const uint64_t scale2 = pack_f2(scale_log2, scale_log2), negm2 = pack_f2(-m_ref, -m_ref);
+          uint64_t part[2] = {0ull, 0ull};           // two packed partial sums (even / odd columns each)
 #pragma unroll
           for (int e2 = 0; e2 < 16; ++e2) {
-            const float p0 = ex2_approx(fmaf(v[2 * e2], scale_log2, -m_ref)), p1 = ex2_approx(fmaf(v[2 * e2 + 1], scale_log2, -m_ref));
-            part[e2 & 1] += p0 + p1;
+            float x0, x1;
+            unpack_f2(fma_f2(pack_f2(v[2 * e2], v[2 * e2 + 1]), scale2, negm2), x0, x1);
+            const float p0 = ex2_approx(x0), p1 = ex2_approx(x1);
+            part[e2 & 1] = add_f2(part[e2 & 1], pack_f2(p0, p1));
             pk[e2] = pack_h2(p0, p1);
           }
-          csum = part[0] + part[1];
+          float s0, s1;
+          unpack_f2(add_f2(part[0], part[1]), s0, s1);
+          csum = s0 + s1;
         };
         weights();
         if (__any_sync(0xffffffffu, !(csum < kSumLimit))) {
