@@ -24,7 +24,7 @@ namespace {
 constexpr int kQWarps = 4;
 constexpr int kInBytes = 8192;                 // 32 rows x 256 B
 constexpr int kOutBytes = 9216;                // largest quantised tile
-constexpr int kPrmBytes = 1024;                // value groups: [32 tokens][4 groups] (zero, 1/scale)
+constexpr int kPrmBytes = 2048;                // value groups: [32 tokens][4 groups] (-zero, -zero, 1/scale, 1/scale)
 constexpr int kWarpSmem = 2 * kInBytes + kOutBytes + kPrmBytes;
 constexpr long long kWaitCycles = 1ll << 30;  // a bounded wait gives up after this many SM cycles
 constexpr uint32_t kSuspendNs = 20000;         // how long one try_wait may keep the warp parked
@@ -113,9 +113,23 @@ __device__ __forceinline__ void group_params(float mn, float mx, float qmax, uin
   z_bits = zb;
 }
 
-// code + 0x4B400000: the low bits of the result hold rint((x - zf) * inv)
-__device__ __forceinline__ uint32_t encode(float x, float zf, float inv) {
-  return __float_as_uint(__fmaf_rn(__fsub_rn(x, zf), inv, kMagic));
+// code + 0x4B400000 = fma(x - z, inv, 1.5 * 2^23): the low bits of the result hold
+// rint((x - z) * inv).  Done for the two 16-bit values of one word at once, as packed fp32 pairs
+// (add.rn.f32x2 and fma.rn.f32x2 round each lane exactly like the scalar instructions; x + (-z)
+// is x - z).
+// negz2 = (-z_lo, -z_hi), inv2 = (inv_lo, inv_hi) as 64-bit register pairs.
+__device__ __forceinline__ uint64_t pack_f2(float a, float b) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};\n" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
+template <bool BF16>
+__device__ __forceinline__ void encode2(uint32_t w, uint64_t negz2, uint64_t inv2, uint32_t& u_lo, uint32_t& u_hi) {
+  const uint64_t x2 = pack_f2(lo_f<BF16>(w), hi_f<BF16>(w));
+  uint64_t d2, r2;
+  asm("add.rn.f32x2 %0, %1, %2;\n" : "=l"(d2) : "l"(x2), "l"(negz2));
+  asm("fma.rn.f32x2 %0, %1, %2, %3;\n" : "=l"(r2) : "l"(d2), "l"(inv2), "l"(pack_f2(kMagic, kMagic)));
+  asm("mov.b64 {%0, %1}, %2;\n" : "=r"(u_lo), "=r"(u_hi) : "l"(r2));
 }
 
 // Four codes of `BITS` bits side by side in the low 4*BITS bits (higher bits: don't care for
@@ -169,12 +183,16 @@ __device__ __forceinline__ void encode_keys(const uint8_t* __restrict__ in, uint
   }
   // payload: this lane's 4 codes of token t are 4*BITS contiguous bits of the (t, quarter) piece
   uint8_t* pay = out + kMetaBytes;
+  const uint64_t negz01 = pack_f2(-zf[0], -zf[1]), negz23 = pack_f2(-zf[2], -zf[3]);
+  const uint64_t inv01 = pack_f2(inv[0], inv[1]), inv23 = pack_f2(inv[2], inv[3]);
   const int q = lane >> 3, l7 = lane & 7;
 #pragma unroll
   for (int t = 0; t < kTileTokens; ++t) {
     const uint2 w = rows[32 * t];
-    const uint32_t p = pack4<BITS>(encode(lo_f<BF16>(w.x), zf[0], inv[0]), encode(hi_f<BF16>(w.x), zf[1], inv[1]),
-                                   encode(lo_f<BF16>(w.y), zf[2], inv[2]), encode(hi_f<BF16>(w.y), zf[3], inv[3]));
+    uint32_t u0, u1, u2, u3;
+    encode2<BF16>(w.x, negz01, inv01, u0, u1);
+    encode2<BF16>(w.y, negz23, inv23, u2, u3);
+    const uint32_t p = pack4<BITS>(u0, u1, u2, u3);
     const int blk = t >> 4, hh = (t >> 3) & 1, g = t & 7;
     if (BITS == 2) {
       pay[(32 * blk + 4 * g + q) * 16 + 8 * hh + l7] = static_cast<uint8_t>(p);
@@ -189,7 +207,7 @@ __device__ __forceinline__ void encode_keys(const uint8_t* __restrict__ in, uint
 // ---- values: groups are 32 channels of one token -----------------------------------------
 template <int BITS, bool BF16>
 __device__ __forceinline__ void encode_values(const uint8_t* __restrict__ in, uint8_t* __restrict__ out,
-                                              float2* __restrict__ prm, int lane) {
+                                              float4* __restrict__ prm, int lane) {
   constexpr float qmax = static_cast<float>((1 << BITS) - 1);
   uint16_t* meta = reinterpret_cast<uint16_t*>(out);
   {
@@ -198,8 +216,6 @@ __device__ __forceinline__ void encode_values(const uint8_t* __restrict__ in, ui
     const int t = lane;
     const uint4* row = reinterpret_cast<const uint4*>(in + t * 256);
     const int blk = t >> 4, half = (t >> 3) & 1, t4 = (t >> 1) & 3, e = t & 1;
-    float4 pz[2];
-    float* pzf = reinterpret_cast<float*>(pz);
 #pragma unroll
     for (int cg = 0; cg < 4; ++cg) {
       uint32_t mn = 0, mx = 0;
@@ -214,13 +230,10 @@ __device__ __forceinline__ void encode_values(const uint8_t* __restrict__ in, ui
       float zf, inv;
       uint16_t sb, zb;
       group_params(fminf(lo_f<BF16>(mn), hi_f<BF16>(mn)), fmaxf(lo_f<BF16>(mx), hi_f<BF16>(mx)), qmax, sb, zb, zf, inv);
-      pzf[2 * cg] = zf;
-      pzf[2 * cg + 1] = inv;
+      prm[4 * t + cg] = make_float4(-zf, -zf, inv, inv);
       meta[256 + ((((blk * 2 + (cg >> 1)) * 4 + t4) * 4 + (cg & 1) * 2 + half) * 2) + e] = sb;
       meta[384 + ((((blk * 4 + cg) * 4 + t4) * 2 + half) * 2) + e] = zb;
     }
-    reinterpret_cast<float4*>(prm)[2 * t] = pz[0];
-    reinterpret_cast<float4*>(prm)[2 * t + 1] = pz[1];
   }
   __syncwarp();
   // codes: lane = channels 4*lane .. 4*lane+3 (group p = lane / 8); one word set per 4 tokens
@@ -236,11 +249,9 @@ __device__ __forceinline__ void encode_values(const uint8_t* __restrict__ in, ui
       for (int bp = 0; bp < 4; ++bp) {
         const int t = 16 * blk + 8 * (bp & 1) + 2 * t4 + (bp >> 1);
         const uint2 w = rows[32 * t];
-        const float2 zi = prm[4 * t + p];
-        u[bp][0] = encode(lo_f<BF16>(w.x), zi.x, zi.y);
-        u[bp][1] = encode(hi_f<BF16>(w.x), zi.x, zi.y);
-        u[bp][2] = encode(lo_f<BF16>(w.y), zi.x, zi.y);
-        u[bp][3] = encode(hi_f<BF16>(w.y), zi.x, zi.y);
+        const ulonglong2 zi = *reinterpret_cast<const ulonglong2*>(prm + 4 * t + p);    // (-z, -z), (inv, inv)
+        encode2<BF16>(w.x, zi.x, zi.y, u[bp][0], u[bp][1]);
+        encode2<BF16>(w.y, zi.x, zi.y, u[bp][2], u[bp][3]);
       }
       const int ln = 4 * g + t4;
       if (BITS == 2) {
@@ -298,7 +309,7 @@ quantize_pack_kernel(Dims dm, CacheView cv, const __grid_constant__ CUtensorMap 
   uint8_t* bufK = smem + warp * kWarpSmem;
   uint8_t* bufV = bufK + kInBytes;
   uint8_t* out = bufV + kInBytes;
-  float2* prm = reinterpret_cast<float2*>(out + kOutBytes);
+  float4* prm = reinterpret_cast<float4*>(out + kOutBytes);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kQWarps * kWarpSmem) + 2 * warp;
   const uint32_t barK = smem_u32(bars), barV = smem_u32(bars + 1);
   if (lane == 0) {
