@@ -335,7 +335,11 @@ __device__ __forceinline__ void copy_rows(const uint8_t* __restrict__ src, uint8
 // tells the softmax threads that O_i is at rest (they rescale it in place when the reference
 // maximum moves).
 constexpr int kSoftmaxWarps = 8, kDequantWarps = 8;   // dequant: 4 warps for keys, 4 for values
-constexpr int kP2Threads = (kSoftmaxWarps + kDequantWarps + 1) * 32;
+// Without a workspace: 8 softmax + 8 dequantise + 1 issue warp.  With one: 16 softmax warps (two
+// per 32 rows, each taking half of a block's columns), the issue warp and two fetch warps.
+__host__ __device__ constexpr int block_threads(bool pre) { return (kSoftmaxWarps + kDequantWarps + (pre ? 3 : 1)) * 32; }
+constexpr int kIssueWarp = kSoftmaxWarps + kDequantWarps;
+constexpr int kExchangeBytes = 256 * 2 * 4 + 2 * 8 * 2 * 4;   // per row and half: one float; per block parity, pair, half: one flag
 constexpr int kTmemCols2 = 512;
 constexpr float kSumLimit = 16384.0f;          // a chunk whose weights sum to less cannot overflow fp16 (65504)
 constexpr int kStages = 2;
@@ -472,7 +476,7 @@ __device__ __forceinline__ uint64_t make_desc_sw128(uint32_t saddr, uint32_t lbo
 }
 
 template <bool BF16, bool PRE>
-__global__ void __launch_bounds__(kP2Threads, 1)
+__global__ void __launch_bounds__(block_threads(PRE), 1)
 prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T, int layer, float scale_log2,
                     float* __restrict__ out, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                     int t_pad) {
@@ -484,6 +488,8 @@ prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T
   uint64_t* bar_mem = reinterpret_cast<uint64_t*>(sV + kStages * kStageBytes);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_mem + BAR_COUNT);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  float* exch = reinterpret_cast<float*>(bar_mem + BAR_COUNT + 2);      // [256 rows][2 halves]
+  volatile int* pair_flag = reinterpret_cast<volatile int*>(exch + 512);  // [2 block parities][8 pairs][2 halves]
   const uint32_t bar0 = smem_addr(bar_mem);
   auto bar = [&](int i) { return bar0 + 8u * i; };
 
@@ -496,21 +502,21 @@ prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T
   const int nb_all = (T + kKvBlock - 1) / kKvBlock;
   const int nb0 = min(2 * pair + 1, nb_all), nb1 = min(2 * pair + 2, nb_all);
 
-  if (warp == kSoftmaxWarps + kDequantWarps) {
+  if (warp == kIssueWarp) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_addr(tmem_slot)), "r"(kTmemCols2) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
   }
   if (tid == 0) {
     for (int i = 0; i < BAR_COUNT; ++i) {
       // kfull / vfull: four dequantising warps, or the one thread that starts the TMA copies
-      const int count = i < BAR_KFREE ? (PRE ? 1 : 4) : ((i >= BAR_PFULL && i < BAR_OFULL) ? 4 : 1);
+      const int count = i < BAR_KFREE ? (PRE ? 1 : 4) : ((i >= BAR_PFULL && i < BAR_OFULL) ? (PRE ? 8 : 4) : 1);
       asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar(i)), "r"(count) : "memory");
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
   }
   // the CTA's 2 x 128 query rows as A operands (rows past the prompt are zero)
-  for (int i = tid; i < 2 * kQTile * 16; i += kP2Threads) {
+  for (int i = tid; i < 2 * kQTile * 16; i += block_threads(PRE)) {
     const int row = i >> 4, U = i & 15;             // row 0..255
     const int pos = 2 * pair * kQTile + row;
     uint4 v = make_uint4(0u, 0u, 0u, 0u);
@@ -536,7 +542,128 @@ prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T
     return false;
   };
 
-  if (warp < kSoftmaxWarps) {
+  if (PRE && warp < kIssueWarp) {
+    // ================= softmax, two threads per query row =================
+    // Warps w and w + 8 share the 32 rows (tensor-memory lanes) of tile i = (w & 7) >> 2: the first
+    // takes columns 0..63 of every block, the second columns 64..127.  Both keep the same
+    // reference maximum; they meet once per block on a named barrier of their 64 threads, which
+    // also orders "every score has been read" before "P overwrites the first half of S".
+    const int half = warp >> 3;                     // which 64 columns
+    const int i = (warp & 7) >> 2;                  // query tile
+    const int nb = i ? nb1 : nb0;
+    const int row = 128 * i + 32 * (warp & 3) + lane;           // 0..255 in the CTA
+    const int qpos = 2 * pair * kQTile + row;
+    const int pair_id = warp & 7;                   // the two warps of these rows
+    const uint32_t lane_addr = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+    const uint32_t s_addr = lane_addr + 128 * i + 64 * half;     // this thread's 64 score columns
+    const uint32_t p_addr = lane_addr + 128 * i + 32 * half;     // where its 32 packed columns of P go
+    const uint32_t o_addr = lane_addr + 256 + 128 * i + 64 * half;   // the half of O it rescales and writes out
+    auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;\n" ::"r"(1 + pair_id) : "memory"); };
+    float m_ref = -INFINITY, l = 0.0f;
+    bool ok = true;
+    for (int kb = 0; kb < nb && ok; ++kb) {
+      ok = __all_sync(0xffffffffu, wait(BAR_SFULL + i, kb));
+      // a warp whose wait ran out still meets its partner on the pair barrier (which has no time
+      // limit of its own) and tells it, so that both leave the loop after the same block
+      if (ok) tc_fence_after();
+      const bool diag = kb >= 2 * pair + i;
+      const int rel = qpos - kb * kKvBlock - 64 * half;          // local columns 0..rel are visible
+      uint32_t pk[32];
+      float csum = 0.0f;
+      // weights of this thread's 64 columns against m_ref; with want_max also their largest score
+      auto weights = [&](bool want_max, float& mx) {
+        csum = 0.0f;
+        mx = -INFINITY;
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          float v[32];
+          tmem_ld32(v, s_addr + 32 * c);
+          if (diag) {
+#pragma unroll
+            for (int e = 0; e < 32; ++e)
+              if (32 * c + e > rel) v[e] = -INFINITY;
+          }
+          if (want_max) {
+#pragma unroll
+            for (int e = 0; e < 32; ++e) mx = fmaxf(mx, v[e]);
+          }
+          const uint64_t scale2 = pack_f2(scale_log2, scale_log2), negm2 = pack_f2(-m_ref, -m_ref);
+          uint64_t part[2] = {0ull, 0ull};
+#pragma unroll
+          for (int e2 = 0; e2 < 16; ++e2) {
+            float x0, x1;
+            unpack_f2(fma_f2(pack_f2(v[2 * e2], v[2 * e2 + 1]), scale2, negm2), x0, x1);
+            const float p0 = ex2_approx(x0), p1 = ex2_approx(x1);
+            part[e2 & 1] = add_f2(part[e2 & 1], pack_f2(p0, p1));
+            pk[16 * c + e2] = pack_h2(p0, p1);
+          }
+          float s0, s1;
+          unpack_f2(add_f2(part[0], part[1]), s0, s1);
+          csum += s0 + s1;
+        }
+      };
+      float mx;
+      if (ok) weights(false, mx);
+      const bool over = ok && __any_sync(0xffffffffu, !(csum < kSumLimit));
+      if (lane == 0) pair_flag[((kb & 1) * 8 + pair_id) * 2 + half] = (over ? 1 : 0) | (ok ? 0 : 2);
+      pair_sync();                                   // both halves of S have been read; flags are visible
+      const int flags = pair_flag[((kb & 1) * 8 + pair_id) * 2] | pair_flag[((kb & 1) * 8 + pair_id) * 2 + 1];
+      if (flags & 2) {
+        ok = false;
+        break;
+      }
+      if (flags & 1) {
+        // Rare (always on the first block): move the reference to the row's largest score of this
+        // block and rescale what was accumulated against the old one.  O_i is at rest: S_i of this
+        // block was issued after the last O_i += P_i V^.
+        weights(true, mx);
+        exch[row * 2 + half] = mx * scale_log2;      // scale_log2 > 0
+        pair_sync();
+        const float m_new = fmaxf(m_ref, ceilf(fmaxf(exch[row * 2], exch[row * 2 + 1])));
+        const float corr = (m_ref == -INFINITY) ? 0.0f : ex2_approx(m_ref - m_new);
+        if (kb > 0) {
+#pragma unroll 1
+          for (int o4 = 0; o4 < 2; ++o4) {
+            float o[32];
+            tmem_ld32(o, o_addr + 32 * o4);
+#pragma unroll
+            for (int e = 0; e < 32; ++e) o[e] *= corr;
+            tmem_st32(o_addr + 32 * o4, o);
+          }
+        }
+        l *= corr;
+        m_ref = m_new;
+        weights(false, mx);
+        pair_sync();                                 // the partner has read its scores again, too
+      }
+      l += csum;
+      tmem_st32u(p_addr, pk);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(BAR_PFULL + i));
+    }
+    if (ok && nb > 0) ok = __all_sync(0xffffffffu, wait(BAR_OFULL + i, 0));
+    // the row's sum is the two halves' sums
+    exch[row * 2 + half] = l;
+    pair_sync();
+    if (ok) {
+      tc_fence_after();
+      const float lt = exch[row * 2] + exch[row * 2 + 1];
+      const float inv = lt > 0.0f ? 1.0f / lt : 0.0f;
+#pragma unroll 1
+      for (int c4 = 0; c4 < 2; ++c4) {
+        float v[32];
+        tmem_ld32(v, o_addr + 32 * c4);
+        if (qpos < T) {
+          float4* dst = reinterpret_cast<float4*>(out + ((static_cast<long long>(b) * T + qpos) * Hq + hq) * kHeadDim + 64 * half + 32 * c4);
+#pragma unroll
+          for (int e = 0; e < 32; e += 4) dst[e >> 2] = make_float4(v[e] * inv, v[e + 1] * inv, v[e + 2] * inv, v[e + 3] * inv);
+        }
+      }
+    } else if (lane == 0) {
+      set_status(cv.status, MOQAE_ERR_TIMEOUT, blockIdx.x, warp);
+    }
+  } else if (warp < kSoftmaxWarps) {
     // ================= softmax: one query row per thread =================
     const int i = warp >> 2;                        // query tile of this warp
     const int nb = i ? nb1 : nb0;
@@ -651,11 +778,10 @@ prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T
     } else if (lane == 0) {
       set_status(cv.status, MOQAE_ERR_TIMEOUT, blockIdx.x, warp);
     }
-  } else if (PRE && warp < kSoftmaxWarps + kDequantWarps) {
-    // ================= fetch: K^ (warp 8) and V^ (warp 12) blocks from the fp16 scratch by TMA =================
-    const int dw = warp - kSoftmaxWarps;
-    if ((dw == 0 || dw == 4) && lane == 0) {
-      const bool is_v = dw == 4;
+  } else if (PRE && warp > kIssueWarp) {
+    // ================= fetch: K^ (warp 17) and V^ (warp 18) blocks from the fp16 scratch by TMA =================
+    if (lane == 0) {
+      const bool is_v = warp == kIssueWarp + 2;
       const CUtensorMap* map = is_v ? &map_v : &map_k;
       const int row0 = (b * H + h) * t_pad;
       for (int kb = 0; kb < nb1; ++kb) {
@@ -668,7 +794,7 @@ prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T
         tma_load_2d(dst + kStageBytes / 2, map, 64, row0 + kb * kKvBlock, full);  // channels 64..127
       }
     }
-  } else if (warp < kSoftmaxWarps + kDequantWarps) {
+  } else if (warp < kIssueWarp) {
     // ================= dequantise: storage tile `sub` of every block =================
     const int dw = warp - kSoftmaxWarps;
     const bool is_v = dw >= 4;
@@ -746,7 +872,7 @@ prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == kSoftmaxWarps + kDequantWarps)
+  if (warp == kIssueWarp)
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(kTmemCols2) : "memory");
 }
 
@@ -786,11 +912,11 @@ long long prefill_workspace_bytes(const Dims& dm, int T) {
 template <bool BF16, bool PRE>
 static cudaError_t launch_attn(const Dims& dm, const CacheView& cv, const void* q, int T, int layer, float scale, float* out,
                                const CUtensorMap& mk, const CUtensorMap& mv, int t_pad, cudaStream_t st) {
-  const size_t smem = 1024 + 2 * kQTileBytes + 2 * kStages * kStageBytes + BAR_COUNT * 8 + 16;
+  const size_t smem = 1024 + 2 * kQTileBytes + 2 * kStages * kStageBytes + BAR_COUNT * 8 + 16 + kExchangeBytes;
   dim3 grid((T + 2 * kQTile - 1) / (2 * kQTile), dm.n_q_heads, dm.batch);
   cudaError_t e = cudaFuncSetAttribute(prefill_attn_kernel<BF16, PRE>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) return e;
-  prefill_attn_kernel<BF16, PRE><<<grid, kP2Threads, smem, st>>>(dm, cv, static_cast<const uint16_t*>(q), T, layer,
+  prefill_attn_kernel<BF16, PRE><<<grid, block_threads(PRE), smem, st>>>(dm, cv, static_cast<const uint16_t*>(q), T, layer,
                                                                  scale * 1.4426950408889634f, out, mk, mv, t_pad);
   return cudaGetLastError();
 }
