@@ -5,19 +5,21 @@
 // A dense contraction, so it runs on the 5th-generation tensor cores: one CTA owns 256
 // consecutive query positions (two tiles of 128) of one query head and walks the cache in
 // blocks of 128 tokens (four storage tiles, in token order through the chunk map).  Per block
-//   dequantise   four warps turn the four packed tiles into fp16 K^ [128 tokens x 128 ch]
-//                (K-major) and V^ [128 x 128] (channel-major) in shared memory, laid out as the
-//                8 x 16-byte core matrices that tcgen05.mma reads without swizzle; K^ of the
-//                next block is produced while the softmax of this one runs;
+//   K^, V^       fp16 operand tiles [128 tokens x 128 channels] in shared memory, two stages.
+//                Without a workspace eight warps expand the packed tiles of the block (core-matrix
+//                layout without swizzle); with one, prefill_dequant_kernel has expanded the whole
+//                layer into fp16 rows beforehand and two threads fetch the block with tiled TMA
+//                copies into the 128-byte swizzled layout;
 //   S_i = Q_i K^T  8 x tcgen05.mma (M 128, N 128, K 16) per query tile, fp32 in tensor memory;
-//   softmax      eight warps, one query row per thread, read S_i with tcgen05.ld, apply the
-//                causal mask, keep a lazily moved reference maximum and the running sum, write
-//                P_i as fp16 into shared memory;
-//   O_i += P_i V^  8 x tcgen05.mma accumulating in tensor memory across blocks (rescaled in place
-//                on the rare blocks where the reference maximum moves).
-// The three roles (softmax, dequantise, MMA issue) run concurrently and meet on mbarriers only.
-// Every wait is bounded; on expiry the CTA records MOQAE_ERR_TIMEOUT, every role stops and the
-// tensor memory is still freed.
+//   softmax      one thread per query row (two with a workspace, 64 columns each) reads S_i with
+//                tcgen05.ld, applies the causal mask, keeps a lazily moved reference maximum and
+//                the running sum, and writes P_i as packed fp16 over the consumed columns of S_i;
+//   O_i += P_i V^  8 x tcgen05.mma with P_i as a tensor-memory operand, accumulating in tensor
+//                memory across blocks (rescaled in place on the rare blocks where the reference
+//                maximum moves).
+// The roles run concurrently and meet on mbarriers (plus one named barrier per pair of softmax
+// warps that share rows).  Every mbarrier wait is bounded; on expiry the CTA records
+// MOQAE_ERR_TIMEOUT, every role stops and the tensor memory is still freed.
 #include <cstring>
 
 #include <cuda.h>
@@ -310,9 +312,11 @@ __device__ __forceinline__ void copy_rows(const uint8_t* __restrict__ src, uint8
 }
 
 // ---- the kernel ----------------------------------------------------------------------------
-// Roles (17 warps): warps 0..3 and 4..7 are the softmax threads of the CTA's two query tiles
-// (one row each, tensor-memory lane = tid % 128); warps 8..11 dequantise the keys and warps
-// 12..15 the values of every block (one storage tile each); warp 16 issues the MMAs.  Shared
+// Roles without a workspace (17 warps): warps 0..3 and 4..7 are the softmax threads of the CTA's
+// two query tiles (one row each, tensor-memory lane = tid % 128); warps 8..11 dequantise the
+// keys and warps 12..15 the values of every block (one storage tile each); warp 16 issues the
+// MMAs.  With a workspace (19 warps): warps 8..15 are a second set of softmax threads (warp w + 8
+// shares the rows of warp w and takes the other 64 columns), warps 17 and 18 fetch K^ and V^.  Shared
 // memory holds the two query tiles and kStages blocks of K^ and of V^; the probabilities are an
 // A operand read from tensor memory.  Tensor memory (512 columns):
 //   S_i   128 columns at 128 i        scores (fp32) of the current block; P_i (packed fp16, 64
@@ -323,10 +327,10 @@ __device__ __forceinline__ void copy_rows(const uint8_t* __restrict__ src, uint8
 // when fed by one issuing thread.  The two tiles alternate: while the softmax threads of one
 // work on S_i, the pipe runs O += P V^ and the next S of the other.  The roles meet only on
 // mbarriers:
-//   kfull[st] / vfull[st]   K^ / V^ of a block are in stage st               (4 dequant warps)
+//   kfull[st] / vfull[st]   K^ / V^ of a block are in stage st               (4 dequant warps, or the TMA bytes)
 //   kfree[st] / vfree[st]   the products that read stage st are done         (tcgen05.commit)
 //   sfull[i]                S_i = Q_i K^T is in tensor memory                (tcgen05.commit)
-//   pfull[i]                P_i is in tensor memory                          (4 softmax warps)
+//   pfull[i]                P_i is in tensor memory                          (the tile's 4 or 8 softmax warps)
 //   ofull[i]                the last O_i += P_i V^ is done                   (tcgen05.commit, once)
 // Stage barriers complete once per kStages blocks, tile barriers once per block, and every
 // waiter follows its barrier completion by completion, so waiting on the parity of the
