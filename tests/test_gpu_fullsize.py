@@ -115,3 +115,56 @@ def test_decode_sampled_heads_whole_context(job):
         ref = O.decode_attn(qh, wl.dtype, oc, wl.chunk)
         ok, e_abs, e_rel = H.attn_tolerance_ok(out[b, h * G:(h + 1) * G][None], ref)
         assert ok, (b, h, e_abs, e_rel)
+
+
+def test_prefill_attention_sampled_rows_at_the_32k_prompt():
+    """Prefill attention at the size the benchmark times it (32 heads, 32768 (+ tail) tokens, chunk
+    128, bf16, seeded mixed map), both with and without the fp16 workspace: sampled (head, position)
+    rows are recomputed by the oracle from the GPU's own packed cache of that head."""
+    wl = W.WORKLOADS["cfg2"]
+    B, Hq, Hkv, chunk, dtype = 1, wl.n_q_heads, wl.n_kv_heads, wl.chunk, wl.dtype
+    T = wl.context + 37
+    C = T // chunk
+    dev = "cuda"
+    cfg = mq.make_config(n_layers=1, n_q_heads=Hq, n_kv_heads=Hkv, chunk=chunk, dtype=dtype, d_in=64,
+                         max_tokens=T, batch=B, tail_capacity=chunk)
+    K, V = synth.keys_values(B, T, Hkv, 128, dtype, 5151, dev, outlier_frac=wl.outlier_frac)
+    q = synth.normal((B, T, Hq, 128), dtype, 5152, dev)
+    cache = mq.moqae_cache_bind(cfg, [C, C, C, C])
+    forced = torch.from_numpy(synth.multinomial_map(B, C, wl.mix, 78)).to(dev)
+    mq.moqae_quantize_kv(cfg, K, V, T, 0, cache, forced_map=forced)
+    outs = []
+    ws = torch.empty(mq.moqae_prefill_attn_workspace(cfg, T), dtype=torch.uint8, device=dev)
+    for workspace in (None, ws):
+        out = torch.full((B, T, Hq, 128), float("nan"), dtype=torch.float32, device=dev)
+        mq.moqae_prefill_attn(cfg, q, T, 0, cache, out, workspace=workspace)
+        torch.cuda.synchronize()
+        assert mq.moqae_poll_status(cache) == 0
+        outs.append(out)
+    gmap = cache.map[0, :, :C].cpu().numpy()
+    slot, count = O.assign_slots(gmap)
+    r = T % chunk
+    abs_tol = 3 * 2.0 ** -11 * float(V.float().abs().max())
+    G = Hq // Hkv
+    rows = [0, 1, 31, 127, 128, 255, 256, 257, 4095, 4096, 17011, wl.context - 1, wl.context, T - 1]
+    for h in (0, 13, Hkv - 1):
+        pools = []
+        for w in range(4):
+            n = int(count[0, w])
+            pools.append(cache.pool(w)[0, 0, h, :max(n, 1)].cpu().numpy()[None, None])
+        oc = dict(pools=pools, map=gmap, slot=slot, count=count, tail_len=r,
+                  tail_k=cache.tail("k")[0, 0, h, :r].cpu().numpy().view(np.uint16)[None, None],
+                  tail_v=cache.tail("v")[0, 0, h, :r].cpu().numpy().view(np.uint16)[None, None])
+        K64, V64 = O.cache_kv_rows_in_order(oc, dtype, chunk, 0, 0)
+        assert K64.shape[0] == T
+        for g in range(G):
+            hq = h * G + g
+            qh = O.to_f64(synth.to_u16(q[0, rows, hq]), dtype)                 # [rows, 128]
+            for n, t in enumerate(rows):
+                s = (K64[:t + 1] @ qh[n]) / np.sqrt(128.0)
+                p = np.exp(s - s.max())
+                want = (p @ V64[:t + 1]) / p.sum()
+                for out in outs:
+                    got = out[0, t, hq].cpu().numpy().astype(np.float64)
+                    err = np.abs(got - want)
+                    assert err.max() <= abs_tol and err.max() <= 1e-2 * max(np.abs(want).max(), 1e-30), (h, g, t, err.max())
