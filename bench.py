@@ -122,12 +122,13 @@ class Job:
 
     N_DISTINCT = 4      # distinct per-layer K/V inputs; layer l reads input l mod 4 (each > L2)
 
-    def __init__(self, wl, device, seed=1234, context=None, force_map=False, rf=1):
+    def __init__(self, wl, device, seed=1234, context=None, force_map=False, rf=1, overlap=True):
         import torch
 
         from paper_2506_07533_b200 import binding as mq
         from paper_2506_07533_b200 import synth
         self.torch, self.mq, self.wl, self.device = torch, mq, wl, device
+        self.overlap = overlap
         T = self.T = context or wl.context
         B, Hkv, Hq = wl.batch, wl.n_kv_heads, wl.n_q_heads
         self.cfg = mq.make_config(n_layers=wl.n_layers, n_q_heads=Hq, n_kv_heads=Hkv, chunk=wl.chunk,
@@ -148,7 +149,7 @@ class Job:
             self.k_new = synth.normal((wl.decode_steps, wl.n_layers, B, Hkv, 128), wl.dtype, seed + 11, device)
             self.v_new = synth.normal((wl.decode_steps, wl.n_layers, B, Hkv, 128), wl.dtype, seed + 12, device)
         self.out = torch.zeros((wl.n_layers, B, Hq, 128), dtype=torch.float32, device=device)
-        self.ws = torch.empty(mq.moqae_decode_attn_workspace(self.cfg), dtype=torch.uint8, device=device)
+        self.ws = torch.zeros(mq.moqae_decode_attn_workspace(self.cfg), dtype=torch.uint8, device=device)
         self.n_splits = self.ws.numel() // (B * Hq * 130 * 4)
         # capacity: room for the calibrated mix with slack, never more than all chunks
         C = T // wl.chunk
@@ -222,8 +223,11 @@ class Job:
     def decode_all(self):
         wl = self.wl
         if wl.decode_steps == 1:
+            # the layers' calls read nothing the call before them writes, so each may start while
+            # the previous one is still finishing (all but the first, which follows other work)
             for l in range(wl.n_layers):
-                self.mq.moqae_decode_attn(self.cfg, self.q[l], l, self.cache, self.out[l], self.ws)
+                flags = self.mq.DECODE_OVERLAP_PREVIOUS if (l > 0 and self.overlap) else 0
+                self.mq.moqae_decode_attn_ex(self.cfg, self.q[l], l, self.cache, self.out[l], self.ws, flags=flags)
             return
         # generation loop: every step appends one token per sequence to each layer's 16-bit tail
         # (routing is not re-run) and attends over the grown cache
@@ -301,7 +305,8 @@ def run_ours(args):
         wl = dataclasses.replace(wl, rs_group=args.rs_group)
     if args.mix:
         wl = dataclasses.replace(wl, mix=tuple(float(x) for x in args.mix.split(",")))
-    job = Job(wl, device, seed=1234 + rank, context=args.context, force_map=bool(args.mix), rf=0 if args.no_rf else 1)
+    job = Job(wl, device, seed=1234 + rank, context=args.context, force_map=bool(args.mix), rf=0 if args.no_rf else 1,
+              overlap=not args.no_overlap)
     torch.cuda.synchronize()
 
     def one_step(ev=None):
@@ -377,7 +382,9 @@ def run_ours(args):
                        "mix_source": "router bias calibrated" if job.forced is None else "forced seeded multinomial map",
                        "l2": "working set per phase >> 126 MB L2; no layer is touched twice in a row",
                        "parallelism": "replicas only" if world > 1 else "single GPU",
-                       "n_splits": job.n_splits},
+                       "n_splits": job.n_splits,
+                       "decode_launches": ("consecutive layers overlap (programmatic dependent launch)"
+                                           if (job.overlap and wl.decode_steps == 1) else "serialised")},
             "phase_ms": {"route": round(ms_route, 4), "quantize_pack": round(ms_quant, 4),
                          "decode_attn": round(ms_dec, 4)},
             "context_tokens_per_s": round(world * wl.batch * job.T * wl.decode_steps / (ms_dec * 1e-3), 1),
@@ -608,6 +615,8 @@ def main():
     ap.add_argument("--mix", default=None,
                     help="four comma-separated shares: skip the router and force a seeded multinomial map "
                          "with this 2/4/8/16-bit mix (e.g. 1,0,0,0 = uniform 2-bit)")
+    ap.add_argument("--no-overlap", action="store_true",
+                    help="serialise the decode launches of consecutive layers (no programmatic dependent launch)")
     ap.add_argument("--e2e-steps", type=int, default=1)
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--reference-tokens", type=int, default=32768)

@@ -212,7 +212,11 @@ int moqae_flush_tail(const moqae_config* cfg, const void* hidden_tail, const voi
                      const float* W3, const float* bias, int32_t layer_group, const moqae_cache* cache,
                      void* stream);
 
-/* Bytes of scratch moqae_decode_attn needs for `cfg` on the current device (host out). */
+/*
+ * Bytes of scratch moqae_decode_attn needs for `cfg` on the current device (host out).
+ * Layout: float [batch][n_q_heads][n_splits][130] split partials, then int32
+ * [batch][n_kv_heads] arrival counters.
+ */
 int moqae_decode_attn_workspace(const moqae_config* cfg, int64_t* out_bytes);
 
 /*
@@ -221,12 +225,39 @@ int moqae_decode_attn_workspace(const moqae_config* cfg, int64_t* out_bytes);
  *   h / (n_q_heads / n_kv_heads), K̂ and V̂ being the dequantised cache rows plus the tail.
  *   q [batch][n_q_heads][128] input dtype; out [batch][n_q_heads][128] float32;
  *   scale <= 0 selects 1/sqrt(128).  An empty cache gives zeros.
- *   workspace: at least moqae_decode_attn_workspace bytes, 16-byte aligned; contents are
- *   scratch (split partials and arrival counters), overwritten by every call.
+ *   workspace: at least moqae_decode_attn_workspace bytes, 16-byte aligned.  ZERO IT ONCE after
+ *   allocating it (cudaMemsetAsync on the same stream is enough): the arrival counters at its end
+ *   must be zero when a call starts, and every completed call leaves them zero, so no call
+ *   clears them and consecutive calls may reuse the buffer as it is.  The partials in front of
+ *   them are plain scratch.  Zero the buffer again after a call that ended in
+ *   MOQAE_ERR_TIMEOUT and before using it with a different configuration.
+ *   Domain: q finite with |q| < 2^40; cache contents as moqae_quantize_kv writes them.  Inside
+ *   that domain no intermediate leaves the fp16 range: each query row is normalised by a power
+ *   of two before it meets the key scales, and the softmax weights are kept <= 2 before they
+ *   meet the value scales.
  */
 int moqae_decode_attn(const moqae_config* cfg, const void* q, int32_t layer,
                       const moqae_cache* cache, float* out, float scale, void* workspace,
                       int64_t workspace_bytes, void* stream);
+
+/*
+ * moqae_decode_attn with flags (flags = 0 is moqae_decode_attn).
+ *   MOQAE_DECODE_OVERLAP_PREVIOUS: the launch is made with programmatic stream serialisation, so
+ *   its CTAs may start while the kernel enqueued on `stream` directly before it is still
+ *   finishing (they take the SM slots that kernel frees), which hides launch latency, the start-up
+ *   of the copy pipelines and the uneven finish of the previous kernel's CTAs.  q, the cache
+ *   tables, pools and tail are then READ before that previous kernel is known to be complete; out
+ *   and workspace are touched only after it is.  The caller therefore promises that the kernel
+ *   directly before this call on the stream does not write anything this call reads - true for a
+ *   run of decode calls over different layers (Limitations section: the attention over the
+ *   quantised cache is the cost that grows with the context), false directly after
+ *   moqae_append_kv, moqae_quantize_kv or moqae_flush_tail of the same cache.  Any other bit in
+ *   flags: MOQAE_ERR_INVALID_ARG.
+ */
+#define MOQAE_DECODE_OVERLAP_PREVIOUS 1
+int moqae_decode_attn_ex(const moqae_config* cfg, const void* q, int32_t layer,
+                         const moqae_cache* cache, float* out, float scale, void* workspace,
+                         int64_t workspace_bytes, int32_t flags, void* stream);
 
 /*
  * Causal attention of the prompt over its own quantised cache (Section 3.1: a block quantises
@@ -269,8 +300,10 @@ int moqae_prefill_attn(const moqae_config* cfg, const void* q, int32_t T, int32_
  *   - The first call on each device looks up the array's device address (that device must be
  *     current, as for every call); make that first call outside any stream capture.
  *   - All calls on one device share the one array, and it keeps whatever the previous call
- *     left there.  Every call overwrites the part it reads, so nothing needs clearing, but two
- *     calls that overlap on the GPU (different streams, no ordering) race on it: order them.
+ *     left there.  The only part that must start at zero, the arrival counters, is cleared by
+ *     every call (a memset node on the caller's stream in front of the kernel); the partials are
+ *     overwritten before they are read.  Two calls that overlap on the GPU (different streams,
+ *     no ordering) race on the array: order them.
  */
 int64_t moqae_decode_attn_static_max_bytes(void);
 int moqae_decode_attn_static(const moqae_config* cfg, const void* q, int32_t layer,

@@ -25,7 +25,8 @@ ERR_WORKSPACE_TOO_SMALL, ERR_CUDA, ERR_TIMEOUT = -5, -6, -7
 EXPORTS = ["moqae_version", "moqae_last_cuda_error", "moqae_error_string", "moqae_cache_bytes",
            "moqae_cache_bind", "moqae_route", "moqae_quantize_kv", "moqae_append_kv",
            "moqae_decode_attn_workspace", "moqae_decode_attn", "moqae_poll_status",
-           "moqae_decode_attn_static", "moqae_decode_attn_static_max_bytes", "moqae_flush_tail", "moqae_prefill_attn", "moqae_prefill_attn_workspace"]
+           "moqae_decode_attn_static", "moqae_decode_attn_static_max_bytes", "moqae_flush_tail", "moqae_prefill_attn",
+           "moqae_prefill_attn_workspace", "moqae_decode_attn_ex"]
 
 
 class MoqaeConfig(C.Structure):
@@ -90,6 +91,8 @@ def lib() -> C.CDLL:
         L.moqae_decode_attn_workspace.argtypes = [C.POINTER(MoqaeConfig), C.POINTER(C.c_int64)]
         L.moqae_decode_attn.argtypes = [C.POINTER(MoqaeConfig), C.c_void_p, C.c_int32, C.POINTER(MoqaeCache),
                                         C.c_void_p, C.c_float, C.c_void_p, C.c_int64, C.c_void_p]
+        L.moqae_decode_attn_ex.argtypes = [C.POINTER(MoqaeConfig), C.c_void_p, C.c_int32, C.POINTER(MoqaeCache),
+                                           C.c_void_p, C.c_float, C.c_void_p, C.c_int64, C.c_int32, C.c_void_p]
         L.moqae_poll_status.argtypes = [C.POINTER(MoqaeCache), C.c_void_p, C.POINTER(C.c_int32)]
         L.moqae_decode_attn_static.argtypes = [C.POINTER(MoqaeConfig), C.c_void_p, C.c_int32,
                                                C.POINTER(MoqaeCache), C.c_void_p, C.c_float, C.c_void_p]
@@ -250,10 +253,21 @@ def moqae_decode_attn_workspace(cfg) -> int:
     return int(out.value)
 
 
+DECODE_OVERLAP_PREVIOUS = 1
+
+
 def moqae_decode_attn(cfg, q, layer, cache: Cache, out, workspace, scale=0.0):
     _check(lib().moqae_decode_attn(C.byref(cfg), _ptr(q), int(layer), C.byref(cache.view), _ptr(out),
                                    C.c_float(scale), _ptr(workspace), int(workspace.numel() * workspace.element_size()),
                                    _stream()), "moqae_decode_attn")
+
+
+def moqae_decode_attn_ex(cfg, q, layer, cache: Cache, out, workspace, flags=0, scale=0.0):
+    """moqae_decode_attn with flags; DECODE_OVERLAP_PREVIOUS lets the launch start while the
+    previous kernel on the stream is finishing (see include/moqae.h for the caller's promise)."""
+    _check(lib().moqae_decode_attn_ex(C.byref(cfg), _ptr(q), int(layer), C.byref(cache.view), _ptr(out),
+                                      C.c_float(scale), _ptr(workspace), int(workspace.numel() * workspace.element_size()),
+                                      int(flags), _stream()), "moqae_decode_attn_ex")
 
 
 def moqae_decode_attn_static_max_bytes() -> int:

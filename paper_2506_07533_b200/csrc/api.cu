@@ -1,4 +1,6 @@
 // C ABI of the library: argument validation and dispatch to the kernel launchers.
+#include <atomic>
+
 #include "common.cuh"
 
 namespace {
@@ -76,6 +78,19 @@ int check_cache(const moqae_cache* k, moqae::CacheView* v) {
 
 namespace moqae {
 void record_cuda_error(cudaError_t e) { g_last_cuda_error = static_cast<int>(e); }
+
+int sm_count_of_current_device() {
+  constexpr int kMaxDevices = 64;
+  static std::atomic<int> cached[kMaxDevices];          // zero = not looked up yet
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 148;
+  int v = cached[dev].load(std::memory_order_relaxed);
+  if (v == 0) {
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) v = 148;
+    cached[dev].store(v, std::memory_order_relaxed);
+  }
+  return v;
+}
 }  // namespace moqae
 
 #pragma GCC visibility push(default)
@@ -234,6 +249,13 @@ int moqae_decode_attn_workspace(const moqae_config* cfg, int64_t* out_bytes) {
 
 int moqae_decode_attn(const moqae_config* cfg, const void* q, int32_t layer, const moqae_cache* cache,
                       float* out, float scale, void* workspace, int64_t workspace_bytes, void* stream) {
+  return moqae_decode_attn_ex(cfg, q, layer, cache, out, scale, workspace, workspace_bytes, 0, stream);
+}
+
+int moqae_decode_attn_ex(const moqae_config* cfg, const void* q, int32_t layer, const moqae_cache* cache,
+                         float* out, float scale, void* workspace, int64_t workspace_bytes, int32_t flags,
+                         void* stream) {
+  if (flags & ~MOQAE_DECODE_OVERLAP_PREVIOUS) return MOQAE_ERR_INVALID_ARG;
   int rc = check_config(cfg);
   if (rc != MOQAE_OK) return rc;
   moqae::CacheView cv;
@@ -247,7 +269,7 @@ int moqae_decode_attn(const moqae_config* cfg, const void* q, int32_t layer, con
   if (workspace_bytes < need) return MOQAE_ERR_WORKSPACE_TOO_SMALL;
   if (!(scale > 0.0f)) scale = 0.08838834764831845f;   // 1/sqrt(128)
   cudaError_t e = moqae::launch_decode(dm, cv, q, layer, out, scale, static_cast<float*>(workspace), s,
-                                       static_cast<cudaStream_t>(stream));
+                                       (flags & MOQAE_DECODE_OVERLAP_PREVIOUS) != 0, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? MOQAE_OK : cuda_fail(e);
 }
 

@@ -62,6 +62,9 @@ __device__ __forceinline__ uint8_t* slot_ptr(const CacheView& cv, const Dims& dm
   return cv.pool[w] + idx * slot_bytes;
 }
 
+// Number of SMs of the device that is current on the calling thread (looked up once per device).
+int sm_count_of_current_device();
+
 // Remember `e` as the code moqae_last_cuda_error() reports on this thread.
 void record_cuda_error(cudaError_t e);
 
@@ -85,9 +88,12 @@ cudaError_t launch_prefill_attn(const Dims& dm, const CacheView& cv, const void*
                                 float* out, void* workspace, cudaStream_t st);
 long long prefill_workspace_bytes(const Dims& dm, int T);
 long long decode_workspace_bytes(const Dims& dm, int n_splits);
+// byte offset and length of the arrival counters inside a decode workspace for `cfg`
+void decode_counter_region(const moqae_config* cfg, long long* offset, long long* bytes);
 cudaError_t launch_decode_mma(const Dims& dm, const CacheView& cv, const void* q, int layer, float scale,
-                              float* ws_o, float* ws_ml, int* arrived, float* out, int n_splits, cudaStream_t st);
+                              float* ws_o, float* ws_ml, int* arrived, float* out, int n_splits, bool overlap_previous,
+                              cudaStream_t st);
 cudaError_t launch_decode(const Dims& dm, const CacheView& cv, const void* q, int layer, float* out,
-                          float scale, float* workspace, int n_splits, cudaStream_t st);
+                          float scale, float* workspace, int n_splits, bool overlap_previous, cudaStream_t st);
 
 }  // namespace moqae

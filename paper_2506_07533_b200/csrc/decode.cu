@@ -13,12 +13,7 @@
 namespace moqae {
 
 int decode_num_splits(const Dims& dm) {
-  static int sms = 0;
-  if (sms == 0) {
-    int dev = 0, v = 148;
-    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev);
-    sms = v > 0 ? v : 148;
-  }
+  const int sms = sm_count_of_current_device();
   // one full wave: every CTA gets the same number of bytes, so a partial second wave would
   // cost a whole extra pass
   const int pairs = dm.batch * dm.n_kv_heads;
@@ -36,15 +31,25 @@ long long decode_workspace_bytes(const Dims& dm, int n_splits) {
   return (bytes + 15) / 16 * 16;
 }
 
+void decode_counter_region(const moqae_config* cfg, long long* offset, long long* bytes) {
+  Dims dm{};
+  dm.batch = cfg->batch;
+  dm.n_q_heads = cfg->n_q_heads;
+  dm.n_kv_heads = cfg->n_kv_heads;
+  const long long rows = static_cast<long long>(dm.batch) * dm.n_q_heads * decode_num_splits(dm);
+  *offset = rows * (kHeadDim + 2) * 4;
+  *bytes = static_cast<long long>(dm.batch) * dm.n_kv_heads * 4;
+}
+
 cudaError_t launch_decode(const Dims& dm, const CacheView& cv, const void* q, int layer, float* out,
-                          float scale, float* workspace, int n_splits, cudaStream_t st) {
+                          float scale, float* workspace, int n_splits, bool overlap_previous, cudaStream_t st) {
   const long long rows = static_cast<long long>(dm.batch) * dm.n_q_heads * n_splits;
   float* ws_o = workspace;
   float* ws_ml = workspace + rows * kHeadDim;
   int* arrived = reinterpret_cast<int*>(ws_ml + rows * 2);
-  cudaError_t e = cudaMemsetAsync(arrived, 0, sizeof(int) * static_cast<size_t>(dm.batch) * dm.n_kv_heads, st);
-  if (e != cudaSuccess) return e;
-  return launch_decode_mma(dm, cv, q, layer, scale, ws_o, ws_ml, arrived, out, n_splits, st);
+  // the counters are zero on entry (the caller zeroes a new workspace once) and the kernel
+  // leaves them zero: the last arrival of every (sequence, kv head) wraps its counter around
+  return launch_decode_mma(dm, cv, q, layer, scale, ws_o, ws_ml, arrived, out, n_splits, overlap_previous, st);
 }
 
 }  // namespace moqae

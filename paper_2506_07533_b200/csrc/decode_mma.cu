@@ -63,12 +63,12 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded by elapsed SM cycles (about half a second), not by the number of attempts.
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, long long limit = kWaitCycles) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   do {
     if (mbar_try_wait(bar, parity)) return true;
-  } while (clock64() - t0 < kWaitCycles);
+  } while (clock64() - t0 < limit);
   return false;
 }
 
@@ -145,7 +145,15 @@ struct State {
   float acc[8][4];   // M-tile mt = 2*cg + hf: rows g / g+8 = channels 32cg+4g+2hf / +1; cols = queries 2t4, 2t4+1
   float oz[4];       // rows 0..3 (lanes g < 4): zero-point term per channel group; row 4 (g == 4): the
                      // running sums l, taken over the SAME rounded weights the values are multiplied by
-  float m[2];        // running maxima (base-2 exponent units) of queries 2t4, 2t4+1
+  float m[2];        // reference maxima (base-2 exponent units) of queries 2t4, 2t4+1
+};
+
+// Per-lane constants of the quantised phases.  Every query row is normalised by a power of two,
+// q' = q * 2^-e with |q'| < 1, before it becomes an fp16 operand, so that q' * s_k can never leave
+// the fp16 range whatever the key scale is; the power of two comes back, exactly, in these factors.
+struct LaneConst {
+  float cs[2];       // raw score sum (units of 2^-24 * 2^-e) -> base-2 logits, queries 2t4 and 2t4+1
+  float cbg;         // the same for the zero-point term of query g (no 2^-24 there)
 };
 
 __device__ __forceinline__ void rescale(State& st, float c0, float c1) {
@@ -156,34 +164,45 @@ __device__ __forceinline__ void rescale(State& st, float c0, float c1) {
   st.oz[0] *= c0; st.oz[1] *= c1; st.oz[2] *= c0; st.oz[3] *= c1;
 }
 
-// Online-softmax update for NV score vectors x[v][4] (d-fragment order: row g q0, row g q1,
-// row g+8 q0, row g+8 q1; already in base-2 units; -inf = masked).  Returns p~ = 2^(6 - kSlack) * p.
-// The reference maximum m is moved lazily: only when some score exceeds it by more than kSlack
-// does the warp reduce the true maximum (three shuffle rounds) and rescale its accumulators;
-// otherwise m stays and the weights are at most 2^6, well inside fp16 either way.
+// Online softmax with a lazily moved reference maximum m: only when some score exceeds m by more
+// than kSlack does the warp reduce the true maximum (three shuffle rounds) and rescale its
+// accumulators; otherwise m stays.  Weights are p~ = 2^(x - m + PK - kSlack) <= 2^PK, with PK
+// chosen per width so that p~ * s_v cannot leave the fp16 range for any scale the quantiser can
+// produce (s_v <= 65504 / (2^b - 1)) while typical products stay well above the subnormals:
+// 2^1 * 21835, 2^3 * 4367, 2^7 * 257 < 65504.  Between phases the state is kept at PK = 0.
 constexpr float kSlack = 3.0f;
+template <int BITS> __host__ __device__ constexpr int pmax_log2() { return BITS == 2 ? 1 : BITS == 4 ? 3 : BITS == 8 ? 7 : 6; }
+
+// xm0 / xm1: this lane's largest scores of queries 2t4 / 2t4+1 in the unit about to be weighted
+__device__ __forceinline__ void move_reference(State& st, float xm0, float xm1) {
+  const bool over = (xm0 > st.m[0] + kSlack) || (xm1 > st.m[1] + kSlack);
+  if (__any_sync(0xffffffffu, over)) {
+#pragma unroll
+    for (int o = 4; o <= 16; o <<= 1) {
+      xm0 = fmaxf(xm0, __shfl_xor_sync(0xffffffffu, xm0, o));
+      xm1 = fmaxf(xm1, __shfl_xor_sync(0xffffffffu, xm1, o));
+    }
+    const float n0 = fmaxf(st.m[0], xm0), n1 = fmaxf(st.m[1], xm1);
+    const float c0 = (st.m[0] == -INFINITY) ? 0.0f : ex2f(st.m[0] - n0);
+    const float c1 = (st.m[1] == -INFINITY) ? 0.0f : ex2f(st.m[1] - n1);
+    rescale(st, c0, c1);
+    st.m[0] = n0; st.m[1] = n1;
+  }
+}
+
+// Update for NV score vectors x[v][4] (d-fragment order: row g q0, row g q1, row g+8 q0,
+// row g+8 q1; already in base-2 units; -inf = masked).  Returns the weights p~ in x.
 template <int NV>
 __device__ __forceinline__ void softmax_update(State& st, float x[NV][4]) {
+  constexpr float kPmaxLog2 = static_cast<float>(pmax_log2<16>());
   float mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll
   for (int v = 0; v < NV; ++v) {
     mx0 = fmaxf(mx0, fmaxf(x[v][0], x[v][2]));
     mx1 = fmaxf(mx1, fmaxf(x[v][1], x[v][3]));
   }
-  const bool over = (mx0 > st.m[0] + kSlack) || (mx1 > st.m[1] + kSlack);
-  if (__any_sync(0xffffffffu, over)) {
-#pragma unroll
-    for (int o = 4; o <= 16; o <<= 1) {
-      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, o));
-      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, o));
-    }
-    const float n0 = fmaxf(st.m[0], mx0), n1 = fmaxf(st.m[1], mx1);
-    const float c0 = (st.m[0] == -INFINITY) ? 0.0f : ex2f(st.m[0] - n0);
-    const float c1 = (st.m[1] == -INFINITY) ? 0.0f : ex2f(st.m[1] - n1);
-    rescale(st, c0, c1);
-    st.m[0] = n0; st.m[1] = n1;
-  }
-  const float o0 = (6.0f - kSlack) - st.m[0], o1 = (6.0f - kSlack) - st.m[1];
+  move_reference(st, mx0, mx1);
+  const float o0 = (kPmaxLog2 - kSlack) - st.m[0], o1 = (kPmaxLog2 - kSlack) - st.m[1];
 #pragma unroll
   for (int v = 0; v < NV; ++v) {
     x[v][0] = ex2f(x[v][0] + o0); x[v][1] = ex2f(x[v][1] + o1);
@@ -191,121 +210,176 @@ __device__ __forceinline__ void softmax_update(State& st, float x[NV][4]) {
   }
 }
 
-// ---- one quantised tile (32 tokens) from shared memory ---------------------------------
-// Lane (g, t4) = (lane / 4, lane % 4).  qb[r], r = 0..15: fp16 pair (q[c_lo(r)], q[c_hi(r)])
+// ---- NT quantised tiles (32 tokens each) from shared memory ----------------------------
+// Lane (g, t4) = (lane / 4, lane % 4).  qb[r], r = 0..15: fp16 pair (q'[c_lo(r)], q'[c_hi(r)])
 // of query g (zero for g >= G) for the channels 32*t4 + .. that key register r carries;
 // qc[r] = qb[r] times the power of two that undoes the register's bit position.
 // G4 (query group of at most 4): B columns 4..7 carry the low parts of the folded queries
 // 0..3, so one MMA chain yields both halves of the exact product and the score of query c
 // is column c plus column c + 4; columns 4..7 then simply mirror 0..3 in everything after.
-template <int BITS, bool G4>
-__device__ __forceinline__ void process_qtile(const uint8_t* __restrict__ tile, State& st,
+// NT = 2 (neighbouring 2-bit tiles, fetched by one copy): one reference-maximum check, one set of
+// zero-point MMAs and one round of bias shuffles serve both tiles.
+template <int BITS, int NT, bool G4>
+__device__ __forceinline__ void process_qunit(const uint8_t* __restrict__ unit, State& st,
                                               const uint32_t (&qc)[16], const uint32_t (&qb)[16],
-                                              float c_score, float c_bias, int lane) {
+                                              const LaneConst& lc, int lane) {
   using F = Fmt<BITS>;
+  constexpr int TB = kMetaBytes + 1024 * BITS;       // bytes per tile
+  constexpr int NB = 2 * NT;                         // 16-token blocks
   const int g = lane >> 2, t4 = lane & 3;
-  const uint8_t* kpay = tile + kMetaBytes;
-  const uint8_t* vpay = kpay + kTileTokens * 16 * BITS;
 
-  // fold the key scales into the query fragment: q*s = hi + lo exactly (two fp16 each), so the
+  // fold the key scales into the query fragments: q'*s = hi + lo exactly (two fp16 each), so the
   // scores carry no rounding besides the fp32 accumulation
-  uint32_t qf[16], ql[G4 ? 1 : 16];
-  {
-    const uint4* sp = reinterpret_cast<const uint4*>(tile) + t4;
-    const uint32_t lo_lane = (G4 && g >= 4) ? 0xffffffffu : 0u;
+  uint32_t qf[NT][16], ql[G4 ? 1 : NT][G4 ? 1 : 16];
+#pragma unroll
+  for (int tl = 0; tl < NT; ++tl) {
+    const uint4* sp = reinterpret_cast<const uint4*>(unit + tl * TB) + t4;
+    const bool lo_lane = G4 && g >= 4;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const uint4 s4 = sp[4 * i];
       const uint32_t sv[4] = {s4.x, s4.y, s4.z, s4.w};
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        const uint32_t hi = hmul2_u32(qc[4 * i + j], sv[j]);
+        uint32_t hi = hmul2_u32(qc[4 * i + j], sv[j]);
         if (G4) {
-          // lanes of columns 0..3: fma(q, s, -0) = hi; lanes of columns 4..7: fma(q, s, -hi) = lo
-          qf[4 * i + j] = hfma2_sub_u32(qc[4 * i + j], sv[j], hi & lo_lane);
+          // lanes of columns 4..7 replace hi by lo = fma(q', s, -hi)
+          if (lo_lane) hi = hfma2_sub_u32(qc[4 * i + j], sv[j], hi);
         } else {
-          qf[4 * i + j] = hi;
-          ql[(4 * i + j) % (G4 ? 1 : 16)] = hfma2_sub_u32(qc[4 * i + j], sv[j], hi);
+          ql[G4 ? 0 : tl][(4 * i + j) % (G4 ? 1 : 16)] = hfma2_sub_u32(qc[4 * i + j], sv[j], hi);
         }
+        qf[tl][4 * i + j] = hi;
       }
     }
   }
-  // zero-point term of the scores: bias[q] = sum_c z_k[c] q[c], exact products.  Here the
-  // queries are the A operand (rows) and the zeros the B operand, the same in every column:
-  // registers 4i, 4i+2 accumulate in row g of `ba`, registers 4i+1, 4i+3 in row g + 8 of `bb`
-  // (the zero array stores each group of four registers in the order 0, 2, 1, 3).
-  float ba[4] = {0.f, 0.f, 0.f, 0.f}, bb[4] = {0.f, 0.f, 0.f, 0.f};
-  {
-    const uint4* zp = reinterpret_cast<const uint4*>(tile + 256) + t4;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const uint4 z4 = zp[4 * i];
-      mma16816<false>(ba, qb[4 * i], qb[4 * i + 1], qb[4 * i + 2], qb[4 * i + 3], z4.x, z4.y);
-      mma16816<false>(bb, qb[4 * i], qb[4 * i + 1], qb[4 * i + 2], qb[4 * i + 3], z4.z, z4.w);
-    }
-  }
-  const float bq = (ba[0] + bb[2]) * c_bias;                 // query g, whatever the column
-  const float bias0 = __shfl_sync(0xffffffffu, bq, 8 * t4);
-  const float bias1 = __shfl_sync(0xffffffffu, bq, 8 * t4 + 4);
 
-  // scores of the two 16-token blocks: rows g and g + 8 of each
-  float x[2][4];
+  // key payload words of every 16-token block: w[b2][hh][j], hh = rows g / g + 8
+  uint32_t w[NB][2][BITS];
 #pragma unroll
-  for (int blk = 0; blk < 2; ++blk) {
-    uint32_t w[2][BITS];           // words of the two row pieces
+  for (int b2 = 0; b2 < NB; ++b2) {
+    const uint8_t* kpay = unit + (b2 >> 1) * TB + kMetaBytes;
+    const int blk = b2 & 1;
     if (BITS == 2) {
-      const uint4 v = *reinterpret_cast<const uint4*>(kpay + (blk * 32 + lane) * 16);
-      w[0][0] = v.x; w[0][1] = v.y; w[1][0] = v.z; w[1][1] = v.w;
+      const uint4 u = *reinterpret_cast<const uint4*>(kpay + (blk * 32 + lane) * 16);
+      w[b2][0][0] = u.x; w[b2][0][1] = u.y; w[b2][1][0] = u.z; w[b2][1][1] = u.w;
     } else if (BITS == 4) {
 #pragma unroll
       for (int hh = 0; hh < 2; ++hh) {
-        const uint4 v = *reinterpret_cast<const uint4*>(kpay + ((2 * blk + hh) * 32 + lane) * 16);
-        w[hh][0] = v.x; w[hh][1] = v.y; w[hh][2 % BITS] = v.z; w[hh][3 % BITS] = v.w;
+        const uint4 u = *reinterpret_cast<const uint4*>(kpay + ((2 * blk + hh) * 32 + lane) * 16);
+        w[b2][hh][0] = u.x; w[b2][hh][1] = u.y; w[b2][hh][2 % BITS] = u.z; w[b2][hh][3 % BITS] = u.w;
       }
     } else {
 #pragma unroll
       for (int hh = 0; hh < 2; ++hh)
 #pragma unroll
         for (int j2 = 0; j2 < 2; ++j2) {
-          const uint4 v = *reinterpret_cast<const uint4*>(kpay + (((2 * blk + hh) * 2 + j2) * 32 + lane) * 16);
-          w[hh][(4 * j2) % BITS] = v.x; w[hh][(4 * j2 + 1) % BITS] = v.y;
-          w[hh][(4 * j2 + 2) % BITS] = v.z; w[hh][(4 * j2 + 3) % BITS] = v.w;
+          const uint4 u = *reinterpret_cast<const uint4*>(kpay + (((2 * blk + hh) * 2 + j2) * 32 + lane) * 16);
+          w[b2][hh][(4 * j2) % BITS] = u.x; w[b2][hh][(4 * j2 + 1) % BITS] = u.y;
+          w[b2][hh][(4 * j2 + 2) % BITS] = u.z; w[b2][hh][(4 * j2 + 3) % BITS] = u.w;
         }
     }
-    uint32_t a[2][16];
+  }
+
+  // Zero-point term of the scores: bias[tile][q] = sum_c z_k[c] q'[c], exact products.  The
+  // queries are the A operand (rows g and g + 8 both hold query g: registers 4i, 4i+2 in row g,
+  // 4i+1, 4i+3 in row g + 8), the zeros the B operand.  B column n carries, for tile (n & 3) >> 1
+  // (NT = 2) or the only tile, the zeros of registers 4i, 4i+2 (n even) or 4i+1, 4i+3 (n odd);
+  // the zero array stores each group of four registers in the order 0, 2, 1, 3.  Element
+  // (g, n even) + element (g + 8, n + 1) is then the full sum for query g: lane (g, t4) finds
+  // both in its own fragment, for tile t4 & 1 (NT = 2).
+  float bd[4] = {0.f, 0.f, 0.f, 0.f};
+  const uint8_t* zp = unit + (NT == 2 ? ((g & 3) >> 1) * TB : 0) + 256 + t4 * 16 + (g & 1) * 8;
+
+  // Raw score sums of the NB blocks (rows g and g + 8 of each).  Step i of a block multiplies key
+  // registers 2i, 2i+1 (made from the payload words right before use) with the folded query; the
+  // steps of all blocks are interleaved so that four independent accumulator chains are always in
+  // flight, and the four zero-point MMAs ride along.
+  constexpr int CH = 4 / NB;                         // accumulator chains per block
+  float sc[NB][CH][4];
 #pragma unroll
-    for (int hh = 0; hh < 2; ++hh)
+  for (int b2 = 0; b2 < NB; ++b2)
 #pragma unroll
-      for (int j = 0; j < BITS; ++j) {
-        const uint32_t wsh = w[hh][j] >> 8;
+    for (int c = 0; c < CH; ++c)
 #pragma unroll
-        for (int rr = 0; rr < F::regs; ++rr)
-          a[hh][j * F::regs + rr] = ext<BITS>(w[hh][j], wsh, rr / F::direct, rr % F::direct);
+      for (int i = 0; i < 4; ++i) sc[b2][c][i] = 0.f;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+#pragma unroll
+    for (int b2 = 0; b2 < NB; ++b2) {
+      uint32_t a[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int r = 2 * i + (k >> 1), hh = k & 1;            // a0: (r0, hh0) a1: (r0, hh1) a2: (r1, hh0) a3: (r1, hh1)
+        const int j = r / F::regs, rr = r % F::regs;
+        const uint32_t word = w[b2][hh][j];
+        a[k] = ext<BITS>(word, word >> 8, rr / F::direct, rr % F::direct);
       }
-    float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-    for (int ks = 0; ks < 8; ks += 2) {
-      mma16816<false>(s0, a[0][2 * ks], a[1][2 * ks], a[0][2 * ks + 1], a[1][2 * ks + 1], qf[2 * ks], qf[2 * ks + 1]);
-      mma16816<false>(s1, a[0][2 * ks + 2], a[1][2 * ks + 2], a[0][2 * ks + 3], a[1][2 * ks + 3], qf[2 * ks + 2], qf[2 * ks + 3]);
+      const int tl = b2 >> 1;
+      mma16816<false>(sc[b2][i % CH], a[0], a[1], a[2], a[3], qf[tl][2 * i], qf[tl][2 * i + 1]);
       if (!G4) {
         constexpr int M = G4 ? 1 : 16;
-        mma16816<false>(s0, a[0][2 * ks], a[1][2 * ks], a[0][2 * ks + 1], a[1][2 * ks + 1], ql[(2 * ks) % M], ql[(2 * ks + 1) % M]);
-        mma16816<false>(s1, a[0][2 * ks + 2], a[1][2 * ks + 2], a[0][2 * ks + 3], a[1][2 * ks + 3], ql[(2 * ks + 2) % M], ql[(2 * ks + 3) % M]);
+        mma16816<false>(sc[b2][i % CH], a[0], a[1], a[2], a[3], ql[G4 ? 0 : tl][(2 * i) % M], ql[G4 ? 0 : tl][(2 * i + 1) % M]);
       }
     }
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      float v = s0[i] + s1[i];
-      if (G4) v += __shfl_xor_sync(0xffffffffu, v, 2);       // column c + column c ^ 4
-      x[blk][i] = fmaf(v, c_score, (i & 1) ? bias1 : bias0);
+    if (i & 1) {
+      const int k = i >> 1;
+      const uint2 z = *reinterpret_cast<const uint2*>(zp + 64 * k);
+      mma16816<false>(bd, qb[4 * k], qb[4 * k + 1], qb[4 * k + 2], qb[4 * k + 3], z.x, z.y);
     }
   }
-  softmax_update<2>(st, x);
+  float bias[NT][2];
+  {
+    const float bq = (bd[0] + bd[3]) * lc.cbg;            // query g, tile t4 & 1
+#pragma unroll
+    for (int tl = 0; tl < NT; ++tl) {
+      bias[tl][0] = __shfl_sync(0xffffffffu, bq, 8 * t4 + (NT == 2 ? tl : 0));
+      bias[tl][1] = __shfl_sync(0xffffffffu, bq, 8 * t4 + 4 + (NT == 2 ? tl : 0));
+    }
+  }
+  float v[NB][4];
+#pragma unroll
+  for (int b2 = 0; b2 < NB; ++b2)
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      float x = sc[b2][0][i];
+      if (CH == 2) x += sc[b2][CH - 1][i];
+      if (G4) x += __shfl_xor_sync(0xffffffffu, x, 2);       // column c + column c ^ 4
+      v[b2][i] = x;
+    }
+
+  // softmax: the factor cs > 0 and the per-tile bias commute with the maximum, so the reference
+  // check runs on the raw sums and every weight costs one FMA and one ex2
+  {
+    float xm0 = -INFINITY, xm1 = -INFINITY;
+#pragma unroll
+    for (int tl = 0; tl < NT; ++tl) {
+      const float r0 = fmaxf(fmaxf(v[2 * tl][0], v[2 * tl][2]), fmaxf(v[2 * tl + 1][0], v[2 * tl + 1][2]));
+      const float r1 = fmaxf(fmaxf(v[2 * tl][1], v[2 * tl][3]), fmaxf(v[2 * tl + 1][1], v[2 * tl + 1][3]));
+      xm0 = fmaxf(xm0, fmaf(r0, lc.cs[0], bias[tl][0]));
+      xm1 = fmaxf(xm1, fmaf(r1, lc.cs[1], bias[tl][1]));
+    }
+    move_reference(st, xm0, xm1);
+    constexpr float kPmaxLog2 = static_cast<float>(pmax_log2<BITS>());
+    const float o0 = (kPmaxLog2 - kSlack) - st.m[0], o1 = (kPmaxLog2 - kSlack) - st.m[1];
+#pragma unroll
+    for (int tl = 0; tl < NT; ++tl) {
+      const float ob0 = bias[tl][0] + o0, ob1 = bias[tl][1] + o1;
+#pragma unroll
+      for (int blk = 0; blk < 2; ++blk) {
+        float* x = v[2 * tl + blk];
+        x[0] = ex2f(fmaf(x[0], lc.cs[0], ob0)); x[1] = ex2f(fmaf(x[1], lc.cs[1], ob1));
+        x[2] = ex2f(fmaf(x[2], lc.cs[0], ob0)); x[3] = ex2f(fmaf(x[3], lc.cs[1], ob1));
+      }
+    }
+  }
 
 #pragma unroll
-  for (int blk = 0; blk < 2; ++blk) {
-    const uint32_t p0 = movmatrix_trans(pack_half2(x[blk][0], x[blk][1]));   // tokens 16blk + 2t4, +1 of query g
-    const uint32_t p1 = movmatrix_trans(pack_half2(x[blk][2], x[blk][3]));   // tokens 16blk + 8 + 2t4, +1
+  for (int b2 = 0; b2 < NB; ++b2) {
+    const uint8_t* tile = unit + (b2 >> 1) * TB;
+    const uint8_t* vpay = tile + kMetaBytes + kTileTokens * 16 * BITS;
+    const int blk = b2 & 1;
+    const uint32_t p0 = movmatrix_trans(pack_half2(v[b2][0], v[b2][1]));   // tokens 16blk + 2t4, +1 of query g
+    const uint32_t p1 = movmatrix_trans(pack_half2(v[b2][2], v[b2][3]));   // tokens 16blk + 8 + 2t4, +1
     {  // zero-point term: rows = channel groups (lanes g < 4)
       uint32_t z0 = (g == 4) ? 0x3C003C00u : 0u, z1 = z0;      // row 4: ones -> sum of the weights
       if (g < 4) {
@@ -326,8 +400,8 @@ __device__ __forceinline__ void process_qtile(const uint8_t* __restrict__ tile, 
     uint32_t wv[NW];
 #pragma unroll
     for (int u = 0; u < BITS / 2; ++u) {
-      const uint4 v = *reinterpret_cast<const uint4*>(vpay + ((blk * (BITS / 2) + u) * 32 + lane) * 16);
-      wv[4 * u] = v.x; wv[4 * u + 1] = v.y; wv[4 * u + 2] = v.z; wv[4 * u + 3] = v.w;
+      const uint4 x4 = *reinterpret_cast<const uint4*>(vpay + ((blk * (BITS / 2) + u) * 32 + lane) * 16);
+      wv[4 * u] = x4.x; wv[4 * u + 1] = x4.y; wv[4 * u + 2] = x4.z; wv[4 * u + 3] = x4.w;
     }
 #pragma unroll
     for (int mt = 0; mt < 8; ++mt) {
@@ -345,21 +419,27 @@ __device__ __forceinline__ void process_qtile(const uint8_t* __restrict__ tile, 
 // power of two that accumulator row `hi` (0: row g, 1: row g + 8) of M-tile mt carries inside
 // a quantised phase, in units of one code (the codes themselves are 2^-24 subnormals)
 template <int BITS> __host__ __device__ constexpr int v_bitpos(int mt, int hi) {
-  return BITS * ((2 * mt + hi) % (8 / BITS));
+  return BITS >= 16 ? 0 : BITS * ((2 * mt + hi) % (BITS >= 16 ? 1 : 8 / BITS));
 }
+// Entering a phase brings the state from the neutral units into the phase's (weights scaled by
+// 2^PK everywhere, and for quantised widths the accumulator rows by their code position); leaving
+// undoes it.  All factors are powers of two.
 template <int BITS>
 __device__ __forceinline__ void phase_scale(State& st, bool enter) {
+  constexpr int pk = pmax_log2<BITS>();
 #pragma unroll
   for (int mt = 0; mt < 8; ++mt)
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      const int e = v_bitpos<BITS>(mt, i >> 1) - 24;          // accumulator = true * 2^e
+      const int e = (BITS == 16 ? 0 : v_bitpos<BITS>(mt, i >> 1) - 24) + pk;     // accumulator = true * 2^e
       st.acc[mt][i] *= enter ? exp2f(static_cast<float>(e)) : exp2f(static_cast<float>(-e));
     }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) st.oz[i] *= enter ? exp2f(static_cast<float>(pk)) : exp2f(static_cast<float>(-pk));
 }
 
 // Query fragments of a quantised phase: qb[r] = (q[c_lo(r)], q[c_hi(r)]) of query g as fp16,
-// qc[r] = qb[r] * 2^(4 - bit position of register r).
+// qc[r] = qb[r] * 2^(-bit position of register r).
 template <int BITS>
 __device__ __forceinline__ void load_q_phase(uint32_t (&qb)[16], uint32_t (&qc)[16], const uint16_t* q_h, int g, int t4) {
   const uint16_t* qrow = q_h + g * kHeadDim + 32 * t4;
@@ -367,7 +447,7 @@ __device__ __forceinline__ void load_q_phase(uint32_t (&qb)[16], uint32_t (&qc)[
   for (int r = 0; r < 16; ++r) {
     const int lo = reg_channel_lo<BITS>(r);
     qb[r] = static_cast<uint32_t>(qrow[lo]) | (static_cast<uint32_t>(qrow[lo + Fmt<BITS>::n / 2]) << 16);
-    qc[r] = hmul2_u32(qb[r], half2_pow2(4 - BITS * reg_m<BITS>(r)));
+    qc[r] = hmul2_u32(qb[r], half2_pow2(-BITS * reg_m<BITS>(r)));
   }
 }
 
@@ -481,7 +561,14 @@ __device__ __forceinline__ void stream_units(Pipe& pp, int n_units, int lane, Sr
   }
   for (int u = 0; u < n_units; ++u) {
     const int s = u % STAGES;
-    if (!mbar_wait_bounded(pp.bars + 8 * s, (pp.parity >> s) & 1u)) { pp.ok = false; return; }
+    if (!mbar_wait_bounded(pp.bars + 8 * s, (pp.parity >> s) & 1u)) {
+      // give the copies still in flight into this ring one more bounded wait each, so that none can
+      // land after the ring has been handed on (the merge reuses it) or the CTA has exited
+      for (int k = u; k < n_units && k < u + STAGES; ++k)
+        mbar_wait_bounded(pp.bars + 8 * (k % STAGES), (pp.parity >> (k % STAGES)) & 1u, kWaitCycles >> 4);
+      pp.ok = false;
+      return;
+    }
     pp.parity ^= (1u << s);
     consume(ring_generic + s * STAGE_BYTES, u);
     __syncwarp();
@@ -509,18 +596,46 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
   uint16_t* q_h = q_in + 8 * kHeadDim;                                             // [8][128] fp16
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kWarps * kRingBytes + 2 * kQBytes);
 
+  // Let a dependent launch (the next decode call, if its caller allowed the overlap) take the SM
+  // slots this grid frees while its slowest CTAs are still running.
+  asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
   const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = lane >> 2, t4 = lane & 3;
   const int G = dm.n_q_heads / dm.n_kv_heads;
 
+  // Every warp finds, for each of the 8 query rows, the power of two 2^e > max |q| (the same
+  // values in all threads), then the CTA writes q (input dtype, for the 16-bit tiles) and
+  // q' = q * 2^-e as fp16 (for the quantised tiles) to shared memory.
+  int q_exp[8];
+#pragma unroll
+  for (int qi = 0; qi < 8; ++qi) {
+    const int qs = G4 ? (qi & 3) : qi;                        // G4: rows 4..7 mirror rows 0..3
+    float mx = 0.0f;
+    if (qs < G) {
+      const uint2 raw4 = *reinterpret_cast<const uint2*>(q + (static_cast<long long>(b) * dm.n_q_heads + h * G + qs) * kHeadDim + 4 * lane);
+      const uint32_t rw[2] = {raw4.x, raw4.y};
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        mx = fmaxf(mx, fabsf(load16_as_float(static_cast<uint16_t>(rw[k >> 1] >> (16 * (k & 1))), BF16 ? MOQAE_DTYPE_BF16 : MOQAE_DTYPE_FP16)));
+    }
+#pragma unroll
+    for (int o = 1; o <= 16; o <<= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    // mx = f * 2^e with f in [1, 2): biased exponent field - 126 gives |q| < 2^e; zero rows take 0
+    const int e = mx > 0.0f ? static_cast<int>((__float_as_uint(mx) >> 23) & 0xffu) - 126 : 0;
+    q_exp[qi] = max(-24, min(e, 40));
+  }
   for (int i = threadIdx.x; i < 8 * kHeadDim; i += kThreads) {
     const int qi = i / kHeadDim, c = i % kHeadDim;
     uint16_t raw = 0;
-    const int qs = G4 ? (qi & 3) : qi;                        // G4: rows 4..7 mirror rows 0..3
+    const int qs = G4 ? (qi & 3) : qi;
     if (qs < G) raw = q[(static_cast<long long>(b) * dm.n_q_heads + h * G + qs) * kHeadDim + c];
     q_in[i] = raw;
-    q_h[i] = BF16 ? __half_as_ushort(__float2half_rn(__uint_as_float(static_cast<uint32_t>(raw) << 16))) : raw;
+    int e = 0;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) e = (k == qi) ? q_exp[k] : e;
+    const float f = load16_as_float(raw, BF16 ? MOQAE_DTYPE_BF16 : MOQAE_DTYPE_FP16);
+    q_h[i] = __half_as_ushort(__float2half_rn(f * __uint_as_float(static_cast<uint32_t>(127 - e) << 23)));
   }
   Pipe pp;
   pp.ring = smem_u32(rings + warp * kRingBytes);
@@ -549,7 +664,19 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
 
   const float log2e = 1.4426950408889634f;
   const float c_bias = scale * log2e;
-  const float c_qscore = c_bias * 1048576.0f;      // scores of quantised tiles carry 2^-20
+  LaneConst lc;                                    // scores of quantised tiles carry 2^-24 * 2^-e
+  {
+    int e0 = 0, e1 = 0, eg = 0;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      e0 = (k == 2 * t4) ? q_exp[k] : e0;
+      e1 = (k == 2 * t4 + 1) ? q_exp[k] : e1;
+      eg = (k == g) ? q_exp[k] : eg;
+    }
+    lc.cs[0] = c_bias * __uint_as_float(static_cast<uint32_t>(127 + 24 + e0) << 23);
+    lc.cs[1] = c_bias * __uint_as_float(static_cast<uint32_t>(127 + 24 + e1) << 23);
+    lc.cbg = c_bias * __uint_as_float(static_cast<uint32_t>(127 + eg) << 23);
+  }
   const uint8_t* my_ring = rings + warp * kRingBytes;
 
   uint32_t qb[16], qc[16];
@@ -573,8 +700,8 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
       stream_units<3, 6144, 1>(pp, n, lane,
           [&](int u, int) { return stream + static_cast<long long>(first + u * kWarps) * 6144; },
           [&](const uint8_t* tiles, int u) {
-            process_qtile<2, G4>(tiles, st, qc, qb, c_qscore, c_bias, lane);
-            if (u < n - 1 || last_bytes == 6144u) process_qtile<2, G4>(tiles + 3072, st, qc, qb, c_qscore, c_bias, lane);
+            if (u < n - 1 || last_bytes == 6144u) process_qunit<2, 2, G4>(tiles, st, qc, qb, lc, lane);
+            else process_qunit<2, 1, G4>(tiles, st, qc, qb, lc, lane);
           }, my_ring, last_bytes);
       phase_scale<2>(st, false);
     }
@@ -589,7 +716,7 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
       load_q_phase<4>(qb, qc, q_h, g, t4);
       stream_units<3, 5120, 1>(pp, n, lane,
           [&](int u, int) { return stream + static_cast<long long>(first + u * kWarps) * 5120; },
-          [&](const uint8_t* tile, int) { process_qtile<4, G4>(tile, st, qc, qb, c_qscore, c_bias, lane); }, my_ring);
+          [&](const uint8_t* tile, int) { process_qunit<4, 1, G4>(tile, st, qc, qb, lc, lane); }, my_ring);
       phase_scale<4>(st, false);
     }
     dealt += rg.hi[1] - rg.lo[1];
@@ -603,7 +730,7 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
       load_q_phase<8>(qb, qc, q_h, g, t4);
       stream_units<2, 9216, 1>(pp, n, lane,
           [&](int u, int) { return stream + static_cast<long long>(first + u * kWarps) * 9216; },
-          [&](const uint8_t* tile, int) { process_qtile<8, G4>(tile, st, qc, qb, c_qscore, c_bias, lane); }, my_ring);
+          [&](const uint8_t* tile, int) { process_qunit<8, 1, G4>(tile, st, qc, qb, lc, lane); }, my_ring);
       phase_scale<8>(st, false);
     }
     dealt += rg.hi[2] - rg.lo[2];
@@ -616,11 +743,13 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
     const int n = first < rg.hi[3] ? (rg.hi[3] - first + kWarps - 1) / kWarps : 0;
     if (n > 0) {
       const uint8_t* stream = slot_ptr(cv, dm, 3, layer, b, h, 0);
+      phase_scale<16>(st, true);
       stream_units<2, 8192, 2>(pp, 2 * n, lane,
           [&](int u, int piece) {
             return stream + static_cast<long long>(first + (u >> 1) * kWarps) * kRawTileBytes + piece * 8192 + (u & 1) * 4096;
           },
           [&](const uint8_t* stg, int) { process_raw16<BF16>(stg, stg + 4096, 16, st, qr, c_bias, lane); }, my_ring);
+      phase_scale<16>(st, false);
     }
   }
   // ---- 16-bit tail (last split, warp 0): rows are staged by hand, swizzled, zero padded
@@ -628,6 +757,7 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
     const int len = cv.tail_len[layer * dm.batch + b];
     const long long tbase = ((static_cast<long long>(layer) * dm.batch + b) * dm.n_kv_heads + h) * dm.tail_capacity * kHeadDim;
     uint8_t* stg = rings;    // warp 0's ring; all its bulk copies have completed
+    phase_scale<16>(st, true);
     for (int t0 = 0; t0 < len; t0 += 16) {
       const int nv = min(16, len - t0);
       __syncwarp();
@@ -645,8 +775,9 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
       __syncwarp();
       process_raw16<BF16>(stg, stg + 4096, nv, st, qr, c_bias, lane);
     }
+    phase_scale<16>(st, false);
   }
-  if (!pp.ok && lane == 0) set_status(cv.status, MOQAE_ERR_TIMEOUT, blockIdx.x, warp);
+  const bool timed_out = !pp.ok;
 
   // ---- merge: lanes -> warp -> CTA -> split partial
   __syncthreads();                       // every warp is done with its ring
@@ -668,6 +799,11 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
     red_ml[(warp * 8 + 2 * t4 + 1) * 2] = st.m[1]; red_ml[(warp * 8 + 2 * t4 + 1) * 2 + 1] = st.oz[1];
   }
   __syncthreads();
+  // Everything up to here only read the caller's inputs and worked in registers and shared memory.
+  // Workspace and output are shared with the previous kernel on the stream when this launch was
+  // allowed to overlap it: wait for that kernel to complete (returns at once otherwise).
+  asm volatile("griddepcontrol.wait;\n" ::: "memory");
+  if (timed_out && lane == 0) set_status(cv.status, MOQAE_ERR_TIMEOUT, blockIdx.x, warp);
   for (int i = threadIdx.x; i < G * kHeadDim; i += kThreads) {
     const int qi = i / kHeadDim, c = i % kHeadDim;
     float m = -INFINITY;
@@ -691,7 +827,11 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
   __shared__ int s_last;
   __threadfence();                       // this CTA's partials are visible device-wide ...
   __syncthreads();
-  if (threadIdx.x == 0) s_last = (atomicAdd(&arrived[b * dm.n_kv_heads + h], 1) == n_splits - 1) ? 1 : 0;
+  // atomicInc wraps: the arrival that finds n_splits - 1 is the last one and leaves the counter at 0
+  // for the next launch, so no launch has to clear it
+  if (threadIdx.x == 0)
+    s_last = (atomicInc(reinterpret_cast<unsigned int*>(&arrived[b * dm.n_kv_heads + h]), static_cast<unsigned int>(n_splits - 1)) ==
+              static_cast<unsigned int>(n_splits - 1)) ? 1 : 0;
   __syncthreads();                       // ... before its arrival is counted
   if (!s_last) return;
   __threadfence();
@@ -717,15 +857,28 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
 int decode_mma_ctas_per_sm() { return 2; }
 
 cudaError_t launch_decode_mma(const Dims& dm, const CacheView& cv, const void* q, int layer, float scale,
-                              float* ws_o, float* ws_ml, int* arrived, float* out, int n_splits, cudaStream_t st) {
+                              float* ws_o, float* ws_ml, int* arrived, float* out, int n_splits, bool overlap_previous,
+                              cudaStream_t st) {
   const size_t smem = static_cast<size_t>(kWarps) * kRingBytes + 2 * kQBytes + kWarps * 6 * 8;
-  dim3 grid(n_splits, dm.n_kv_heads, dm.batch);
   const bool g4 = dm.n_q_heads / dm.n_kv_heads <= 4;
   auto launch = [&](auto kernel) -> cudaError_t {
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return e;
-    kernel<<<grid, kThreads, smem, st>>>(dm, cv, static_cast<const uint16_t*>(q), layer, scale, ws_o, ws_ml, arrived, out, n_splits);
-    return cudaSuccess;
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3(n_splits, dm.n_kv_heads, dm.batch);
+    lc.blockDim = dim3(kThreads, 1, 1);
+    lc.dynamicSmemBytes = smem;
+    lc.stream = st;
+    // programmatic dependent launch: this grid's CTAs may become resident as soon as every CTA of
+    // the previous kernel on the stream has started and SM slots free up; the kernel itself waits
+    // for that kernel's completion (griddepcontrol.wait) before its first global write
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = overlap_previous ? 1 : 0;
+    return cudaLaunchKernelEx(&lc, kernel, dm, cv, static_cast<const uint16_t*>(q), layer, scale, ws_o, ws_ml, arrived, out,
+                              n_splits);
   };
   cudaError_t e;
   if (dm.dtype == MOQAE_DTYPE_BF16) e = g4 ? launch(decode_mma_kernel<true, true>) : launch(decode_mma_kernel<true, false>);

@@ -65,6 +65,17 @@ int moqae_decode_attn_static(const moqae_config* cfg, const void* q, int32_t lay
     moqae::record_cuda_error(e);
     return MOQAE_ERR_CUDA;
   }
+  // The array is shared by every configuration that is ever used on this device, so the place
+  // where this one keeps its arrival counters may hold another one's partials: clear it here
+  // (moqae_decode_attn itself relies on the caller having zeroed its workspace once).
+  long long off = 0, len = 0;
+  moqae::decode_counter_region(cfg, &off, &len);
+  e = cudaMemsetAsync(static_cast<unsigned char*>(scratch) + off, 0, static_cast<size_t>(len),
+                      static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) {
+    moqae::record_cuda_error(e);
+    return MOQAE_ERR_CUDA;
+  }
   // Same kernels, same argument checks; only the home of the partials differs.
   return moqae_decode_attn(cfg, q, layer, cache, out, scale, scratch, moqae::kStaticScratchBytes, stream);
 }

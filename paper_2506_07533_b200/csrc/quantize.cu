@@ -511,15 +511,7 @@ __global__ void flush_reset_kernel(Dims dm, CacheView cv, int group) {
     cv.tail_len[l * dm.batch + b] = 0;
 }
 
-int sm_count() {
-  static int sms = 0;
-  if (sms == 0) {
-    int dev = 0, v = 148;
-    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev);
-    sms = v > 0 ? v : 148;
-  }
-  return sms;
-}
+int sm_count() { return sm_count_of_current_device(); }
 
 }  // namespace
 

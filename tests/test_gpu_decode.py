@@ -26,7 +26,7 @@ def decode_case(B, T, Hq, Hkv, chunk, dtype, bmap, seed, from_oracle_cache, q_sc
     else:
         fm = torch.from_numpy(bmap).cuda() if bmap.size else None
         mq.moqae_quantize_kv(cfg, K.cuda(), V.cuda(), T, layer, cache, forced_map=fm)
-    ws = torch.empty(mq.moqae_decode_attn_workspace(cfg), dtype=torch.uint8, device="cuda")
+    ws = torch.zeros(mq.moqae_decode_attn_workspace(cfg), dtype=torch.uint8, device="cuda")
     out = torch.full((B, Hq, 128), float("nan"), dtype=torch.float32, device="cuda")
     mq.moqae_decode_attn(cfg, q.cuda(), layer, cache, out, ws)
     torch.cuda.synchronize()
@@ -73,11 +73,92 @@ def test_edge_cases():
     decode_case(1, 256, 2, 2, 64, 0, np.array([[0, 0, 0, 0]], np.uint8), 84, False, q_scale=4.0)  # peaky softmax
 
 
+def test_overlapped_chain_of_layers_matches_oracle():
+    # decode calls over consecutive layers, each allowed to start while the previous one finishes
+    # (MOQAE_DECODE_OVERLAP_PREVIOUS): the shared workspace and the outputs must come out as in
+    # separate, serialised calls, several times over
+    B, T, Hq, Hkv, chunk, dtype, L = 2, 64 * 7 + 13, 8, 2, 64, 1, 4
+    cfg = mq.make_config(n_layers=L, n_q_heads=Hq, n_kv_heads=Hkv, chunk=chunk, dtype=dtype, d_in=64,
+                         max_tokens=T, batch=B)
+    cache = mq.moqae_cache_bind(cfg, [7, 7, 7, 7], zero_pools=True)
+    refs, qs = [], []
+    for l in range(L):
+        K, V = H.make_kv(B, T, Hkv, dtype, 300 + l)
+        bmap = np.random.RandomState(300 + l).randint(0, 4, size=(B, T // chunk)).astype(np.uint8)
+        mq.moqae_quantize_kv(cfg, K.cuda(), V.cuda(), T, l, cache, forced_map=torch.from_numpy(bmap).cuda())
+        q = synth.normal((B, Hq, 128), dtype, 400 + l, "cpu")
+        ocache = O.quantize_kv(synth.to_u16(K), synth.to_u16(V), dtype, chunk, bmap)
+        refs.append(O.decode_attn(synth.to_u16(q), dtype, ocache, chunk))
+        qs.append(q.cuda())
+    torch.cuda.synchronize()
+    ws = torch.zeros(mq.moqae_decode_attn_workspace(cfg), dtype=torch.uint8, device="cuda")
+    out = torch.full((L, B, Hq, 128), float("nan"), dtype=torch.float32, device="cuda")
+    for rep in range(3):
+        for l in range(L):
+            flags = mq.DECODE_OVERLAP_PREVIOUS if (l > 0 or rep > 0) else 0
+            mq.moqae_decode_attn_ex(cfg, qs[l], l, cache, out[l], ws, flags=flags)
+    torch.cuda.synchronize()
+    for l in range(L):
+        ok, e_abs, e_rel = H.attn_tolerance_ok(out[l].cpu().numpy(), refs[l])
+        assert ok, (l, e_abs, e_rel)
+    assert mq.moqae_poll_status(cache) == 0
+    with pytest.raises(mq.MoqaeError) as e:
+        mq.moqae_decode_attn_ex(cfg, qs[0], 0, cache, out[0], ws, flags=2)
+    assert e.value.code == mq.ERR_INVALID_ARG
+
+
+def scaled_case(bits_index, kv_range, q_abs, dtype, seed):
+    """Uniform-width cache whose K/V groups span about `kv_range` and queries of magnitude about
+    `q_abs`: the products q * s_k and p * s_v reach far beyond what N(0,1) inputs produce."""
+    B, T, Hq, Hkv, chunk = 1, 128 * 3 + 5, 4, 2, 128
+    rs = np.random.RandomState(seed)
+    tdt = synth.torch_dtype(dtype)
+    K = torch.from_numpy(rs.uniform(-0.5, 0.5, size=(B, T, Hkv, 128)).astype(np.float32) * kv_range).to(tdt)
+    V = torch.from_numpy(rs.uniform(-0.5, 0.5, size=(B, T, Hkv, 128)).astype(np.float32) * kv_range).to(tdt)
+    q = torch.from_numpy(rs.choice([-1.0, 1.0], size=(B, Hq, 128)).astype(np.float32) * q_abs *
+                         rs.uniform(0.5, 1.0, size=(B, Hq, 128)).astype(np.float32)).to(tdt)
+    bmap = np.full((B, T // chunk), bits_index, np.uint8)
+    ocache = O.quantize_kv(synth.to_u16(K), synth.to_u16(V), dtype, chunk, bmap)
+    # a softmax scale that keeps the logits of such inputs in a range where several tokens matter
+    scale = 4.0 / (q_abs * kv_range * np.sqrt(128.0))
+    ref = O.decode_attn(synth.to_u16(q), dtype, ocache, chunk, scale=scale)
+    cfg = mq.make_config(n_layers=1, n_q_heads=Hq, n_kv_heads=Hkv, chunk=chunk, dtype=dtype, d_in=64,
+                         max_tokens=T, batch=B)
+    cache = mq.moqae_cache_bind(cfg, [3, 3, 3, 3], zero_pools=True)
+    H.upload_oracle_cache(cache, ocache, 0)
+    ws = torch.zeros(mq.moqae_decode_attn_workspace(cfg), dtype=torch.uint8, device="cuda")
+    out = torch.full((B, Hq, 128), float("nan"), dtype=torch.float32, device="cuda")
+    mq.moqae_decode_attn(cfg, q.cuda(), 0, cache, out, ws, scale=scale)
+    torch.cuda.synchronize()
+    got = out.cpu().numpy()
+    assert np.isfinite(got).all()
+    # outputs are of the order of kv_range: the tolerances scale with it
+    err = np.abs(got - ref)
+    assert err.max() <= 2e-3 * max(1.0, kv_range), (err.max(), kv_range)
+    assert (err.max(-1) / np.abs(ref).max(-1)).max() <= 1e-2
+
+
+@pytest.mark.parametrize("w", [0, 1, 2])
+@pytest.mark.parametrize("kv_range", [1e3, 8e3, 3e4])
+def test_large_group_ranges_and_queries_stay_finite_and_accurate(w, kv_range):
+    # group ranges of thousands at 2 bits give key / value scales of thousands: the folded query
+    # q * s_k and the scaled weight p * s_v must not leave the fp16 range
+    scaled_case(w, kv_range, 8.0, 0, 500 + w)
+    scaled_case(w, kv_range, 8.0, 1, 510 + w)
+
+
+def test_tiny_and_huge_queries():
+    scaled_case(0, 4.0, 1e-3, 0, 520)
+    scaled_case(1, 4.0, 3e4, 0, 521)
+    scaled_case(0, 2e4, 6e4, 0, 522)
+    scaled_case(2, 4.0, 1e6, 1, 523)
+
+
 def test_empty_cache_gives_zeros():
     cfg = mq.make_config(n_layers=1, n_q_heads=2, n_kv_heads=2, chunk=32, dtype=0, d_in=64,
                          max_tokens=32, batch=1)
     cache = mq.moqae_cache_bind(cfg, [1, 1, 1, 1])
-    ws = torch.empty(mq.moqae_decode_attn_workspace(cfg), dtype=torch.uint8, device="cuda")
+    ws = torch.zeros(mq.moqae_decode_attn_workspace(cfg), dtype=torch.uint8, device="cuda")
     out = torch.full((1, 2, 128), float("nan"), dtype=torch.float32, device="cuda")
     q = synth.normal((1, 2, 128), 0, 1, "cuda")
     mq.moqae_decode_attn(cfg, q, 0, cache, out, ws)
@@ -96,7 +177,7 @@ def test_append_then_decode_matches_oracle_with_longer_tail():
     Kc, Vc = K.cuda(), V.cuda()
     mq.moqae_quantize_kv(cfg, Kc[:, :T].contiguous(), Vc[:, :T].contiguous(), T, 0, cache,
                          forced_map=torch.from_numpy(bmap).cuda())
-    ws = torch.empty(mq.moqae_decode_attn_workspace(cfg), dtype=torch.uint8, device="cuda")
+    ws = torch.zeros(mq.moqae_decode_attn_workspace(cfg), dtype=torch.uint8, device="cuda")
     out = torch.empty((B, Hq, 128), dtype=torch.float32, device="cuda")
     for step in range(5):
         mq.moqae_append_kv(cfg, Kc[:, T + step].contiguous(), Vc[:, T + step].contiguous(), 0, cache)
@@ -121,14 +202,18 @@ def test_decode_is_deterministic_and_leaves_neighbours_alone():
                          max_tokens=T, batch=B)
     cache = mq.moqae_cache_bind(cfg, [5, 5, 5, 5], zero_pools=True)
     mq.moqae_quantize_kv(cfg, K.cuda(), V.cuda(), T, 0, cache, forced_map=torch.from_numpy(bmap).cuda())
-    ws = torch.empty(mq.moqae_decode_attn_workspace(cfg), dtype=torch.uint8, device="cuda")
+    ws = torch.zeros(mq.moqae_decode_attn_workspace(cfg), dtype=torch.uint8, device="cuda")
     q = synth.normal((B, Hq, 128), dtype, 96, "cuda")
     n = B * Hq * 128
     buf = torch.full((n + 64,), -7.25, dtype=torch.float32, device="cuda")      # 32 canary floats on either side
     out = buf[32:32 + n].view(B, Hq, 128)
     mq.moqae_decode_attn(cfg, q, 0, cache, out, ws)
     first = out.clone()
-    ws.fill_(0xAB)                                                                # stale scratch must not matter
+    # stale partials must not matter; the arrival counters behind them (one int32 per sequence and
+    # kv head) are the only part a call relies on, and every call leaves them zero again
+    n_partial_bytes = ws.numel() - (B * Hkv * 4 + 15) // 16 * 16
+    ws[:n_partial_bytes].fill_(0xAB)
+    assert (ws[n_partial_bytes:] == 0).all()
     mq.moqae_decode_attn(cfg, q, 0, cache, out, ws)
     torch.cuda.synchronize()
     assert torch.equal(first, out)

@@ -84,7 +84,7 @@ def test_flush_adds_one_routed_chunk(dtype, gated):
         assert (cache.slot[g, :, :C].cpu().numpy() == slot).all()
         assert (cache.count[g].cpu().numpy() == count).all()
     # packed bytes of every layer equal the oracle's on the full context with the GPU's map
-    ws = torch.empty(mq.moqae_decode_attn_workspace(cfg), dtype=torch.uint8, device="cuda")
+    ws = torch.zeros(mq.moqae_decode_attn_workspace(cfg), dtype=torch.uint8, device="cuda")
     for l in range(L):
         K, V = KV[l]
         gmap = cache.map[l // rs, :, :C].cpu().numpy()

@@ -44,7 +44,7 @@ def job():
     # width is present whatever the untrained synthetic router prefers
     forced = torch.from_numpy(synth.multinomial_map(B, C, wl.mix, 77)).to(dev)
     mq.moqae_quantize_kv(cfg, K, V, T, 0, cache, forced_map=forced)
-    ws = torch.empty(mq.moqae_decode_attn_workspace(cfg), dtype=torch.uint8, device=dev)
+    ws = torch.zeros(mq.moqae_decode_attn_workspace(cfg), dtype=torch.uint8, device=dev)
     out = torch.full((B, Hq, 128), float("nan"), dtype=torch.float32, device=dev)
     mq.moqae_decode_attn(cfg, q, 0, cache, out, ws)
     torch.cuda.synchronize()

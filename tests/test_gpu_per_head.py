@@ -34,7 +34,7 @@ def test_per_head_routing_as_head_major_batch():
     cache = mq.moqae_cache_bind(cfg, [C, C, C, C], zero_pools=True)
     mq.moqae_route(cfg, hidden.cuda(), T, W1.cuda(), W2.cuda(), W3.cuda(), bias.cuda(), 0, cache)
     mq.moqae_quantize_kv(cfg, Kh.cuda(), Vh.cuda(), T, 0, cache)
-    ws = torch.empty(mq.moqae_decode_attn_workspace(cfg), dtype=torch.uint8, device="cuda")
+    ws = torch.zeros(mq.moqae_decode_attn_workspace(cfg), dtype=torch.uint8, device="cuda")
     out = torch.full((B * Hkv, G, 128), float("nan"), dtype=torch.float32, device="cuda")
     mq.moqae_decode_attn(cfg, q.cuda(), 0, cache, out, ws)
     torch.cuda.synchronize()

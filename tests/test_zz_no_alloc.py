@@ -33,7 +33,7 @@ def _setup(B, T, Hq, Hkv, chunk, dtype, seed):
 def test_static_scratch_matches_workspace_entry_point_twice():
     cfg, cache = _setup(B=2, T=64 * 7 + 13, Hq=8, Hkv=2, chunk=64, dtype=1, seed=321)
     assert mq.moqae_decode_attn_workspace(cfg) <= mq.moqae_decode_attn_static_max_bytes()
-    ws = torch.empty(mq.moqae_decode_attn_workspace(cfg), dtype=torch.uint8, device="cuda")
+    ws = torch.zeros(mq.moqae_decode_attn_workspace(cfg), dtype=torch.uint8, device="cuda")
     for call in range(2):                       # second call finds the first call's partials in the array
         q = synth.normal((2, 8, 128), 1, 500 + call, "cuda")
         want = torch.full((2, 8, 128), float("nan"), dtype=torch.float32, device="cuda")
