@@ -162,33 +162,21 @@ def reachable_winners(votes_row: np.ndarray, fragile_tokens_experts, fragile_alt
     """Winners a chunk can reach when each fragile token may flip to its runner-up.
 
     votes_row [M]; fragile_tokens_experts / fragile_alt: lists of the current and
-    the runner-up expert of each fragile token.  Exhaustive for few tokens,
-    otherwise a conservative superset (any expert whose best-case count can reach
-    the best-case-for-others maximum).
+    the runner-up expert of each fragile token.  Exact for any number of tokens:
+    the set of reachable vote vectors is grown token by token (a token either keeps
+    its expert or moves its vote to the runner-up), and every vector's winner under
+    the tie rule of Eq. 2 (first maximum) is collected.
     """
-    M = len(votes_row)
-    nf = len(fragile_tokens_experts)
-    winners = set()
-    if nf <= 12:
-        for mask in range(1 << nf):
-            v = votes_row.astype(np.int64).copy()
-            for i in range(nf):
-                if mask >> i & 1:
-                    v[fragile_tokens_experts[i]] -= 1
-                    v[fragile_alt[i]] += 1
-            winners.add(int(np.argmax(v)))
-        return winners
-    gain = np.zeros(M, dtype=np.int64)
-    loss = np.zeros(M, dtype=np.int64)
+    states = {tuple(int(v) for v in votes_row)}
     for cur, alt in zip(fragile_tokens_experts, fragile_alt):
-        loss[cur] += 1
-        gain[alt] += 1
-    for k in range(M):
-        best_k = votes_row[k] + gain[k]
-        others = [votes_row[j] - loss[j] for j in range(M) if j != k]
-        if best_k >= max(others):
-            winners.add(k)
-    return winners
+        moved = set()
+        for v in states:
+            w = list(v)
+            w[cur] -= 1
+            w[alt] += 1
+            moved.add(tuple(w))
+        states |= moved
+    return {int(np.argmax(np.asarray(v))) for v in states}
 
 
 def layer_group(layer: int, rs_group: int) -> int:

@@ -194,84 +194,16 @@ def _random_tile(rs, bits):
 
 @pytest.mark.parametrize("bits", BITS)
 def test_pack_layout_seen_from_the_consuming_lanes(bits):
-    """Independent statement of the format: read a packed tile the way the 32 lanes of the
-    decode kernel do (16-byte units per lane, registers = a word, or the word shifted right by
-    8, masked at one code position in both half-words) and find every code and every scale /
-    zero where the tensor-core fragments need it.  Nothing here uses the oracle's location
-    functions."""
+    """Independent statement of the format (tests/lane_reader.py): reading a packed tile the way
+    the 32 lanes of the decode kernel do finds every code and every scale / zero where the
+    tensor-core fragments need it.  The reader uses none of the oracle's location functions."""
+    from tests.lane_reader import read_tile_as_lanes
     rs = RS(100 + bits)
     t = _random_tile(rs, bits)
-    blob = O.pack_tile(t, bits)
-    n = 32 // bits
-    mask = (1 << bits) - 1
-    hw = blob[:1024].view(np.uint16)
-    kpay = blob[1024:1024 + 512 * bits]
-    vpay = blob[1024 + 512 * bits:]
-
-    def unit(pay, idx):
-        return pay[16 * idx:16 * idx + 16].view(np.uint32)
-
-    for blk in range(2):
-        for g in range(8):
-            for t4 in range(4):
-                lane = 4 * g + t4
-                # ---- key rows 16blk+g (hh = 0) and 16blk+g+8 (hh = 1), channels 32*t4 .. +31
-                for hh in range(2):
-                    tok = 16 * blk + 8 * hh + g
-                    if bits == 2:
-                        words = unit(kpay, 32 * blk + lane)[2 * hh:2 * hh + 2]
-                    elif bits == 4:
-                        words = unit(kpay, 32 * (2 * blk + hh) + lane)
-                    else:
-                        words = np.concatenate([unit(kpay, 32 * (2 * (2 * blk + hh) + j) + lane) for j in range(2)])
-                    assert len(words) == bits
-                    r = 0
-                    for j in range(bits):
-                        for s_ in range(2):
-                            ws = int(words[j]) >> (8 * s_)
-                            for m in range(n // 4):
-                                lo_ch = 32 * t4 + j * n + s_ * (n // 4) + m
-                                hi_ch = lo_ch + n // 2
-                                assert (ws >> (bits * m)) & mask == t["k_codes"][tok, lo_ch]
-                                assert (ws >> (16 + bits * m)) & mask == t["k_codes"][tok, hi_ch]
-                                if blk == 0 and hh == 0 and g == 0:
-                                    # register r of this lane: its scale / zero pair
-                                    # scales: the lane's i-th 16-byte unit holds registers 4i .. 4i+3;
-                                    # zeros: the same unit holds them in the order 4i, 4i+2, 4i+1, 4i+3
-                                    unit_hw = ((r >> 2) * 4 + t4) * 8
-                                    spos, zpos = (r & 3), (0, 2, 1, 3)[r & 3]
-                                    assert hw[unit_hw + 2 * spos] == t["k_scale"][lo_ch].view(np.uint16)
-                                    assert hw[unit_hw + 2 * spos + 1] == t["k_scale"][hi_ch].view(np.uint16)
-                                    assert hw[128 + unit_hw + 2 * zpos] == t["k_zero"][lo_ch].view(np.uint16)
-                                    assert hw[128 + unit_hw + 2 * zpos + 1] == t["k_zero"][hi_ch].view(np.uint16)
-                                r += 1
-                    assert r == 16
-                # ---- values: channel rows of this lane, tokens 16blk + 8half + 2t4 + e
-                words = np.concatenate([unit(vpay, (blk * (bits // 2) + u) * 32 + lane) for u in range(bits // 2)])
-                assert len(words) == 2 * bits
-                for w in range(2 * bits):
-                    for slot in range(8 // bits):
-                        R = w * (8 // bits) + slot
-                        ch = 32 * (R >> 2) + 4 * g + (R & 3)
-                        for half in range(2):
-                            ws = int(words[w]) >> (8 * half)
-                            for e in range(2):
-                                tok = 16 * blk + 8 * half + 2 * t4 + e
-                                assert (ws >> (bits * slot + 16 * e)) & mask == t["v_codes"][tok, ch]
-                if g == 0:
-                    for cp in range(2):
-                        base = ((blk * 2 + cp) * 4 + t4) * 8
-                        for k in range(4):
-                            cg, half = 2 * cp + (k >> 1), k & 1
-                            for e in range(2):
-                                tok = 16 * blk + 8 * half + 2 * t4 + e
-                                assert hw[256 + base + 2 * k + e] == t["v_scale"][cg, tok].view(np.uint16)
-                if g < 4:
-                    base = ((blk * 4 + g) * 4 + t4) * 4
-                    for half in range(2):
-                        for e in range(2):
-                            tok = 16 * blk + 8 * half + 2 * t4 + e
-                            assert hw[384 + base + 2 * half + e] == t["v_zero"][g, tok].view(np.uint16)
+    got = read_tile_as_lanes(O.pack_tile(t, bits), bits)
+    for k in t:
+        assert (got[k].view(np.uint16 if got[k].dtype == np.float16 else np.uint8) ==
+                t[k].view(np.uint16 if t[k].dtype == np.float16 else np.uint8)).all(), k
 
 
 @pytest.mark.parametrize("bits", BITS)

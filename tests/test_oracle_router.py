@@ -128,6 +128,28 @@ def test_reachable_winners():
     assert O.reachable_winners(np.array([9, 1, 0, 0]), [0], [1]) == {0}
 
 
+@pytest.mark.parametrize("nf", [1, 5, 12, 13, 16])
+def test_reachable_winners_against_enumeration_of_every_flip_pattern(nf):
+    # brute force written out here: try all 2^nf subsets of flipped tokens (also beyond a dozen
+    # tokens, where an earlier version of the function fell back to a superset)
+    rs = RS(40 + nf)
+    for trial in range(6):
+        votes = rs.randint(0, 6, size=4) + np.array([nf, 0, 0, 0]) // 2
+        cur = [int(x) for x in rs.randint(0, 4, size=nf)]
+        alt = [int((c + rs.randint(1, 4)) % 4) for c in cur]
+        for c in cur:
+            votes[c] += 1                       # every fragile token's current vote is in the histogram
+        want = set()
+        for mask in range(1 << nf):
+            v = votes.astype(np.int64).copy()
+            for i in range(nf):
+                if mask >> i & 1:
+                    v[cur[i]] -= 1
+                    v[alt[i]] += 1
+            want.add(int(np.argmax(v)))
+        assert O.reachable_winners(votes, cur, alt) == want
+
+
 def _embed_three_experts(W1, W2, W3, bias):
     """A {2, 4, 16}-bit router written as the four-expert one: the 8-bit expert gets zero weights
     and a logit no token can choose."""
