@@ -58,6 +58,50 @@ def compare_pools(cache, ocache, layer):
         assert (cache.tail("v")[layer, :, :, :r].cpu().numpy().view(np.uint16) == ocache["tail_v"]).all()
 
 
+TAU = 1e-4      # a token whose top-2 logits differ by less than TAU * max|P| may flip in float32
+
+
+def check_routed_chunk(rows_u16, dtype, W1_u16, W2_u16, W3, bias, got_votes, got_winner, abs_margin=None):
+    """One chunk's vote histogram and winner from the GPU against the oracle router run on the
+    chunk's hidden rows [chunk, d_in]: exact unless near-tie tokens exist; then the histograms may
+    differ by at most those tokens and the winner must be reachable by flipping them between
+    their two best experts.  Returns True if the chunk was fragile."""
+    chunk = rows_u16.shape[0]
+    ref = O.route(rows_u16[None], dtype, chunk, W1_u16, W2_u16, W3, bias, rf_first_chunk=False)
+    thr = abs_margin if abs_margin is not None else TAU * np.maximum(ref["pmax"][0], 1e-30)
+    frag = np.where(ref["margin"][0] < thr)[0]
+    diff = np.asarray(got_votes).astype(np.int64) - ref["votes"][0, 0]
+    assert diff.sum() == 0 and np.abs(diff).sum() // 2 <= len(frag), (diff, len(frag))
+    if len(frag) == 0:
+        assert (diff == 0).all() and int(got_winner) == int(ref["map"][0, 0])
+        return False
+    x = O.to_f64(rows_u16[frag], dtype)
+    P = O.router_logits(x, O.to_f64(W1_u16, dtype), None if W2_u16 is None else O.to_f64(W2_u16, dtype),
+                        None if W3 is None else np.asarray(W3, np.float32).astype(np.float64),
+                        None if bias is None else np.asarray(bias, np.float32).astype(np.float64))
+    order = np.argsort(-P, axis=1, kind="stable")
+    assert int(got_winner) in O.reachable_winners(ref["votes"][0, 0], list(order[:, 0]), list(order[:, 1]))
+    return True
+
+
+def oracle_cache_of_head(cache, layer, b, h, C):
+    """The GPU's own packed cache of one (layer, sequence, kv head), in the form the oracle's
+    decode functions take (one sequence, one head): its bytes, its map-derived tables, its tail."""
+    g = layer // cache.cfg.rs_group
+    gmap = cache.map[g, b:b + 1, :C].cpu().numpy()
+    slot, count = O.assign_slots(gmap)
+    assert (cache.slot[g, b:b + 1, :C].cpu().numpy() == slot).all()
+    assert (cache.count[g, b:b + 1].cpu().numpy() == count).all()
+    pools = []
+    for w in range(4):
+        n = int(count[0, w])
+        pools.append(cache.pool(w)[layer, b, h, :max(n, 1)].cpu().numpy()[None, None])
+    r = int(cache.tail_len[layer, b].item())
+    return dict(pools=pools, map=gmap, slot=slot, count=count, tail_len=r,
+                tail_k=cache.tail("k")[layer, b, h, :r].cpu().numpy().view(np.uint16)[None, None],
+                tail_v=cache.tail("v")[layer, b, h, :r].cpu().numpy().view(np.uint16)[None, None])
+
+
 def attn_tolerance_ok(got, ref, abs_tol=2e-3, rel_tol=1e-2):
     """max-abs error <= abs_tol and, per (batch, head) row, max|err| / max|ref| <= rel_tol."""
     err = np.abs(got.astype(np.float64) - ref)

@@ -61,15 +61,12 @@ def test_router_sampled_chunks(job):
     rs = np.random.RandomState(5)
     picks = [(b, c) for b in range(wl.batch) for c in rs.choice(np.arange(1, C), 6, replace=False)]
     picks += [(0, 1), (wl.batch - 1, C - 1)]
+    n_fragile = 0
     for b, c in picks:
-        rows = job["hidden"][b, c * wl.chunk:(c + 1) * wl.chunk].unsqueeze(0)
-        ref = O.route(synth.to_u16(rows), wl.dtype, wl.chunk, w1, w2, W3.cpu().numpy(), bias.cpu().numpy(),
-                      rf_first_chunk=False)
-        frag = np.where(ref["margin"][0] < TAU * np.maximum(ref["pmax"][0], 1e-30))[0]
-        diff = gvotes[b, c].astype(np.int64) - ref["votes"][0, 0]
-        assert diff.sum() == 0 and np.abs(diff).sum() // 2 <= len(frag), (b, c, diff, len(frag))
-        if len(frag) == 0:
-            assert gmap[b, c] == ref["map"][0, 0]
+        rows = job["hidden"][b, c * wl.chunk:(c + 1) * wl.chunk]
+        n_fragile += H.check_routed_chunk(synth.to_u16(rows), wl.dtype, w1, w2, W3.cpu().numpy(), bias.cpu().numpy(),
+                                          gvotes[b, c], gmap[b, c])
+    assert n_fragile <= len(picks) // 2
     slot, count = O.assign_slots(gmap)
     assert (job["routed"]["slot"] == slot).all() and (job["routed"]["count"] == count).all()
 
