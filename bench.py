@@ -77,25 +77,36 @@ class ClockSampler:
             self.p = None
 
     def stop(self):
+        """Ends the sampling; returns the summary of the begin()..end() window."""
+        if self.p is not None:
+            self.p.terminate()
+            try:
+                self.p.wait(timeout=5)
+            except Exception:
+                self.p.kill()
+            self.f.flush()
+            self.f.seek(0)
+            self.lines = self.f.read().splitlines()
+            try:
+                os.unlink(self.f.name)
+            except OSError:
+                pass
+        return self.summary(self.t_begin, self.t_end)
+
+    def summary(self, t_begin, t_end):
+        """Median SM clock and the throttle reasons seen between two host time stamps."""
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.p is None:
             return out
-        self.p.terminate()
-        try:
-            self.p.wait(timeout=5)
-        except Exception:
-            self.p.kill()
-        self.f.flush()
-        self.f.seek(0)
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for line in self.f.read().splitlines():
+        for line in getattr(self, "lines", []):
             parts = [x.strip() for x in line.split(",")]
             if len(parts) < 9:
                 continue
             try:
                 when = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f")
-                if self.t_begin and self.t_end and not (self.t_begin <= when <= self.t_end):
+                if t_begin and t_end and not (t_begin <= when <= t_end):
                     continue
                 sm.append(float(parts[1]))
                 mx.append(float(parts[2]))
@@ -104,10 +115,6 @@ class ClockSampler:
             for n, v in zip(names, parts[5:9]):
                 if v.lower().startswith("active"):
                     reasons.add(n)
-        try:
-            os.unlink(self.f.name)
-        except OSError:
-            pass
         if sm:
             out = {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)),
                    "reasons": sorted(reasons), "samples": len(sm)}
@@ -276,6 +283,38 @@ def whole_job_gbs(bytes_per_rank, ms, world):
     return world * bytes_per_rank / (ms * 1e6)
 
 
+def free_port() -> int:
+    import socket
+    with socket.socket(socket.AF_INET, socket.SOCK_STREAM) as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def spawn_command(n_ranks: int, argv: list) -> list:
+    """Command line that runs this script as `n_ranks` ranks on this node (one per GPU)."""
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n_ranks}",
+            "--master-addr", "127.0.0.1", "--master-port", str(free_port()), os.path.abspath(__file__), *argv]
+
+
+def run_rendezvous_check(args):
+    """The multi-rank skeleton of run_ours without a GPU: process group (gloo), barrier, the
+    maximum over ranks of stub timings, one JSON line from rank 0."""
+    import torch
+    import torch.distributed as dist
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1:
+        dist.init_process_group("gloo")
+        dist.barrier()
+    ms = max_over_ranks([10.0 + rank], torch.device("cpu"), world)[0]
+    if rank == 0:
+        print(json.dumps({"rendezvous_check": True, "n_gpus": world, "requested_gpus": args.gpus,
+                          "ms_max_over_ranks": ms, "value": whole_job_gbs(1e9, ms, world)}), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -347,20 +386,29 @@ def run_ours(args):
     sampler.end()
     if world > 1:
         dist.barrier()
-    clocks = sampler.stop()
     total_ms = t0.elapsed_time(t1)
     ms_route = sum(e[0].elapsed_time(e[1]) for e in events) / args.steps
     ms_quant = sum(e[1].elapsed_time(e[2]) for e in events) / args.steps
     ms_dec = sum(e[2].elapsed_time(e[3]) for e in events) / args.steps
 
-    # end to end: inputs start in pinned host memory, result read back, every step
+    # end to end, right after the timed steps (same power state): the decode calls with the
+    # queries coming from and the outputs going to pinned host memory, then the whole step with
+    # every input on the host
+    t_e2e0 = datetime.datetime.now()
     if args.e2e_steps > 0:
+        e2e_dec = measure_e2e_decode(job, max(5, args.e2e_steps), torch)
+    else:
+        e2e_dec = {"ms": float("nan"), "h2d": 0, "d2h": 0, "steps": 0}
+    t_e2e1 = datetime.datetime.now()
+    clocks = sampler.stop()
+    clocks_e2e = sampler.summary(t_e2e0, t_e2e1)
+    if args.e2e_step_steps > 0:
         e2e = measure_e2e(job, args, torch)
     else:
         e2e = {"ms_dec": float("nan"), "ms_step": float("nan"), "h2d": 0, "d2h": 0, "steps": 0}
 
     total_ms, ms_route, ms_quant, ms_dec, e2e_ms_dec, e2e_ms_step = max_over_ranks(
-        [total_ms, ms_route, ms_quant, ms_dec, e2e["ms_dec"], e2e["ms_step"]], device, world)
+        [total_ms, ms_route, ms_quant, ms_dec, e2e_dec["ms"], e2e["ms_step"]], device, world)
 
     if rank == 0:
         peak, peak_kind = read_peaks()
@@ -406,10 +454,17 @@ def run_ours(args):
                                 "unit": "GB/s", "frac": round(b_route / (ms_route * 1e6) / peak, 4)}
                                if b_route else None),
             "e2e": {"value": round(world * b_dec / (e2e_ms_dec * 1e6), 1), "unit": "GB/s",
-                    "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
-                    "ms_per_step": round(e2e_ms_step, 3), "steps": e2e["steps"],
-                    "note": "host-resident hidden, K, V, q copied in and out read back inside the timed step; "
-                            "value = decode-phase bytes / (decode phase incl. q upload and out download)"},
+                    "h2d_bytes_per_step": e2e_dec["h2d"], "d2h_bytes_per_step": e2e_dec["d2h"],
+                    "ms_per_step": round(e2e_ms_dec, 4), "steps": e2e_dec["steps"], "clocks": clocks_e2e,
+                    "note": "the metric through the library's calls with host buffers: per step the queries of all "
+                            "layers are copied from pinned host memory, the decode calls run, out is read back; "
+                            "value = decode bytes of the step / that time"},
+            "e2e_step": {"value": round(world * (b_route + b_quant + b_dec) / (e2e_ms_step * 1e6), 1), "unit": "GB/s",
+                         "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
+                         "ms_per_step": round(e2e_ms_step, 3), "steps": e2e["steps"],
+                         "note": "whole step (route + quantise+pack + decode) with hidden states, K, V and q copied "
+                                 "from pinned host memory every step and out read back: bound by the host link; "
+                                 "value = algorithmic bytes of the whole step / that time"},
         }
         if world == 1 and not args.no_prefill_attn:
             # a second kernel family (tensor-bound) reported beside the headline, never part of it
@@ -463,9 +518,41 @@ def measure_prefill_attn(job, torch, reps=3):
             "peak_source": src, "flops": flops, "status": job.mq.moqae_poll_status(job.cache)}
 
 
+def measure_e2e_decode(job, steps, torch):
+    """The metric end to end through the library's calls with HOST buffers: every step copies the
+    queries of all layers from pinned host memory, runs the decode calls and reads `out` back; the
+    timed region holds exactly these copies.  Returns ms per step and the bytes copied."""
+    h_q = job.q.cpu().pin_memory()
+    h_out = torch.empty(job.out.shape, dtype=torch.float32).pin_memory()
+    d_q = torch.empty_like(job.q)
+    new_tok = []
+    if job.wl.decode_steps > 1:                      # the generated tokens' K/V rows also start on the host
+        new_tok = [(job.k_new, job.k_new.cpu().pin_memory()), (job.v_new, job.v_new.cpu().pin_memory())]
+    h2d = h_q.numel() * 2 + sum(h.numel() * 2 for _, h in new_tok)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    saved = job.q
+    job.q = d_q
+    try:
+        for s in range(steps + 2):                   # two warm-up passes
+            if s == 2:
+                ev[0].record()
+            d_q.copy_(h_q, non_blocking=True)
+            for d_t, h_t in new_tok:
+                d_t.copy_(h_t, non_blocking=True)
+            job.decode_all()
+            h_out.copy_(job.out, non_blocking=True)
+        ev[1].record()
+        torch.cuda.synchronize()
+    finally:
+        job.q = saved
+    return {"ms": ev[0].elapsed_time(ev[1]) / steps, "h2d": int(h2d), "d2h": int(h_out.numel() * 4), "steps": steps}
+
+
 def measure_e2e(job, args, torch):
+    """The whole step (route + quantise+pack + decode) with hidden states, K, V and q starting in
+    pinned host memory and `out` read back: PCIe-bound by construction."""
     wl = job.wl
-    steps = max(1, min(args.e2e_steps, args.steps))
+    steps = max(1, args.e2e_step_steps)
     h_kv = [(K.cpu().pin_memory(), V.cpu().pin_memory()) for K, V in job.kv]
     h_hidden = [h.cpu().pin_memory() for h in job.hidden]
     h_q = job.q.cpu().pin_memory()
@@ -617,7 +704,13 @@ def main():
                          "with this 2/4/8/16-bit mix (e.g. 1,0,0,0 = uniform 2-bit)")
     ap.add_argument("--no-overlap", action="store_true",
                     help="serialise the decode launches of consecutive layers (no programmatic dependent launch)")
-    ap.add_argument("--e2e-steps", type=int, default=1)
+    ap.add_argument("--e2e-steps", type=int, default=5,
+                    help="timed steps of the end-to-end decode measurement (0 skips it; at least 5 otherwise)")
+    ap.add_argument("--e2e-step-steps", type=int, default=1,
+                    help="timed whole steps with every input copied from the host (0 skips it)")
+    ap.add_argument("--rendezvous-check", action="store_true",
+                    help="only start the ranks, form the process group on CPU (gloo), exchange stub timings and "
+                         "print the line's multi-rank fields: checks the launch path on a box without GPUs")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--reference-tokens", type=int, default=32768)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -628,6 +721,12 @@ def main():
         args.warmup = 3
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started as plain `python bench.py --gpus N`: start the N ranks ourselves, one per GPU
+        sys.exit(subprocess.call(spawn_command(args.gpus, sys.argv[1:])))
+    if args.rendezvous_check:
+        run_rendezvous_check(args)
     else:
         run_ours(args)
 

@@ -45,3 +45,29 @@ def test_single_rank_and_throughput():
     assert bench.max_over_ranks([3.0, 4.0], torch.device("cpu"), 1) == [3.0, 4.0]
     # 4 replicas, 2 GB each, slowest takes 1 ms -> 8 GB / ms = 8000 GB/s
     assert abs(bench.whole_job_gbs(2e9, 1.0, 4) - 8000.0) < 1e-9
+
+
+def test_plain_gpus_2_starts_two_ranks_that_meet():
+    """`python bench.py --gpus 2` with no rank variables in the environment starts its two ranks
+    itself; with --rendezvous-check they form the process group on CPU, reduce stub timings with the
+    same max-over-ranks code as the real run and rank 0 prints one line."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--rendezvous-check"],
+                       capture_output=True, text=True, timeout=300, env=env, cwd=ROOT)
+    assert p.returncode == 0, p.stderr[-2000:]
+    lines = [l for l in p.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1                              # rank 0 alone prints
+    line = json.loads(lines[0])
+    assert line["n_gpus"] == 2 and line["requested_gpus"] == 2
+    assert line["ms_max_over_ranks"] == 11.0            # the slower rank's time
+    assert abs(line["value"] - 2 * 1e9 / (11.0 * 1e6)) < 1e-9
+
+
+def test_spawn_command_is_one_rank_per_gpu_on_localhost():
+    import bench
+    cmd = bench.spawn_command(4, ["--gpus", "4", "--steps", "2"])
+    assert "--nproc-per-node=4" in cmd and "--nnodes=1" in cmd
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1"
+    assert cmd[-4:] == ["--gpus", "4", "--steps", "2"]

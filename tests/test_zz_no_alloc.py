@@ -12,6 +12,8 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import moqae_oracle as O
+
 from paper_2506_07533_b200 import binding as mq
 from paper_2506_07533_b200 import synth
 from tests import helpers as H
@@ -27,6 +29,7 @@ def _setup(B, T, Hq, Hkv, chunk, dtype, seed):
     cap = [T // chunk] * 4
     cache = mq.moqae_cache_bind(cfg, cap, zero_pools=True)
     mq.moqae_quantize_kv(cfg, K.cuda(), V.cuda(), T, 0, cache, forced_map=torch.from_numpy(bmap).cuda())
+    cache.oracle = O.quantize_kv(synth.to_u16(K), synth.to_u16(V), dtype, chunk, bmap)
     return cfg, cache
 
 
@@ -43,7 +46,26 @@ def test_static_scratch_matches_workspace_entry_point_twice():
         torch.cuda.synchronize()
         ok, e_abs, e_rel = H.attn_tolerance_ok(got.cpu().numpy(), want.cpu().numpy().astype(np.float64))
         assert ok, (call, e_abs, e_rel)
+        ref = O.decode_attn(synth.to_u16(q), 1, cache.oracle, 64)          # and against the CPU oracle
+        ok, e_abs, e_rel = H.attn_tolerance_ok(got.cpu().numpy(), ref)
+        assert ok, (call, e_abs, e_rel)
     assert mq.moqae_poll_status(cache) == 0
+
+
+def test_static_scratch_is_shared_by_different_configurations():
+    # The one array serves every configuration used on the device, and each lays its partials and
+    # arrival counters out differently: where a small problem keeps its counters, a larger one
+    # writes partials.  Alternating between two problems must still give each its right answer.
+    small = _setup(B=1, T=32 * 5, Hq=2, Hkv=2, chunk=32, dtype=0, seed=331)
+    large = _setup(B=3, T=64 * 6 + 5, Hq=8, Hkv=4, chunk=64, dtype=1, seed=332)
+    for rnd in range(3):
+        for (cfg, cache), (B, Hq, chunk, dtype) in ((small, (1, 2, 32, 0)), (large, (3, 8, 64, 1))):
+            q = synth.normal((B, Hq, 128), dtype, 600 + rnd, "cuda")
+            got = torch.full((B, Hq, 128), float("nan"), dtype=torch.float32, device="cuda")
+            mq.moqae_decode_attn_static(cfg, q, 0, cache, got)
+            torch.cuda.synchronize()
+            ok, e_abs, e_rel = H.attn_tolerance_ok(got.cpu().numpy(), O.decode_attn(synth.to_u16(q), dtype, cache.oracle, chunk))
+            assert ok, (rnd, B, e_abs, e_rel)
 
 
 def test_static_scratch_rejects_oversized_problem():
