@@ -185,6 +185,25 @@ int moqae_quantize_kv(const moqae_config* cfg, const void* K, const void* V, int
                       void* stream);
 
 /*
+ * The K and V projections of one layer fused with moqae_quantize_kv (Section 3.1: the chunks are
+ * quantised with the configuration the router has just determined, then the block goes on with
+ * its computation): K = hidden Wk^T and V = hidden Wv^T are computed on the tensor cores, rounded
+ * to the input dtype exactly as a separate projection would have stored them, and quantised and
+ * packed from the accumulators; the 16-bit K/V rows never exist in device memory.
+ *   hidden [batch][T][d_in] input dtype (the block's hidden states, the router's input);
+ *   Wk, Wv [n_kv_heads * 128][d_in] input dtype, row-major (one row per output channel);
+ *   products accumulate in float32 in an unspecified order; d_in must be a multiple of 64.
+ *   forced_map, chunk placement, the tail and POOL_FULL reporting are those of
+ *   moqae_quantize_kv applied to the rounded K and V.
+ *   k_rounded, v_rounded: both NULL, or [batch][T][n_kv_heads][128] input-dtype buffers that
+ *   receive the rounded rows as well (for checking; costs the traffic the fusion saves).
+ */
+int moqae_project_quantize_kv(const moqae_config* cfg, const void* hidden, const void* Wk,
+                              const void* Wv, int32_t T, int32_t layer, const uint8_t* forced_map,
+                              const moqae_cache* cache, void* k_rounded, void* v_rounded,
+                              void* stream);
+
+/*
  * Append one decoded token per sequence to the 16-bit tail of `layer` (tokens that do not
  * fill a chunk stay 16-bit, Section 3.2).  k_new, v_new [batch][n_kv_heads][128].  A full
  * tail sets status[0] = MOQAE_ERR_POOL_FULL and drops the token.

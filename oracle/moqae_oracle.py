@@ -601,6 +601,34 @@ def decode_attn(q_u16: np.ndarray, dtype: int, cache: dict, chunk: int, scale=No
     return out
 
 
+def round_to_16bit(x64: np.ndarray, dtype: int) -> np.ndarray:
+    """float64 -> bit patterns (uint16) of the nearest fp16 / bf16 value, ties to even, in ONE
+    rounding: the value is divided by the spacing of the target format at its magnitude (a power
+    of two, so the division is exact), rounded to an integer with rint, and multiplied back."""
+    x64 = np.asarray(x64, dtype=np.float64)
+    sig, emin = (11, -14) if dtype == DT_FP16 else (8, -126)          # significant bits, smallest normal exponent
+    _, e = np.frexp(x64)                                              # |x| = m * 2^e, m in [0.5, 1)
+    quantum = np.ldexp(1.0, np.maximum(e, emin + 1) - sig)
+    y = np.rint(x64 / quantum) * quantum                              # exactly representable in the target format
+    if dtype == DT_FP16:
+        return y.astype(np.float16).view(np.uint16)
+    return (y.astype(np.float32).view(np.uint32) >> 16).astype(np.uint16)
+
+
+def project_kv(hidden_u16: np.ndarray, Wk_u16: np.ndarray, Wv_u16: np.ndarray, dtype: int, n_kv_heads: int):
+    """The key / value projections that feed the quantiser (Section 3.1: the chunks a block
+    quantises are its own keys and values): K = hidden Wk^T, V = hidden Wv^T from the exact
+    values of the 16-bit inputs in float64, then one rounding to the 16-bit dtype.
+    hidden [B, T, D]; Wk, Wv [H_kv * 128, D] -> K_u16, V_u16 [B, T, H_kv, 128]."""
+    x = to_f64(hidden_u16, dtype)
+    B, T, _ = x.shape
+    K64 = x @ to_f64(Wk_u16, dtype).T
+    V64 = x @ to_f64(Wv_u16, dtype).T
+    shape = (B, T, n_kv_heads, HEAD_DIM)
+    return (round_to_16bit(K64, dtype).reshape(shape), round_to_16bit(V64, dtype).reshape(shape),
+            K64.reshape(shape), V64.reshape(shape))
+
+
 def cache_bytes(count: np.ndarray, chunk: int, n_kv_heads: int, tail_len: int) -> int:
     """Closed form of the bytes a cache holds: sum_w count_w * slot_bytes_w per head,
     plus 512 bytes per tail token per head."""

@@ -26,7 +26,7 @@ EXPORTS = ["moqae_version", "moqae_last_cuda_error", "moqae_error_string", "moqa
            "moqae_cache_bind", "moqae_route", "moqae_quantize_kv", "moqae_append_kv",
            "moqae_decode_attn_workspace", "moqae_decode_attn", "moqae_poll_status",
            "moqae_decode_attn_static", "moqae_decode_attn_static_max_bytes", "moqae_flush_tail", "moqae_prefill_attn",
-           "moqae_prefill_attn_workspace", "moqae_decode_attn_ex"]
+           "moqae_prefill_attn_workspace", "moqae_decode_attn_ex", "moqae_project_quantize_kv"]
 
 
 class MoqaeConfig(C.Structure):
@@ -81,6 +81,9 @@ def lib() -> C.CDLL:
                                   C.c_void_p]
         L.moqae_quantize_kv.argtypes = [C.POINTER(MoqaeConfig), C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
                                         C.c_void_p, C.POINTER(MoqaeCache), C.c_void_p]
+        L.moqae_project_quantize_kv.argtypes = [C.POINTER(MoqaeConfig), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
+                                                C.c_int32, C.c_void_p, C.POINTER(MoqaeCache), C.c_void_p, C.c_void_p,
+                                                C.c_void_p]
         L.moqae_append_kv.argtypes = [C.POINTER(MoqaeConfig), C.c_void_p, C.c_void_p, C.c_int32,
                                       C.POINTER(MoqaeCache), C.c_void_p]
         L.moqae_flush_tail.argtypes = [C.POINTER(MoqaeConfig), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
@@ -223,6 +226,12 @@ def moqae_route(cfg, hidden, T, W1, W2, W3, bias, layer_group, cache: Cache, vot
 def moqae_quantize_kv(cfg, K, V, T, layer, cache: Cache, forced_map=None):
     _check(lib().moqae_quantize_kv(C.byref(cfg), _ptr(K), _ptr(V), int(T), int(layer), _ptr(forced_map),
                                    C.byref(cache.view), _stream()), "moqae_quantize_kv")
+
+
+def moqae_project_quantize_kv(cfg, hidden, Wk, Wv, T, layer, cache: Cache, forced_map=None, k_rounded=None, v_rounded=None):
+    _check(lib().moqae_project_quantize_kv(C.byref(cfg), _ptr(hidden), _ptr(Wk), _ptr(Wv), int(T), int(layer),
+                                           _ptr(forced_map), C.byref(cache.view), _ptr(k_rounded), _ptr(v_rounded),
+                                           _stream()), "moqae_project_quantize_kv")
 
 
 def moqae_append_kv(cfg, k_new, v_new, layer, cache: Cache):

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmoqae.so")
-SOURCES = ["api.cu", "route.cu", "quantize.cu", "decode.cu", "decode_mma.cu", "decode_static.cu", "prefill.cu"]
+SOURCES = ["api.cu", "route.cu", "quantize.cu", "decode.cu", "decode_mma.cu", "decode_static.cu", "prefill.cu", "project.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--expt-relaxed-constexpr"]
 

@@ -200,6 +200,32 @@ int moqae_quantize_kv(const moqae_config* cfg, const void* K, const void* V, int
   return e == cudaSuccess ? MOQAE_OK : cuda_fail(e);
 }
 
+int moqae_project_quantize_kv(const moqae_config* cfg, const void* hidden, const void* Wk, const void* Wv, int32_t T,
+                              int32_t layer, const uint8_t* forced_map, const moqae_cache* cache, void* k_rounded,
+                              void* v_rounded, void* stream) {
+  int rc = check_config(cfg);
+  if (rc != MOQAE_OK) return rc;
+  moqae::CacheView cv;
+  rc = check_cache(cache, &cv);
+  if (rc != MOQAE_OK) return rc;
+  if (T < 0 || T > cfg->max_tokens || layer < 0 || layer >= cfg->n_layers) return MOQAE_ERR_INVALID_ARG;
+  if (T > 0 && (!hidden || !Wk || !Wv)) return MOQAE_ERR_INVALID_ARG;
+  if ((k_rounded == nullptr) != (v_rounded == nullptr)) return MOQAE_ERR_INVALID_ARG;
+  if (cfg->d_in % 64 != 0) return MOQAE_ERR_UNSUPPORTED;
+  if (!aligned16(hidden) || !aligned16(Wk) || !aligned16(Wv) || !aligned16(k_rounded) || !aligned16(v_rounded))
+    return MOQAE_ERR_MISALIGNED;
+  if (T % cfg->chunk > cfg->tail_capacity) return MOQAE_ERR_POOL_FULL;
+  if (cfg->tail_capacity > 0 && (!cache->tail_k || !cache->tail_v)) return MOQAE_ERR_INVALID_ARG;
+  const moqae::Dims dm = dims_of(cfg);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (forced_map) {
+    cudaError_t e = moqae::launch_finalize_map(dm, cv, layer / cfg->rs_group, T / cfg->chunk, forced_map, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+  }
+  cudaError_t e = moqae::launch_project_quantize(dm, cv, hidden, Wk, Wv, T, layer, k_rounded, v_rounded, st);
+  return e == cudaSuccess ? MOQAE_OK : cuda_fail(e);
+}
+
 int moqae_append_kv(const moqae_config* cfg, const void* k_new, const void* v_new, int32_t layer,
                     const moqae_cache* cache, void* stream) {
   int rc = check_config(cfg);

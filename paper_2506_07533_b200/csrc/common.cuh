@@ -82,6 +82,8 @@ cudaError_t launch_quantize(const Dims& dm, const CacheView& cv, const void* K, 
                             int layer, cudaStream_t st);
 cudaError_t launch_append(const Dims& dm, const CacheView& cv, const void* k_new, const void* v_new,
                           int layer, cudaStream_t st);
+cudaError_t launch_project_quantize(const Dims& dm, const CacheView& cv, const void* hidden, const void* Wk, const void* Wv,
+                                    int T, int layer, void* dbg_k, void* dbg_v, cudaStream_t st);
 int decode_num_splits(const Dims& dm);
 int decode_mma_ctas_per_sm();
 cudaError_t launch_prefill_attn(const Dims& dm, const CacheView& cv, const void* q, int T, int layer, float scale,

@@ -28,7 +28,7 @@
 // the cache's status word and stops consuming.
 #include <cuda_bf16.h>
 
-#include "common.cuh"
+#include "ptx.cuh"
 
 namespace moqae {
 
@@ -38,40 +38,6 @@ constexpr int kWarps = 6;
 constexpr int kThreads = kWarps * 32;
 constexpr int kRingBytes = 18432;             // per warp: 6 x 3 KiB = 3 x 5 KiB(+) = 2 x 9 KiB = 2 x 8 KiB(+)
 constexpr int kQBytes = 8 * kHeadDim * 2;     // one 8-query fragment source, 16-bit
-constexpr long long kWaitCycles = 1ll << 30;  // a bounded wait gives up after this many SM cycles
-constexpr uint32_t kSuspendNs = 20000;         // how long one try_wait may keep the warp parked
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, int count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n"
-               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-// One try_wait with a suspend-time hint: the hardware parks the warp until the phase completes
-// or the hint runs out, so a waiting warp takes no issue slots from the working ones.
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\nselp.u32 %0, 1, 0, p;\n}\n"
-               : "=r"(ok) : "r"(bar), "r"(parity), "r"(kSuspendNs) : "memory");
-  return ok != 0;
-}
-// Bounded by elapsed SM cycles (about half a second), not by the number of attempts.
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, long long limit = kWaitCycles) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const long long t0 = clock64();
-  do {
-    if (mbar_try_wait(bar, parity)) return true;
-  } while (clock64() - t0 < limit);
-  return false;
-}
-
 template <bool BF16>
 __device__ __forceinline__ void mma16816(float d[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                          uint32_t b0, uint32_t b1) {

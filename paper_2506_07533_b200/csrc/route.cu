@@ -13,10 +13,9 @@
 //
 // finalize_map_kernel: per sequence, chunk winner (first maximum), routing freezing,
 // per-width counts and slot = rank among earlier chunks of the same width.
-#include <cuda.h>
 #include <cuda_bf16.h>
 
-#include "common.cuh"
+#include "ptx.cuh"
 
 namespace moqae {
 
@@ -29,39 +28,6 @@ constexpr int kBoxBytes = 16 * 128;  // 16 token rows
 constexpr int kBoxesPerStage = 4;
 constexpr int kStageBytes = kBoxesPerStage * kBoxBytes;
 constexpr int kStages = 2;
-constexpr long long kWaitCycles = 1ll << 30;  // a bounded wait gives up after this many SM cycles
-constexpr uint32_t kSuspendNs = 20000;         // how long one try_wait may keep the warp parked
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, int count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
-  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];\n"
-               ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
-}
-// One try_wait with a suspend-time hint: the hardware parks the warp until the phase completes
-// or the hint runs out, so a waiting warp takes no issue slots from the working ones.
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\nselp.u32 %0, 1, 0, p;\n}\n"
-               : "=r"(ok) : "r"(bar), "r"(parity), "r"(kSuspendNs) : "memory");
-  return ok != 0;
-}
-// Bounded by elapsed SM cycles (about half a second), not by the number of attempts.
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const long long t0 = clock64();
-  do {
-    if (mbar_try_wait(bar, parity)) return true;
-  } while (clock64() - t0 < kWaitCycles);
-  return false;
-}
 __device__ __forceinline__ void ldmatrix_x4(uint32_t (&a)[4], uint32_t addr) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
                : "=r"(a[0]), "=r"(a[1]), "=r"(a[2]), "=r"(a[3]) : "r"(addr));
@@ -338,22 +304,6 @@ __global__ void flush_finalize_kernel(Dims dm, CacheView cv, int group) {
 }
 
 }  // namespace
-
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn encode_tiled_fn() {
-  static EncodeTiledFn fn = [] {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
-        qres != cudaDriverEntryPointSuccess)
-      p = nullptr;
-    return reinterpret_cast<EncodeTiledFn>(p);
-  }();
-  return fn;
-}
 
 // Launch the scoring + voting kernel over hidden [batch][T][d_in]: chunks first..C-1 of every sequence.
 static cudaError_t launch_score_vote(const Dims& dm, const CacheView& cv, const void* hidden, int T, int first,
