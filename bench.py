@@ -472,12 +472,57 @@ def run_ours(args):
                 line["prefill_attn"] = measure_prefill_attn(job, torch)
             except Exception as exc:                      # the headline line must not depend on it
                 line["prefill_attn"] = {"error": f"{type(exc).__name__}: {exc}"}
+        if world == 1 and not args.no_project and job.hidden and wl.d_in % 64 == 0:
+            try:
+                line["project_quantize"] = measure_project_quantize(job, torch)
+            except Exception as exc:
+                line["project_quantize"] = {"error": f"{type(exc).__name__}: {exc}"}
         if not args.no_cpu_baseline and world == 1:
             line["cpu_baseline"] = cpu_baseline(wl, budget_s=args.cpu_seconds)
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
+
+
+def measure_project_quantize(job, torch, reps=3):
+    """K/V projection fused with quantise+pack (layer 0, the workload's hidden states as the block
+    input, random weights): device time of `reps` launches after one warm-up.  Tensor-bound:
+    FLOPs = 2 * tokens * d_in * 2 * n_kv_heads * 128; the HBM side (hidden states read once per
+    unit row + packed bytes written) is reported beside it."""
+    wl, T = job.wl, job.T
+    from paper_2506_07533_b200 import synth
+    from paper_2506_07533_b200 import workloads as W
+    n_out = wl.n_kv_heads * 128
+    Wk = synth.normal((n_out, wl.d_in), wl.dtype, 4001, job.device, std=wl.d_in ** -0.5)
+    Wv = synth.normal((n_out, wl.d_in), wl.dtype, 4002, job.device, std=wl.d_in ** -0.5)
+    hidden = job.hidden[0]
+    job.mq.moqae_project_quantize_kv(job.cfg, hidden, Wk, Wv, T, 0, job.cache)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    ev[0].record()
+    for _ in range(reps):
+        job.mq.moqae_project_quantize_kv(job.cfg, hidden, Wk, Wv, T, 0, job.cache)
+    ev[1].record()
+    torch.cuda.synchronize()
+    ms = ev[0].elapsed_time(ev[1]) / reps
+    flops = 2.0 * wl.batch * T * wl.d_in * 2 * n_out
+    cnt = job.counts()
+    hbm = wl.batch * T * wl.d_in * 2 + 2 * n_out * wl.d_in * 2 + W.cache_bytes_per_layer(cnt[0], wl.chunk, wl.n_kv_heads, T % wl.chunk)
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            pk = json.load(f)
+        peak, sustained, src = float(pk["bf16_tflops"]), float(pk.get("bf16_tflops_sustained", 0.0)) or None, "of measured"
+    except Exception:
+        peak, sustained, src = 1590.0, 1400.0, "of fallback"
+    hbm_peak, _ = read_peaks()
+    tf = flops / (ms * 1e9)
+    return {"ms": round(ms, 3), "tflops": round(tf, 1), "bound": "tensor", "peak": peak, "frac": round(tf / peak, 4),
+            "peak_sustained": sustained, "frac_of_sustained": round(tf / sustained, 4) if sustained else None,
+            "peak_source": src, "flops": flops, "hbm_bytes": int(hbm), "hbm_gbs": round(hbm / (ms * 1e6), 1),
+            "hbm_frac": round(hbm / (ms * 1e6) / hbm_peak, 4),
+            "saved_bytes_vs_unfused": int(2 * 2 * wl.batch * T * n_out * 2),
+            "note": "the 16-bit K/V rows (written by a separate projection, read by quantise+pack) never exist",
+            "status": job.mq.moqae_poll_status(job.cache)}
 
 
 def measure_prefill_attn(job, torch, reps=3):
@@ -698,6 +743,7 @@ def main():
     ap.add_argument("--prefill-attn", action="store_true",
                     help="(default at one GPU; kept for old command lines) also time the causal prefill attention of layer 0 over its quantised cache")
     ap.add_argument("--no-prefill-attn", action="store_true", help="skip the prefill-attention measurement")
+    ap.add_argument("--no-project", action="store_true", help="skip the fused projection+quantise measurement")
     ap.add_argument("--no-rf", action="store_true", help="switch routing freezing off (chunk 0 is routed too)")
     ap.add_argument("--mix", default=None,
                     help="four comma-separated shares: skip the router and force a seeded multinomial map "
