@@ -208,7 +208,8 @@ def assign_slots(bmap: np.ndarray, n_experts: int = N_EXPERTS):
 # Quantiser (group-wise asymmetric min-max, group 32)
 # ----------------------------------------------------------------------------
 def quantize_groups(x32: np.ndarray, bits: int):
-    """Quantise along the LAST axis, which must have length 32 (one group).
+    """Quantise along the LAST axis (one group: 32 elements, or the 8 / 16 tokens of a
+    short chunk for key groups, see `quantize_tile`).
 
     Canonical sequence; "binary32" steps are single IEEE operations rounded to
     nearest even unless a direction is stated:
@@ -226,7 +227,7 @@ def quantize_groups(x32: np.ndarray, bits: int):
     Dequantised value (defined, not computed here): code * s + z.
     """
     x32 = np.asarray(x32, dtype=np.float32)
-    assert x32.shape[-1] == GROUP
+    assert 1 <= x32.shape[-1] <= GROUP        # key groups of chunks shorter than 32 tokens are shorter
     qmax = np.float32((1 << bits) - 1)
     mn = x32.min(axis=-1)
     mx = x32.max(axis=-1)
@@ -254,13 +255,34 @@ def quantize_tile(K32: np.ndarray, V32: np.ndarray, bits: int):
     Returns dict with k_scale/k_zero fp16 [128], k_codes uint8 [32,128],
     v_scale/v_zero fp16 [4, 32] ([channel group, token]), v_codes uint8 [32,128].
     """
-    assert K32.shape == (TILE_TOKENS, HEAD_DIM) and V32.shape == (TILE_TOKENS, HEAD_DIM)
-    ks, kz, kc = quantize_groups(K32.T, bits)                   # [128, 32] groups over tokens
-    vg = V32.reshape(TILE_TOKENS, HEAD_DIM // GROUP, GROUP)     # [32, 4, 32]
-    vs, vz, vc = quantize_groups(vg, bits)                      # vs [32, 4]
-    return dict(k_scale=ks, k_zero=kz, k_codes=np.ascontiguousarray(kc.T),
-                v_scale=np.ascontiguousarray(vs.T), v_zero=np.ascontiguousarray(vz.T),
-                v_codes=vc.reshape(TILE_TOKENS, HEAD_DIM))
+    n = K32.shape[0]
+    assert K32.shape == (n, HEAD_DIM) and V32.shape == (n, HEAD_DIM) and n in (8, 16, TILE_TOKENS)
+    ks, kz, kc = quantize_groups(K32.T, bits)                   # [128, n] groups over the tile's tokens
+    vg = V32.reshape(n, HEAD_DIM // GROUP, GROUP)               # [n, 4, 32]
+    vs, vz, vc = quantize_groups(vg, bits)                      # vs [n, 4]
+    t = dict(k_scale=ks, k_zero=kz, k_codes=np.ascontiguousarray(kc.T),
+             v_scale=np.ascontiguousarray(vs.T), v_zero=np.ascontiguousarray(vz.T),
+             v_codes=vc.reshape(n, HEAD_DIM))
+    if n < TILE_TOKENS:
+        # A chunk of 8 or 16 tokens (the small chunk sizes of the paper's chunk-size ablation) is
+        # one tile whose remaining token positions are padding: codes 0, value scale / zero 0.
+        # Its key groups are the chunk's own tokens of one channel ("per channel within the
+        # chunk" with fewer than 32 tokens to group).
+        pad = TILE_TOKENS - n
+        t["k_codes"] = np.concatenate([t["k_codes"], np.zeros((pad, HEAD_DIM), np.uint8)])
+        t["v_codes"] = np.concatenate([t["v_codes"], np.zeros((pad, HEAD_DIM), np.uint8)])
+        t["v_scale"] = np.concatenate([t["v_scale"], np.zeros((HEAD_DIM // GROUP, pad), np.float16)], axis=1)
+        t["v_zero"] = np.concatenate([t["v_zero"], np.zeros((HEAD_DIM // GROUP, pad), np.float16)], axis=1)
+    return t
+
+
+def tile_tokens(chunk: int) -> int:
+    """Token positions of a tile that hold tokens: 32, or the whole chunk if it is shorter."""
+    return min(chunk, TILE_TOKENS)
+
+
+def tiles_per_chunk(chunk: int) -> int:
+    return max(1, chunk // TILE_TOKENS)
 
 
 def dequantize_tile(t: dict):
@@ -292,7 +314,8 @@ def tile_bytes(bits: int) -> int:
 
 
 def slot_bytes(bits: int, chunk: int) -> int:
-    return (chunk // TILE_TOKENS) * tile_bytes(bits)
+    """A chunk of 32 j tokens is j tiles; a chunk of 8 or 16 tokens is one (padded) tile."""
+    return max(1, chunk // TILE_TOKENS) * tile_bytes(bits)
 
 
 def key_code_location(t: int, c: int, bits: int):
@@ -488,7 +511,7 @@ def quantize_kv(K_u16: np.ndarray, V_u16: np.ndarray, dtype: int, chunk: int,
     trailing T mod chunk tokens are kept as raw 16-bit rows (Section 3.2).
     """
     B, T, H, d = K_u16.shape
-    assert d == HEAD_DIM and chunk % TILE_TOKENS == 0
+    assert d == HEAD_DIM and (chunk % TILE_TOKENS == 0 or chunk in (8, 16))
     C = T // chunk
     assert bmap.shape == (B, C)
     slot, count = assign_slots(bmap)
@@ -496,7 +519,7 @@ def quantize_kv(K_u16: np.ndarray, V_u16: np.ndarray, dtype: int, chunk: int,
         capacity = [max(1, int(count[:, w].max())) for w in range(N_EXPERTS)]
     pools = [np.zeros((B, H, capacity[w], slot_bytes(EXPERT_BITS[w], chunk)), dtype=np.uint8)
              for w in range(N_EXPERTS)]
-    tpc = chunk // TILE_TOKENS
+    tpc, nt = tiles_per_chunk(chunk), tile_tokens(chunk)
     for b in range(B):
         for c in range(C):
             w = int(bmap[b, c])
@@ -505,9 +528,12 @@ def quantize_kv(K_u16: np.ndarray, V_u16: np.ndarray, dtype: int, chunk: int,
             for h in range(H):
                 for j in range(tpc):
                     t0 = c * chunk + j * TILE_TOKENS
-                    Kt = K_u16[b, t0:t0 + TILE_TOKENS, h]
-                    Vt = V_u16[b, t0:t0 + TILE_TOKENS, h]
+                    Kt = K_u16[b, t0:t0 + nt, h]
+                    Vt = V_u16[b, t0:t0 + nt, h]
                     if bits == 16:
+                        if nt < TILE_TOKENS:                   # short chunk: zero rows fill the tile
+                            zr = np.zeros((TILE_TOKENS - nt, HEAD_DIM), np.uint16)
+                            Kt, Vt = np.concatenate([Kt, zr]), np.concatenate([Vt, zr])
                         blob = pack_raw_tile(Kt, Vt)
                     else:
                         blob = pack_tile(quantize_tile(to_f32(Kt, dtype), to_f32(Vt, dtype), bits), bits)
@@ -547,7 +573,7 @@ def cache_kv_rows(cache: dict, dtype: int, chunk: int, b: int, h: int):
     """All cached rows of (sequence b, kv head h) as float64 K̂, V̂ [n, 128],
     pool by pool then the tail (softmax attention does not depend on key order)."""
     Ks, Vs = [], []
-    tpc = chunk // TILE_TOKENS
+    tpc, nt = tiles_per_chunk(chunk), tile_tokens(chunk)
     for w in range(N_EXPERTS):
         bits = EXPERT_BITS[w]
         tb = tile_bytes(bits)
@@ -557,12 +583,12 @@ def cache_kv_rows(cache: dict, dtype: int, chunk: int, b: int, h: int):
                 tile = blob[j * tb:(j + 1) * tb]
                 if bits == 16:
                     Ku, Vu = unpack_raw_tile(tile)
-                    Ks.append(to_f64(Ku, dtype))
-                    Vs.append(to_f64(Vu, dtype))
+                    Ks.append(to_f64(Ku[:nt], dtype))
+                    Vs.append(to_f64(Vu[:nt], dtype))
                 else:
                     Kh, Vh = dequantize_tile(unpack_tile(tile, bits))
-                    Ks.append(Kh)
-                    Vs.append(Vh)
+                    Ks.append(Kh[:nt])
+                    Vs.append(Vh[:nt])
     if cache["tail_len"] > 0:
         Ks.append(to_f64(cache["tail_k"][b, h, :cache["tail_len"]], dtype))
         Vs.append(to_f64(cache["tail_v"][b, h, :cache["tail_len"]], dtype))
@@ -647,7 +673,7 @@ def cache_kv_rows_in_order(cache: dict, dtype: int, chunk: int, b: int, h: int):
     """Cached rows of (sequence b, kv head h) in TOKEN order as float64 K̂, V̂ [T, 128]:
     chunk c comes from pool map[b, c], slot slot[b, c]; the tail follows."""
     Ks, Vs = [], []
-    tpc = chunk // TILE_TOKENS
+    tpc, nt = tiles_per_chunk(chunk), tile_tokens(chunk)
     C = cache["map"].shape[1]
     for c in range(C):
         w = int(cache["map"][b, c])
@@ -658,12 +684,12 @@ def cache_kv_rows_in_order(cache: dict, dtype: int, chunk: int, b: int, h: int):
             tile = blob[j * tb:(j + 1) * tb]
             if bits == 16:
                 Ku, Vu = unpack_raw_tile(tile)
-                Ks.append(to_f64(Ku, dtype))
-                Vs.append(to_f64(Vu, dtype))
+                Ks.append(to_f64(Ku[:nt], dtype))
+                Vs.append(to_f64(Vu[:nt], dtype))
             else:
                 Kh, Vh = dequantize_tile(unpack_tile(tile, bits))
-                Ks.append(Kh)
-                Vs.append(Vh)
+                Ks.append(Kh[:nt])
+                Vs.append(Vh[:nt])
     if cache["tail_len"] > 0:
         Ks.append(to_f64(cache["tail_k"][b, h, :cache["tail_len"]], dtype))
         Vs.append(to_f64(cache["tail_v"][b, h, :cache["tail_len"]], dtype))

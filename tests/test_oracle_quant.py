@@ -287,3 +287,78 @@ def test_mixed_map_places_chunks_in_pools():
     ref = O.quantize_tile(O.to_f32(K[0, 192:224, 0], 1), O.to_f32(V[0, 192:224, 0], 1), 2)
     for k in ref:
         assert (t[k] == ref[k]).all()
+
+
+# ---- chunks shorter than a tile (8 and 16 tokens, the small sizes of the chunk-size ablation) ----
+@pytest.mark.parametrize("chunk", [8, 16])
+@pytest.mark.parametrize("bits", BITS)
+def test_short_chunk_tile_groups_are_the_chunks_own_tokens(chunk, bits):
+    rs = RS(300 + chunk + bits)
+    K = (rs.randn(chunk, 128) * np.exp(rs.randn(1, 128))).astype(np.float16).astype(np.float32)
+    V = rs.randn(chunk, 128).astype(np.float16).astype(np.float32)
+    t = O.quantize_tile(K, V, bits)
+    assert t["k_codes"].shape == (32, 128) and t["v_scale"].shape == (4, 32)
+    # padding positions carry nothing
+    assert (t["k_codes"][chunk:] == 0).all() and (t["v_codes"][chunk:] == 0).all()
+    assert (t["v_scale"][:, chunk:] == 0).all() and (t["v_zero"][:, chunk:] == 0).all()
+    # the key group of a channel is its `chunk` tokens: zero = its minimum, and the s/2 bound holds
+    assert (t["k_zero"].astype(np.float32) == K.min(0)).all()
+    Kh, Vh = O.dequantize_tile(t)
+    assert (np.abs(Kh[:chunk] - K) <= t["k_scale"].astype(np.float64)[None, :] / 2 * (1 + 2e-7) + 1e-12).all()
+    vs = np.repeat(t["v_scale"].astype(np.float64).T[:chunk], 32, axis=1)
+    assert (np.abs(Vh[:chunk] - V) <= vs / 2 * (1 + 2e-7) + 1e-12).all()
+    # the group maximum reaches the top code (or one below), the minimum code 0
+    kc = t["k_codes"][:chunk]
+    nonconst = t["k_scale"] > 0
+    assert (kc.min(0) == 0).all() and (kc.max(0)[nonconst] >= (1 << bits) - 2).all()
+    # a value group is 32 channels of one token, exactly as in a full tile
+    full = O.quantize_tile(np.concatenate([K, K, K, K])[:32], np.concatenate([V, V, V, V])[:32], bits)
+    assert (full["v_codes"][:chunk] == t["v_codes"][:chunk]).all()
+    assert (full["v_scale"][:, :chunk] == t["v_scale"][:, :chunk]).all()
+    # pack / unpack keeps everything, padding included
+    u = O.unpack_tile(O.pack_tile(t, bits), bits)
+    for k in t:
+        assert (u[k] == t[k]).all(), k
+
+
+@pytest.mark.parametrize("chunk", [8, 16])
+def test_short_chunks_cache_sizes_rows_and_sixteen_bit_exactness(chunk):
+    K, V = _small_kv(T=chunk * 9 + 3, dtype=1)
+    B, T, H, _ = K.shape
+    C = T // chunk
+    bmap = RS(chunk).randint(0, 4, size=(B, C)).astype(np.uint8)
+    cache = O.quantize_kv(K, V, 1, chunk, bmap)
+    # one (padded) tile per chunk: slot bytes are those of a single tile
+    for w, bits in enumerate(O.EXPERT_BITS):
+        assert cache["pools"][w].shape[-1] == O.tile_bytes(bits) == O.slot_bytes(bits, chunk)
+    assert cache["tail_len"] == 3
+    for b in range(B):
+        for h in range(H):
+            Kh, Vh = O.cache_kv_rows_in_order(cache, 1, chunk, b, h)
+            assert Kh.shape == (T, 128)                       # padding positions are not tokens
+            for c in range(C):
+                sl = slice(c * chunk, (c + 1) * chunk)
+                if bmap[b, c] == 3:                           # 16-bit chunks are exact
+                    assert (Kh[sl] == O.to_f64(K[b, sl, h], 1)).all() and (Vh[sl] == O.to_f64(V[b, sl, h], 1)).all()
+                else:                                         # others within half a scale of the chunk's own range
+                    x = O.to_f64(K[b, sl, h], 1)
+                    rng = x.max(0) - x.min(0)
+                    bits = O.EXPERT_BITS[bmap[b, c]]
+                    assert (np.abs(Kh[sl] - x) <= rng[None, :] / ((1 << bits) - 1) / 2 * 1.01 + 1e-3 * np.abs(x).max()).all()
+            assert (Kh[C * chunk:] == O.to_f64(K[b, C * chunk:, h], 1)).all()
+            # the pool-by-pool walk sees the same multiset of rows
+            Kp, _ = O.cache_kv_rows(cache, 1, chunk, b, h)
+            assert Kp.shape == Kh.shape and np.allclose(np.sort(Kp.sum(1)), np.sort(Kh.sum(1)))
+
+
+def test_short_chunks_all_sixteen_bit_attention_equals_plain_attention():
+    K, V = _small_kv(T=8 * 11 + 5, dtype=0)
+    B, T, H, _ = K.shape
+    bmap = np.full((B, T // 8), 3, np.uint8)
+    cache = O.quantize_kv(K, V, 0, 8, bmap)
+    q = RS(3).randn(B, H, 128).astype(np.float16)
+    out = O.decode_attn(q.view(np.uint16), 0, cache, 8)
+    for b in range(B):
+        for h in range(H):
+            ref = O.softmax_attention(q[b, h].astype(np.float64), O.to_f64(K[b, :, h], 0), O.to_f64(V[b, :, h], 0), 1 / np.sqrt(128))
+            assert np.abs(out[b, h] - ref).max() < 1e-12
