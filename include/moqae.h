@@ -23,8 +23,10 @@
  *   - No C++ types or exceptions cross this boundary.
  *
  * Fixed by this build: head_dim = 128, quantisation group = 32, experts = 4 with bit widths
- * {2, 4, 8, 16} at expert indices {0, 1, 2, 3}, chunk a multiple of 32, 16 <= d_in and
- * d_in a multiple of 32, n_q_heads / n_kv_heads in {1, .., 8}.
+ * {2, 4, 8, 16} at expert indices {0, 1, 2, 3}, chunk a multiple of 32 or one of the short
+ * sizes 8 and 16, 32 <= d_in and d_in a multiple of 32, n_q_heads / n_kv_heads in {1, .., 8}.
+ * Error state: the code of the last failed CUDA runtime call is kept per host thread
+ * (moqae_last_cuda_error); nothing else outlives a call.
  *
  * Storage format of the cache (what moqae_quantize_kv writes and moqae_decode_attn reads)
  *   tile   = 32 consecutive tokens of one chunk and one kv head.
@@ -56,7 +58,11 @@
  *     Dequantised value = code * scale + zero.
  *   16-bit tile, 16384 bytes: 32 key rows then 32 value rows of 256 bytes in the input dtype;
  *     16-byte unit U of row t is stored at (U & 8) | ((U xor t) & 7).
- *   slot   = the chunk/32 tiles of one chunk and one kv head, in token order.
+ *   slot   = the chunk/32 tiles of one chunk and one kv head, in token order.  A chunk of 8 or 16
+ *     tokens is ONE tile: its tokens sit at token positions 0 .. chunk-1, the other positions are
+ *     padding (codes 0, value scale and zero 0, raw rows 0) that no kernel attends to, and its key
+ *     scale / zero of a channel are taken over the chunk's own tokens.  moqae_prefill_attn and
+ *     moqae_project_quantize_kv refuse such configurations (MOQAE_ERR_UNSUPPORTED).
  *   pool[w] = [n_layers][batch][n_kv_heads][capacity[w]] slots of width w.
  *   map/slot/count/votes tables are per routing-sharing group: [n_groups][batch][max_chunks]
  *     (count: [n_groups][batch][4], votes: [n_groups][batch][max_chunks][4]),

@@ -190,7 +190,7 @@ class Cache:
     def pool(self, w):
         """uint8 view [n_layers, batch, n_kv_heads, capacity_w, slot_bytes_w]."""
         tb = 16384 if w == 3 else 1024 + 1024 * EXPERT_BITS[w]
-        sb = (self.cfg.chunk // 32) * tb
+        sb = max(1, self.cfg.chunk // 32) * tb      # a chunk of 8 or 16 tokens is one (padded) tile
         n = self.cfg.n_layers * self.cfg.batch * self.cfg.n_kv_heads * self.capacity[w] * sb
         return self.buffers[w][:n].view(self.cfg.n_layers, self.cfg.batch, self.cfg.n_kv_heads,
                                         self.capacity[w], sb)

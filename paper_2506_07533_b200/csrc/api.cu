@@ -26,7 +26,7 @@ int check_config(const moqae_config* c) {
     return MOQAE_ERR_UNSUPPORTED;
   for (int w = 0; w < 4; ++w)
     if (c->expert_bits[w] != moqae::bits_of_expert(w)) return MOQAE_ERR_UNSUPPORTED;
-  if (c->chunk % moqae::kTileTokens != 0) return MOQAE_ERR_UNSUPPORTED;
+  if (c->chunk % moqae::kTileTokens != 0 && c->chunk != 8 && c->chunk != 16) return MOQAE_ERR_UNSUPPORTED;
   if (c->dtype != MOQAE_DTYPE_FP16 && c->dtype != MOQAE_DTYPE_BF16) return MOQAE_ERR_UNSUPPORTED;
   if (c->n_q_heads % c->n_kv_heads != 0) return MOQAE_ERR_INVALID_ARG;
   if (c->n_q_heads / c->n_kv_heads > moqae::kMaxQueryGroup) return MOQAE_ERR_UNSUPPORTED;
@@ -119,7 +119,7 @@ int moqae_cache_bytes(const moqae_config* cfg, const int64_t capacity[4], int64_
   if (rc != MOQAE_OK) return rc;
   if (!capacity || !out_bytes) return MOQAE_ERR_INVALID_ARG;
   const int64_t lbh = static_cast<int64_t>(cfg->n_layers) * cfg->batch * cfg->n_kv_heads;
-  const int64_t tpc = cfg->chunk / moqae::kTileTokens;
+  const int64_t tpc = moqae::tiles_per_chunk_of(cfg->chunk);
   for (int w = 0; w < 4; ++w) {
     if (capacity[w] < 0) return MOQAE_ERR_INVALID_ARG;
     out_bytes[w] = lbh * capacity[w] * tpc * moqae::tile_bytes_of_expert(w);
@@ -211,7 +211,7 @@ int moqae_project_quantize_kv(const moqae_config* cfg, const void* hidden, const
   if (T < 0 || T > cfg->max_tokens || layer < 0 || layer >= cfg->n_layers) return MOQAE_ERR_INVALID_ARG;
   if (T > 0 && (!hidden || !Wk || !Wv)) return MOQAE_ERR_INVALID_ARG;
   if ((k_rounded == nullptr) != (v_rounded == nullptr)) return MOQAE_ERR_INVALID_ARG;
-  if (cfg->d_in % 64 != 0) return MOQAE_ERR_UNSUPPORTED;
+  if (cfg->d_in % 64 != 0 || cfg->chunk < moqae::kTileTokens) return MOQAE_ERR_UNSUPPORTED;
   if (!aligned16(hidden) || !aligned16(Wk) || !aligned16(Wv) || !aligned16(k_rounded) || !aligned16(v_rounded))
     return MOQAE_ERR_MISALIGNED;
   if (T % cfg->chunk > cfg->tail_capacity) return MOQAE_ERR_POOL_FULL;
@@ -315,6 +315,7 @@ int moqae_prefill_attn(const moqae_config* cfg, const void* q, int32_t T, int32_
   rc = check_cache(cache, &cv);
   if (rc != MOQAE_OK) return rc;
   if (T < 0 || T > cfg->max_tokens || layer < 0 || layer >= cfg->n_layers) return MOQAE_ERR_INVALID_ARG;
+  if (cfg->chunk < moqae::kTileTokens) return MOQAE_ERR_UNSUPPORTED;     // walks the cache in whole 32-token tiles
   if (T > 0 && (!q || !out)) return MOQAE_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(out) || !aligned16(workspace)) return MOQAE_ERR_MISALIGNED;
   if (workspace && workspace_bytes < moqae::prefill_workspace_bytes(dims_of(cfg), T)) return MOQAE_ERR_WORKSPACE_TOO_SMALL;

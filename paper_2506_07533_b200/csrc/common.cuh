@@ -22,6 +22,11 @@ __host__ __device__ constexpr int tile_bytes_of_expert(int w) {
   return w == 3 ? kRawTileBytes : kMetaBytes + 1024 * (2 << w);
 }
 
+// A chunk of 32 j tokens is j tiles; a chunk of 8 or 16 tokens is one tile whose first `chunk`
+// token positions hold tokens (the rest is padding: codes 0, never attended).
+__host__ __device__ constexpr int tiles_per_chunk_of(int chunk) { return chunk >= kTileTokens ? chunk / kTileTokens : 1; }
+__host__ __device__ constexpr int tile_tokens_of(int chunk) { return chunk >= kTileTokens ? kTileTokens : chunk; }
+
 // Everything a kernel needs to find its way around a cache (passed by value).
 struct CacheView {
   uint8_t* pool[4];
@@ -56,7 +61,7 @@ __device__ __forceinline__ float load16_as_float(uint16_t u, int dtype) {
 // Address of slot `slot` of (layer, b, h) in pool w.
 __device__ __forceinline__ uint8_t* slot_ptr(const CacheView& cv, const Dims& dm, int w, int layer,
                                              int b, int h, long long slot) {
-  const long long slot_bytes = static_cast<long long>(dm.chunk / kTileTokens) * tile_bytes_of_expert(w);
+  const long long slot_bytes = static_cast<long long>(tiles_per_chunk_of(dm.chunk)) * tile_bytes_of_expert(w);
   const long long idx = ((static_cast<long long>(layer) * dm.batch + b) * dm.n_kv_heads + h) *
                             cv.capacity[w] + slot;
   return cv.pool[w] + idx * slot_bytes;

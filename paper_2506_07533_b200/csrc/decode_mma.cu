@@ -188,7 +188,7 @@ __device__ __forceinline__ void softmax_update(State& st, float x[NV][4]) {
 template <int BITS, int NT, bool G4>
 __device__ __forceinline__ void process_qunit(const uint8_t* __restrict__ unit, State& st,
                                               const uint32_t (&qc)[16], const uint32_t (&qb)[16],
-                                              const LaneConst& lc, int lane) {
+                                              const LaneConst& lc, int lane, int n_valid) {
   using F = Fmt<BITS>;
   constexpr int TB = kMetaBytes + 1024 * BITS;       // bytes per tile
   constexpr int NB = 2 * NT;                         // 16-token blocks
@@ -312,6 +312,16 @@ __device__ __forceinline__ void process_qunit(const uint8_t* __restrict__ unit, 
       if (G4) x += __shfl_xor_sync(0xffffffffu, x, 2);       // column c + column c ^ 4
       v[b2][i] = x;
     }
+  if (n_valid < kTileTokens) {
+    // tiles of a chunk shorter than 32 tokens: positions n_valid (8 or 16) .. 31 are padding and get
+    // weight zero (row g of block 0 is token g, row g + 8 token g + 8, block 1 tokens 16..31)
+#pragma unroll
+    for (int b2 = 0; b2 < NB; ++b2) {
+      const bool lo_ok = (b2 & 1) == 0, hi_ok = (b2 & 1) == 0 && n_valid > 8;
+      if (!lo_ok) v[b2][0] = v[b2][1] = -INFINITY;
+      if (!hi_ok) v[b2][2] = v[b2][3] = -INFINITY;
+    }
+  }
 
   // softmax: the factor cs > 0 and the per-tile bias commute with the maximum, so the reference
   // check runs on the raw sums and every weight costs one FMA and one ex2
@@ -616,7 +626,8 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
 
   const int group = layer / dm.rs_group;
   const int32_t* cnt = cv.count + (static_cast<long long>(group) * dm.batch + b) * 4;
-  const int tpc = dm.chunk / kTileTokens;
+  const int tpc = tiles_per_chunk_of(dm.chunk);
+  const int n_valid = tile_tokens_of(dm.chunk);      // token positions of a tile that hold tokens
   const SplitRange rg = split_range(cnt, cv.capacity, tpc, split, n_splits);
 
   State st;
@@ -666,8 +677,8 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
       stream_units<3, 6144, 1>(pp, n, lane,
           [&](int u, int) { return stream + static_cast<long long>(first + u * kWarps) * 6144; },
           [&](const uint8_t* tiles, int u) {
-            if (u < n - 1 || last_bytes == 6144u) process_qunit<2, 2, G4>(tiles, st, qc, qb, lc, lane);
-            else process_qunit<2, 1, G4>(tiles, st, qc, qb, lc, lane);
+            if (u < n - 1 || last_bytes == 6144u) process_qunit<2, 2, G4>(tiles, st, qc, qb, lc, lane, n_valid);
+            else process_qunit<2, 1, G4>(tiles, st, qc, qb, lc, lane, n_valid);
           }, my_ring, last_bytes);
       phase_scale<2>(st, false);
     }
@@ -682,7 +693,7 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
       load_q_phase<4>(qb, qc, q_h, g, t4);
       stream_units<3, 5120, 1>(pp, n, lane,
           [&](int u, int) { return stream + static_cast<long long>(first + u * kWarps) * 5120; },
-          [&](const uint8_t* tile, int) { process_qunit<4, 1, G4>(tile, st, qc, qb, lc, lane); }, my_ring);
+          [&](const uint8_t* tile, int) { process_qunit<4, 1, G4>(tile, st, qc, qb, lc, lane, n_valid); }, my_ring);
       phase_scale<4>(st, false);
     }
     dealt += rg.hi[1] - rg.lo[1];
@@ -696,7 +707,7 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
       load_q_phase<8>(qb, qc, q_h, g, t4);
       stream_units<2, 9216, 1>(pp, n, lane,
           [&](int u, int) { return stream + static_cast<long long>(first + u * kWarps) * 9216; },
-          [&](const uint8_t* tile, int) { process_qunit<8, 1, G4>(tile, st, qc, qb, lc, lane); }, my_ring);
+          [&](const uint8_t* tile, int) { process_qunit<8, 1, G4>(tile, st, qc, qb, lc, lane, n_valid); }, my_ring);
       phase_scale<8>(st, false);
     }
     dealt += rg.hi[2] - rg.lo[2];
@@ -714,7 +725,10 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
           [&](int u, int piece) {
             return stream + static_cast<long long>(first + (u >> 1) * kWarps) * kRawTileBytes + piece * 8192 + (u & 1) * 4096;
           },
-          [&](const uint8_t* stg, int) { process_raw16<BF16>(stg, stg + 4096, 16, st, qr, c_bias, lane); }, my_ring);
+          [&](const uint8_t* stg, int u) {
+            const int nv = min(16, n_valid - 16 * (u & 1));   // a short chunk's tile: rows past n_valid are padding
+            if (nv > 0) process_raw16<BF16>(stg, stg + 4096, nv, st, qr, c_bias, lane);
+          }, my_ring);
       phase_scale<16>(st, false);
     }
   }

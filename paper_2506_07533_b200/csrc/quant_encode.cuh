@@ -89,7 +89,8 @@ template <int BITS> __device__ __forceinline__ int key_meta_index(int c) {
 
 // ---- keys: lane owns channels 4*lane .. 4*lane+3 over the tile's 32 tokens --------------
 template <int BITS, bool BF16>
-__device__ __forceinline__ void encode_keys(const uint8_t* __restrict__ in, uint8_t* __restrict__ out, int lane) {
+__device__ __forceinline__ void encode_keys(const uint8_t* __restrict__ in, uint8_t* __restrict__ out, int lane,
+                                            int n_valid = kTileTokens) {
   constexpr float qmax = static_cast<float>((1 << BITS) - 1);
   const uint2* rows = reinterpret_cast<const uint2*>(in) + lane;         // row t at rows[32 * t]
   uint32_t mn01, mn23, mx01, mx23;
@@ -99,7 +100,8 @@ __device__ __forceinline__ void encode_keys(const uint8_t* __restrict__ in, uint
   }
 #pragma unroll
   for (int t = 1; t < kTileTokens; ++t) {
-    const uint2 w = rows[32 * t];
+    // rows past n_valid are padding of a short chunk: the group is the chunk's own tokens
+    const uint2 w = rows[t < n_valid ? 32 * t : 0];
     mn01 = min2<BF16>(mn01, w.x); mx01 = max2<BF16>(mx01, w.x);
     mn23 = min2<BF16>(mn23, w.y); mx23 = max2<BF16>(mx23, w.y);
   }
@@ -128,7 +130,8 @@ __device__ __forceinline__ void encode_keys(const uint8_t* __restrict__ in, uint
     uint32_t u0, u1, u2, u3;
     encode2<BF16>(w.x, negz01, inv01, u0, u1);
     encode2<BF16>(w.y, negz23, inv23, u2, u3);
-    const uint32_t p = pack4<BITS>(u0, u1, u2, u3);
+    uint32_t p = pack4<BITS>(u0, u1, u2, u3);
+    if (t >= n_valid) p = 0u;                  // padding positions carry code 0
     const int blk = t >> 4, hh = (t >> 3) & 1, g = t & 7;
     if (BITS == 2) {
       pay[(32 * blk + 4 * g + q) * 16 + 8 * hh + l7] = static_cast<uint8_t>(p);
@@ -143,7 +146,7 @@ __device__ __forceinline__ void encode_keys(const uint8_t* __restrict__ in, uint
 // ---- values: groups are 32 channels of one token -----------------------------------------
 template <int BITS, bool BF16>
 __device__ __forceinline__ void encode_values(const uint8_t* __restrict__ in, uint8_t* __restrict__ out,
-                                              float4* __restrict__ prm, int lane) {
+                                              float4* __restrict__ prm, int lane, int n_valid = kTileTokens) {
   constexpr float qmax = static_cast<float>((1 << BITS) - 1);
   uint16_t* meta = reinterpret_cast<uint16_t*>(out);
   {
@@ -166,6 +169,9 @@ __device__ __forceinline__ void encode_values(const uint8_t* __restrict__ in, ui
       float zf, inv;
       uint16_t sb, zb;
       group_params(fminf(lo_f<BF16>(mn), hi_f<BF16>(mn)), fmaxf(lo_f<BF16>(mx), hi_f<BF16>(mx)), qmax, sb, zb, zf, inv);
+      if (t >= n_valid) {                      // padding token: scale 0, zero 0, every code 0
+        sb = 0; zb = 0; zf = 0.0f; inv = 0.0f;
+      }
       prm[4 * t + cg] = make_float4(-zf, -zf, inv, inv);
       meta[256 + ((((blk * 2 + (cg >> 1)) * 4 + t4) * 4 + (cg & 1) * 2 + half) * 2) + e] = sb;
       meta[384 + ((((blk * 4 + cg) * 4 + t4) * 2 + half) * 2) + e] = zb;
@@ -188,6 +194,10 @@ __device__ __forceinline__ void encode_values(const uint8_t* __restrict__ in, ui
         const ulonglong2 zi = *reinterpret_cast<const ulonglong2*>(prm + 4 * t + p);    // (-z, -z), (inv, inv)
         encode2<BF16>(w.x, zi.x, zi.y, u[bp][0], u[bp][1]);
         encode2<BF16>(w.y, zi.x, zi.y, u[bp][2], u[bp][3]);
+        if (t >= n_valid) {                    // padding token: code 0 whatever the row holds
+#pragma unroll
+          for (int k = 0; k < 4; ++k) u[bp][k] = __float_as_uint(kMagic);
+        }
       }
       const int ln = 4 * g + t4;
       if (BITS == 2) {
@@ -220,13 +230,16 @@ __device__ __forceinline__ void encode_values(const uint8_t* __restrict__ in, ui
 }
 
 // 16-bit tile half (keys or values): rows copied in the input dtype, 16-byte units swizzled.
-__device__ __forceinline__ void copy_raw_rows(const uint8_t* __restrict__ in, uint8_t* __restrict__ dst, int lane) {
+__device__ __forceinline__ void copy_raw_rows(const uint8_t* __restrict__ in, uint8_t* __restrict__ dst, int lane,
+                                              int n_valid = kTileTokens) {
 #pragma unroll
   for (int i = 0; i < 16; ++i) {
     const int idx = i * 32 + lane;
     const int row = idx >> 4, U = idx & 15;
     const int up = (U & 8) | ((U ^ row) & 7);
-    *reinterpret_cast<uint4*>(dst + row * 256 + up * 16) = *reinterpret_cast<const uint4*>(in + row * 256 + U * 16);
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);      // rows past a short chunk's tokens are zero
+    if (row < n_valid) v = *reinterpret_cast<const uint4*>(in + row * 256 + U * 16);
+    *reinterpret_cast<uint4*>(dst + row * 256 + up * 16) = v;
   }
 }
 

@@ -53,7 +53,8 @@ quantize_pack_kernel(Dims dm, CacheView cv, const __grid_constant__ CUtensorMap 
   __syncwarp();
 
   const int H = dm.n_kv_heads;
-  const int tpc = dm.chunk / kTileTokens;
+  const int tpc = tiles_per_chunk_of(dm.chunk);
+  const int n_valid = tile_tokens_of(dm.chunk);      // rows of a tile that hold tokens (a short chunk: the rest is padding)
   const int C = T / dm.chunk;
   const long long stride = static_cast<long long>(gridDim.x) * kQWarps;
   const int group = layer / dm.rs_group;
@@ -134,16 +135,16 @@ quantize_pack_kernel(Dims dm, CacheView cv, const __grid_constant__ CUtensorMap 
     if (!mbar_wait_bounded(barK, parity)) { failed = 1; break; }
     if (valid) {
       if (w == 3) {
-        copy_raw_rows(bufK, tile, lane);
+        copy_raw_rows(bufK, tile, lane, n_valid);
       } else {
         if (store_pending) {                  // the previous tile's bulk store must have read `out`
           if (lane == 0) bulk_store_wait_read();
           __syncwarp();
           store_pending = false;
         }
-        if (w == 0) encode_keys<2, BF16>(bufK, out, lane);
-        else if (w == 1) encode_keys<4, BF16>(bufK, out, lane);
-        else encode_keys<8, BF16>(bufK, out, lane);
+        if (w == 0) encode_keys<2, BF16>(bufK, out, lane, n_valid);
+        else if (w == 1) encode_keys<4, BF16>(bufK, out, lane, n_valid);
+        else encode_keys<8, BF16>(bufK, out, lane, n_valid);
       }
     }
     __syncwarp();                             // every lane is done reading bufK
@@ -153,11 +154,11 @@ quantize_pack_kernel(Dims dm, CacheView cv, const __grid_constant__ CUtensorMap 
     if (!mbar_wait_bounded(barV, parity)) { failed = 2; break; }
     if (valid) {
       if (w == 3) {
-        copy_raw_rows(bufV, tile + 8192, lane);
+        copy_raw_rows(bufV, tile + 8192, lane, n_valid);
       } else {
-        if (w == 0) encode_values<2, BF16>(bufV, out, prm, lane);
-        else if (w == 1) encode_values<4, BF16>(bufV, out, prm, lane);
-        else encode_values<8, BF16>(bufV, out, prm, lane);
+        if (w == 0) encode_values<2, BF16>(bufV, out, prm, lane, n_valid);
+        else if (w == 1) encode_values<4, BF16>(bufV, out, prm, lane, n_valid);
+        else encode_values<8, BF16>(bufV, out, prm, lane, n_valid);
       }
     }
     __syncwarp();
@@ -263,7 +264,7 @@ static bool make_tile_map(CUtensorMap* m, const void* base, long long rows, long
 cudaError_t launch_quantize(const Dims& dm, const CacheView& cv, const void* K, const void* V, int T,
                             int layer, cudaStream_t st) {
   const int C = T / dm.chunk;
-  const long long n_tiles = static_cast<long long>(dm.batch) * C * (dm.chunk / kTileTokens) * dm.n_kv_heads;
+  const long long n_tiles = static_cast<long long>(dm.batch) * C * tiles_per_chunk_of(dm.chunk) * dm.n_kv_heads;
   if (n_tiles > 0) {
     CUtensorMap mapK, mapV;
     const long long rows = static_cast<long long>(dm.batch) * T, cols = static_cast<long long>(dm.n_kv_heads) * kHeadDim;
@@ -292,7 +293,7 @@ cudaError_t launch_quantize(const Dims& dm, const CacheView& cv, const void* K, 
 
 // Pack the full tails of `layer` into the chunk that launch_flush_route has just added to the tables.
 cudaError_t launch_flush_quantize(const Dims& dm, const CacheView& cv, int layer, cudaStream_t st) {
-  const long long n_tiles = static_cast<long long>(dm.batch) * (dm.chunk / kTileTokens) * dm.n_kv_heads;
+  const long long n_tiles = static_cast<long long>(dm.batch) * tiles_per_chunk_of(dm.chunk) * dm.n_kv_heads;
   CUtensorMap mapK, mapV;
   const long long rows = static_cast<long long>(dm.n_layers) * dm.batch * dm.n_kv_heads * dm.tail_capacity;
   if (!make_tile_map(&mapK, cv.tail_k, rows, kHeadDim) || !make_tile_map(&mapV, cv.tail_v, rows, kHeadDim))

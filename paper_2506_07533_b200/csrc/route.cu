@@ -90,8 +90,12 @@ route_score_vote_kernel(Dims dm, int32_t* __restrict__ votes /* [batch][max_chun
 
   const int g = lane >> 2, t4 = lane & 3;
   const int C = T / dm.chunk;
-  const int blocks_per_chunk = dm.chunk / 16;
+  // The hidden rows are walked in blocks of 16 tokens.  A chunk of 16 j tokens is j blocks; with
+  // chunks of 8 tokens one block holds two chunks (rows 0..7 and 8..15 vote separately).
+  const bool two_chunks = dm.chunk == 8;
+  const int blocks_per_chunk = two_chunks ? 1 : dm.chunk / 16;
   const int routed_chunks = C - first_chunk;
+  const int blocks_per_seq = two_chunks ? (routed_chunks + 1) / 2 : routed_chunks * blocks_per_chunk;
   float w3[4][4], bs[4];
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
@@ -106,10 +110,10 @@ route_score_vote_kernel(Dims dm, int32_t* __restrict__ votes /* [batch][max_chun
   const long long total_units = my_blocks * n_stages;                      // this warp's stream of stages
 
   auto block_coords = [&](long long blk, int& b, int& c, int& row) {
-    const int sub = static_cast<int>(blk % blocks_per_chunk);
-    const long long r = blk / blocks_per_chunk;
-    c = first_chunk + static_cast<int>(r % routed_chunks);
-    b = static_cast<int>(r / routed_chunks);
+    const int i = static_cast<int>(blk % blocks_per_seq);
+    b = static_cast<int>(blk / blocks_per_seq);
+    const int sub = two_chunks ? 0 : i % blocks_per_chunk;
+    c = first_chunk + (two_chunks ? 2 * i : i / blocks_per_chunk);
     row = b * T + c * dm.chunk + sub * 16;
   };
   auto issue = [&](long long u) {       // lane 0: stage u of this warp's stream
@@ -203,12 +207,19 @@ route_score_vote_kernel(Dims dm, int32_t* __restrict__ votes /* [batch][max_chun
     if (append_after) c_row = append_after[4 * b] + append_after[4 * b + 1] + append_after[4 * b + 2] + append_after[4 * b + 3];
     if (c_row >= dm.max_chunks) continue;
     int32_t* vrow = votes + (static_cast<long long>(b) * dm.max_chunks + c_row) * 4;
+    // rows 8..15 of the block: the same chunk, or (chunks of 8 tokens) the next one if it exists
+    const bool hi_counts = !two_chunks || (c + 1 < C && c_row + 1 < dm.max_chunks);
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
       const unsigned m1 = __ballot_sync(0xffffffffu, t4 == 0 && e_lo == k);
       const unsigned m2 = __ballot_sync(0xffffffffu, t4 == 0 && e_hi == k);
-      const int cnt = __popc(m1) + __popc(m2);
-      if (lane == 0 && cnt) atomicAdd(vrow + k, cnt);
+      if (two_chunks) {
+        if (lane == 0 && m1) atomicAdd(vrow + k, __popc(m1));
+        if (lane == 0 && m2 && hi_counts) atomicAdd(vrow + 4 + k, __popc(m2));
+      } else {
+        const int cnt = __popc(m1) + __popc(m2);
+        if (lane == 0 && cnt) atomicAdd(vrow + k, cnt);
+      }
     }
   }
   if (!ok) {
@@ -310,7 +321,8 @@ static cudaError_t launch_score_vote(const Dims& dm, const CacheView& cv, const 
                                      const void* W1, const void* W2, const float* W3, const float* bias,
                                      int32_t* votes, const int32_t* append_after, cudaStream_t st) {
   const int C = T / dm.chunk;
-  const long long n_blocks16 = static_cast<long long>(dm.batch) * (C > first ? C - first : 0) * (dm.chunk / 16);
+  const int routed = C > first ? C - first : 0;
+  const long long n_blocks16 = static_cast<long long>(dm.batch) * (dm.chunk == 8 ? (routed + 1) / 2 : routed * (dm.chunk / 16));
   if (n_blocks16 <= 0) return cudaSuccess;
   int dev = 0, sms = 148, smem_max = 0;
   cudaGetDevice(&dev);
