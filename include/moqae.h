@@ -64,9 +64,10 @@
  *     scale / zero of a channel are taken over the chunk's own tokens.  moqae_prefill_attn and
  *     moqae_project_quantize_kv refuse such configurations (MOQAE_ERR_UNSUPPORTED).
  *   pool[w] = [n_layers][batch][n_kv_heads][capacity[w]] slots of width w.
- *   map/slot/count/votes tables are per routing-sharing group: [n_groups][batch][max_chunks]
- *     (count: [n_groups][batch][4], votes: [n_groups][batch][max_chunks][4]),
- *     n_groups = ceil(n_layers / rs_group), max_chunks = max_tokens / chunk.
+ *   map/slot/count/votes tables are per routing-sharing group: [n_groups][rows][max_chunks]
+ *     (count: [n_groups][rows][4], votes: [n_groups][rows][max_chunks][4]),
+ *     n_groups = ceil(n_layers / rs_group), max_chunks = max_tokens / chunk, rows = batch, or
+ *     batch * n_kv_heads with per-head routing (cfg->per_head_routing).
  *   tail_k / tail_v = [n_layers][batch][n_kv_heads][tail_capacity][128] rows in the input
  *     dtype (tokens that do not fill a chunk stay 16-bit, Section 3.2); tail_len =
  *     int32 [n_layers][batch].
@@ -112,6 +113,12 @@ typedef struct moqae_config {
   int32_t max_tokens;      /* largest context the tables are sized for */
   int32_t tail_capacity;   /* rows per (layer, batch, kv head) in the 16-bit tail */
   int32_t batch;
+  int32_t per_head_routing; /* 0: one map per (group, sequence), shared by all kv heads (router input =
+                               the block's hidden state).  1: one map per (group, sequence, kv head),
+                               routed on that head's own 128-wide rows (Section 3.2: D = the
+                               embedding dimension within each attention head): d_in must be 128,
+                               hidden is [batch][T][n_kv_heads][128], and map / slot / count /
+                               votes have batch * n_kv_heads rows per group, row b * n_kv_heads + h */
 } moqae_config;
 
 /* View of a cache: device pointers supplied by the caller (see moqae_cache_bytes for sizes). */
@@ -154,7 +161,9 @@ int moqae_cache_bind(const moqae_config* cfg, const int64_t capacity[4],
 
 /*
  * Router of one routing-sharing group (Section 3.2, Eq. 1 and Eq. 2; Section 3.4).
- *   hidden  [batch][T][d_in] input-dtype rows of the group's FIRST layer.
+ *   hidden  [batch][T][d_in] input-dtype rows of the group's FIRST layer; with per-head routing
+ *           [batch][T][n_kv_heads][128] (token-major), head h of sequence b being routed on its own
+ *           rows into table row b * n_kv_heads + h.
  *   W1, W2  [d_in][4] input dtype; W3 [4][4] float32 row-major; bias [4] float32.
  *           W2 = W3 = NULL selects the linear router P = C W1 + bias; all non-NULL selects
  *           Eq. 1, P = SiLU((C W1) * (C W2)) W3 + bias.  bias may be NULL (zero).
@@ -173,8 +182,8 @@ int moqae_route(const moqae_config* cfg, const void* hidden, int32_t T, const vo
  * Quantise and pack the keys and values of one layer (prefill).
  *   K, V [batch][T][n_kv_heads][128] input dtype.
  *   forced_map: NULL = use the map routed for the layer's group; otherwise uint8
- *   [batch][T/chunk] expert indices that REPLACE the group's map (slot and count are
- *   recomputed) before quantising.
+ *   [rows][T/chunk] expert indices (rows as in the tables above) that REPLACE the group's map
+ *   (slot and count are recomputed) before quantising.
  *   Chunk c of sequence b goes to pool[map] slot `slot[b][c]` of every kv head; trailing
  *   T mod chunk tokens are copied to the tail and tail_len[layer][b] is set.
  *   A chunk whose slot index is >= capacity is skipped and status[0] becomes

@@ -34,7 +34,8 @@ class MoqaeConfig(C.Structure):
                 ("head_dim", C.c_int32), ("chunk", C.c_int32), ("group", C.c_int32),
                 ("dtype", C.c_int32), ("n_experts", C.c_int32), ("expert_bits", C.c_int32 * 4),
                 ("rs_group", C.c_int32), ("rf_first_chunk", C.c_int32), ("d_in", C.c_int32),
-                ("max_tokens", C.c_int32), ("tail_capacity", C.c_int32), ("batch", C.c_int32)]
+                ("max_tokens", C.c_int32), ("tail_capacity", C.c_int32), ("batch", C.c_int32),
+                ("per_head_routing", C.c_int32)]
 
 
 class MoqaeCache(C.Structure):
@@ -122,7 +123,7 @@ def _stream():
 
 
 def make_config(*, n_layers, n_q_heads, n_kv_heads, chunk, dtype, d_in, max_tokens, batch, rs_group=1,
-                rf_first_chunk=1, tail_capacity=None) -> MoqaeConfig:
+                rf_first_chunk=1, tail_capacity=None, per_head_routing=False) -> MoqaeConfig:
     cfg = MoqaeConfig()
     cfg.n_layers, cfg.n_q_heads, cfg.n_kv_heads = n_layers, n_q_heads, n_kv_heads
     cfg.head_dim, cfg.chunk, cfg.group, cfg.dtype, cfg.n_experts = 128, chunk, 32, dtype, 4
@@ -130,6 +131,7 @@ def make_config(*, n_layers, n_q_heads, n_kv_heads, chunk, dtype, d_in, max_toke
     cfg.rs_group, cfg.rf_first_chunk, cfg.d_in = rs_group, int(rf_first_chunk), d_in
     cfg.max_tokens, cfg.batch = max_tokens, batch
     cfg.tail_capacity = chunk if tail_capacity is None else tail_capacity
+    cfg.per_head_routing = int(bool(per_head_routing))
     return cfg
 
 
@@ -160,6 +162,12 @@ class Cache:
     def max_chunks(self):
         return self.cfg.max_tokens // self.cfg.chunk
 
+    @property
+    def table_rows(self):
+        """Rows of the map / slot / count / votes tables per group: one per sequence, or one per
+        (sequence, kv head) with per-head routing."""
+        return self.cfg.batch * (self.cfg.n_kv_heads if self.cfg.per_head_routing else 1)
+
     def table(self, idx, dtype, shape):
         n = 1
         for d in shape:
@@ -169,19 +177,19 @@ class Cache:
 
     @property
     def map(self):
-        return self.table(4, torch.uint8, (self.n_groups, self.cfg.batch, self.max_chunks))
+        return self.table(4, torch.uint8, (self.n_groups, self.table_rows, self.max_chunks))
 
     @property
     def slot(self):
-        return self.table(5, torch.int32, (self.n_groups, self.cfg.batch, self.max_chunks))
+        return self.table(5, torch.int32, (self.n_groups, self.table_rows, self.max_chunks))
 
     @property
     def count(self):
-        return self.table(6, torch.int32, (self.n_groups, self.cfg.batch, 4))
+        return self.table(6, torch.int32, (self.n_groups, self.table_rows, 4))
 
     @property
     def votes(self):
-        return self.table(7, torch.int32, (self.n_groups, self.cfg.batch, self.max_chunks, 4))
+        return self.table(7, torch.int32, (self.n_groups, self.table_rows, self.max_chunks, 4))
 
     @property
     def tail_len(self):

@@ -31,6 +31,8 @@ int check_config(const moqae_config* c) {
   if (c->n_q_heads % c->n_kv_heads != 0) return MOQAE_ERR_INVALID_ARG;
   if (c->n_q_heads / c->n_kv_heads > moqae::kMaxQueryGroup) return MOQAE_ERR_UNSUPPORTED;
   if (c->d_in < 32 || c->d_in % 32 != 0) return MOQAE_ERR_UNSUPPORTED;
+  if (c->per_head_routing != 0 && c->per_head_routing != 1) return MOQAE_ERR_INVALID_ARG;
+  if (c->per_head_routing && c->d_in != moqae::kHeadDim) return MOQAE_ERR_UNSUPPORTED;
   return MOQAE_OK;
 }
 
@@ -47,6 +49,8 @@ moqae::Dims dims_of(const moqae_config* c) {
   d.max_chunks = c->max_tokens / c->chunk;
   d.tail_capacity = c->tail_capacity;
   d.batch = c->batch;
+  d.per_head = c->per_head_routing ? 1 : 0;
+  d.n_tseq = d.per_head ? c->batch * c->n_kv_heads : c->batch;
   return d;
 }
 
@@ -96,7 +100,7 @@ int sm_count_of_current_device() {
 #pragma GCC visibility push(default)
 extern "C" {
 
-int moqae_version(void) { return 100; }
+int moqae_version(void) { return 200; }
 
 int moqae_last_cuda_error(void) { return g_last_cuda_error; }
 
@@ -124,10 +128,11 @@ int moqae_cache_bytes(const moqae_config* cfg, const int64_t capacity[4], int64_
     if (capacity[w] < 0) return MOQAE_ERR_INVALID_ARG;
     out_bytes[w] = lbh * capacity[w] * tpc * moqae::tile_bytes_of_expert(w);
   }
-  const int64_t tbl = static_cast<int64_t>(n_groups(cfg)) * cfg->batch * (cfg->max_tokens / cfg->chunk);
+  const int64_t rows = cfg->per_head_routing ? static_cast<int64_t>(cfg->batch) * cfg->n_kv_heads : cfg->batch;
+  const int64_t tbl = static_cast<int64_t>(n_groups(cfg)) * rows * (cfg->max_tokens / cfg->chunk);
   out_bytes[4] = tbl;                                   // map, uint8
   out_bytes[5] = tbl * 4;                               // slot
-  out_bytes[6] = static_cast<int64_t>(n_groups(cfg)) * cfg->batch * 4 * 4;   // count
+  out_bytes[6] = static_cast<int64_t>(n_groups(cfg)) * rows * 4 * 4;         // count
   out_bytes[7] = tbl * 16;                              // votes
   out_bytes[8] = lbh * cfg->tail_capacity * moqae::kHeadDim * 2;
   out_bytes[9] = out_bytes[8];
@@ -211,7 +216,7 @@ int moqae_project_quantize_kv(const moqae_config* cfg, const void* hidden, const
   if (T < 0 || T > cfg->max_tokens || layer < 0 || layer >= cfg->n_layers) return MOQAE_ERR_INVALID_ARG;
   if (T > 0 && (!hidden || !Wk || !Wv)) return MOQAE_ERR_INVALID_ARG;
   if ((k_rounded == nullptr) != (v_rounded == nullptr)) return MOQAE_ERR_INVALID_ARG;
-  if (cfg->d_in % 64 != 0 || cfg->chunk < moqae::kTileTokens) return MOQAE_ERR_UNSUPPORTED;
+  if (cfg->d_in % 64 != 0 || cfg->chunk < moqae::kTileTokens || cfg->per_head_routing) return MOQAE_ERR_UNSUPPORTED;
   if (!aligned16(hidden) || !aligned16(Wk) || !aligned16(Wv) || !aligned16(k_rounded) || !aligned16(v_rounded))
     return MOQAE_ERR_MISALIGNED;
   if (T % cfg->chunk > cfg->tail_capacity) return MOQAE_ERR_POOL_FULL;
@@ -252,6 +257,7 @@ int moqae_flush_tail(const moqae_config* cfg, const void* hidden_tail, const voi
   if ((W2 == nullptr) != (W3 == nullptr)) return MOQAE_ERR_INVALID_ARG;
   if (layer_group < 0 || layer_group >= n_groups(cfg)) return MOQAE_ERR_INVALID_ARG;
   if (cfg->tail_capacity < cfg->chunk || !cache->tail_k || !cache->tail_v) return MOQAE_ERR_POOL_FULL;
+  if (cfg->per_head_routing) return MOQAE_ERR_UNSUPPORTED;               // the flush keeps one table row per sequence
   if (!aligned16(hidden_tail) || !aligned16(W1) || !aligned16(W2) || !aligned16(W3) || !aligned16(bias))
     return MOQAE_ERR_MISALIGNED;
   const moqae::Dims dm = dims_of(cfg);
@@ -316,6 +322,7 @@ int moqae_prefill_attn(const moqae_config* cfg, const void* q, int32_t T, int32_
   if (rc != MOQAE_OK) return rc;
   if (T < 0 || T > cfg->max_tokens || layer < 0 || layer >= cfg->n_layers) return MOQAE_ERR_INVALID_ARG;
   if (cfg->chunk < moqae::kTileTokens) return MOQAE_ERR_UNSUPPORTED;     // walks the cache in whole 32-token tiles
+  if (cfg->per_head_routing) return MOQAE_ERR_UNSUPPORTED;               // reads one map per sequence
   if (T > 0 && (!q || !out)) return MOQAE_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(out) || !aligned16(workspace)) return MOQAE_ERR_MISALIGNED;
   if (workspace && workspace_bytes < moqae::prefill_workspace_bytes(dims_of(cfg), T)) return MOQAE_ERR_WORKSPACE_TOO_SMALL;

@@ -44,7 +44,14 @@ struct CacheView {
 struct Dims {
   int n_layers, n_q_heads, n_kv_heads, chunk, dtype, rs_group, rf_first_chunk, d_in;
   int max_chunks, tail_capacity, batch;
+  int per_head;        // 1: one table row per (sequence, kv head) instead of one per sequence
+  int n_tseq;          // table rows per routing-sharing group: batch, or batch * n_kv_heads
 };
+
+// table row of (sequence b, kv head h)
+__host__ __device__ __forceinline__ int table_row(const Dims& dm, int b, int h) {
+  return dm.per_head ? b * dm.n_kv_heads + h : b;
+}
 
 __device__ __forceinline__ void set_status(int32_t* status, int code, int d0, int d1) {
   if (atomicCAS(status, 0, code) == 0) {

@@ -625,7 +625,7 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
   __syncthreads();
 
   const int group = layer / dm.rs_group;
-  const int32_t* cnt = cv.count + (static_cast<long long>(group) * dm.batch + b) * 4;
+  const int32_t* cnt = cv.count + (static_cast<long long>(group) * dm.n_tseq + table_row(dm, b, h)) * 4;
   const int tpc = tiles_per_chunk_of(dm.chunk);
   const int n_valid = tile_tokens_of(dm.chunk);      // token positions of a tile that hold tokens
   const SplitRange rg = split_range(cnt, cv.capacity, tpc, split, n_splits);

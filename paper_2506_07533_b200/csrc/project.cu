@@ -52,11 +52,6 @@ constexpr long long kProjWait = 1ll << 31;      // about a second of SM cycles
 
 enum { PB_FULL = 0, PB_EMPTY = kPStages, PB_ACC_FULL = 2 * kPStages, PB_ACC_EMPTY = 2 * kPStages + 2, PB_COUNT = 2 * kPStages + 4 };
 
-// tiled TMA load, three coordinates (innermost first)
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
-  asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];\n"
-               ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
-}
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(bar) : "memory");
 }

@@ -58,8 +58,8 @@ quantize_pack_kernel(Dims dm, CacheView cv, const __grid_constant__ CUtensorMap 
   const int C = T / dm.chunk;
   const long long stride = static_cast<long long>(gridDim.x) * kQWarps;
   const int group = layer / dm.rs_group;
-  const uint8_t* map_g = cv.map + static_cast<long long>(group) * dm.batch * dm.max_chunks;
-  const int32_t* slot_g = cv.slot + static_cast<long long>(group) * dm.batch * dm.max_chunks;
+  const uint8_t* map_g = cv.map + static_cast<long long>(group) * dm.n_tseq * dm.max_chunks;
+  const int32_t* slot_g = cv.slot + static_cast<long long>(group) * dm.n_tseq * dm.max_chunks;
 
   const int32_t* count_g = cv.count + static_cast<long long>(group) * dm.batch * 4;
   auto tile_ref = [&](long long id) {
@@ -75,7 +75,7 @@ quantize_pack_kernel(Dims dm, CacheView cv, const __grid_constant__ CUtensorMap 
       r.b = static_cast<int>(x / C);
       r.x = r.h * kHeadDim;
       r.y = r.b * T + c * dm.chunk + r.j * kTileTokens;
-      const long long tbl = static_cast<long long>(r.b) * dm.max_chunks + c;
+      const long long tbl = static_cast<long long>(table_row(dm, r.b, r.h)) * dm.max_chunks + c;
       r.w = map_g[tbl];                      // loaded one tile ahead of their use
       r.slot = slot_g[tbl];
     } else {

@@ -114,7 +114,8 @@ route_score_vote_kernel(Dims dm, int32_t* __restrict__ votes /* [batch][max_chun
     b = static_cast<int>(blk / blocks_per_seq);
     const int sub = two_chunks ? 0 : i % blocks_per_chunk;
     c = first_chunk + (two_chunks ? 2 * i : i / blocks_per_chunk);
-    row = b * T + c * dm.chunk + sub * 16;
+    // b is the table row: a sequence, or with per-head routing (sequence, kv head) = (b / H, b % H)
+    row = (dm.per_head ? b / dm.n_kv_heads : b) * T + c * dm.chunk + sub * 16;
   };
   auto issue = [&](long long u) {       // lane 0: stage u of this warp's stream
     const long long blk = blk0 + (u / n_stages) * blk_stride;
@@ -126,8 +127,9 @@ route_score_vote_kernel(Dims dm, int32_t* __restrict__ votes /* [batch][max_chun
     const int nb = min(kBoxesPerStage, n_boxes - box0);
     const uint32_t bar = smem_u32(bars + slot);
     mbar_expect_tx(bar, nb * kBoxBytes);
+    const int head = dm.per_head ? b % dm.n_kv_heads : 0;     // middle coordinate: which 128-wide row of the token
     for (int i = 0; i < nb; ++i)
-      tma_load_2d(smem_u32(ring + slot * kStageBytes + i * kBoxBytes), &map_hidden, (box0 + i) * kBoxCols, row, bar);
+      tma_load_3d(smem_u32(ring + slot * kStageBytes + i * kBoxBytes), &map_hidden, (box0 + i) * kBoxCols, head, row, bar);
   };
   if (lane == 0)
     for (long long u = 0; u < kStages && u < total_units; ++u) issue(u);
@@ -235,7 +237,7 @@ finalize_map_kernel(Dims dm, CacheView cv, int group, int n_chunks, const uint8_
   __shared__ int s_cnt[256][4];
   const int b = blockIdx.x;
   const int tid = threadIdx.x;
-  const long long base = (static_cast<long long>(group) * dm.batch + b) * dm.max_chunks;
+  const long long base = (static_cast<long long>(group) * dm.n_tseq + b) * dm.max_chunks;
   uint8_t* map = cv.map + base;
   int32_t* slot = cv.slot + base;
   const int32_t* votes = cv.votes + base * 4;
@@ -270,7 +272,7 @@ finalize_map_kernel(Dims dm, CacheView cv, int group, int n_chunks, const uint8_
       s_cnt[i][tid] = run;
       run += v;
     }
-    cv.count[(static_cast<long long>(group) * dm.batch + b) * 4 + tid] = run;
+    cv.count[(static_cast<long long>(group) * dm.n_tseq + b) * 4 + tid] = run;
   }
   __syncthreads();
 #pragma unroll
@@ -322,7 +324,7 @@ static cudaError_t launch_score_vote(const Dims& dm, const CacheView& cv, const 
                                      int32_t* votes, const int32_t* append_after, cudaStream_t st) {
   const int C = T / dm.chunk;
   const int routed = C > first ? C - first : 0;
-  const long long n_blocks16 = static_cast<long long>(dm.batch) * (dm.chunk == 8 ? (routed + 1) / 2 : routed * (dm.chunk / 16));
+  const long long n_blocks16 = static_cast<long long>(dm.n_tseq) * (dm.chunk == 8 ? (routed + 1) / 2 : routed * (dm.chunk / 16));
   if (n_blocks16 <= 0) return cudaSuccess;
   int dev = 0, sms = 148, smem_max = 0;
   cudaGetDevice(&dev);
@@ -332,11 +334,14 @@ static cudaError_t launch_score_vote(const Dims& dm, const CacheView& cv, const 
   EncodeTiledFn enc = encode_tiled_fn();
   if (!enc) return cudaErrorNotSupported;
   CUtensorMap map;
-  const cuuint64_t gdim[2] = {static_cast<cuuint64_t>(dm.d_in), static_cast<cuuint64_t>(dm.batch) * T};
-  const cuuint64_t gstride[1] = {static_cast<cuuint64_t>(dm.d_in) * 2};
-  const cuuint32_t box[2] = {kBoxCols, 16};
-  const cuuint32_t estr[2] = {1, 1};
-  if (enc(&map, CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, const_cast<void*>(hidden), gdim, gstride, box, estr,
+  // viewed as [batch * T tokens][rows per token][d_in]: one row per token, or with per-head routing
+  // the token's n_kv_heads rows of 128 channels; a box is 16 tokens of ONE such row
+  const cuuint64_t per_tok = dm.per_head ? dm.n_kv_heads : 1;
+  const cuuint64_t gdim[3] = {static_cast<cuuint64_t>(dm.d_in), per_tok, static_cast<cuuint64_t>(dm.batch) * T};
+  const cuuint64_t gstride[2] = {static_cast<cuuint64_t>(dm.d_in) * 2, static_cast<cuuint64_t>(dm.d_in) * 2 * per_tok};
+  const cuuint32_t box[3] = {kBoxCols, 1, 16};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  if (enc(&map, CU_TENSOR_MAP_DATA_TYPE_UINT16, 3, const_cast<void*>(hidden), gdim, gstride, box, estr,
           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return cudaErrorInvalidValue;
@@ -371,9 +376,9 @@ cudaError_t launch_route(const Dims& dm, const CacheView& cv, const void* hidden
                          const void* W2, const float* W3, const float* bias, int group,
                          int32_t* votes_out, cudaStream_t st) {
   const int C = T / dm.chunk;
-  const long long tbl = static_cast<long long>(group) * dm.batch * dm.max_chunks;
+  const long long tbl = static_cast<long long>(group) * dm.n_tseq * dm.max_chunks;
   int32_t* votes = cv.votes + tbl * 4;
-  cudaError_t e = cudaMemsetAsync(votes, 0, sizeof(int32_t) * 4 * static_cast<size_t>(dm.batch) * dm.max_chunks, st);
+  cudaError_t e = cudaMemsetAsync(votes, 0, sizeof(int32_t) * 4 * static_cast<size_t>(dm.n_tseq) * dm.max_chunks, st);
   if (e != cudaSuccess) return e;
   e = launch_score_vote(dm, cv, hidden, T, dm.rf_first_chunk ? 1 : 0, W1, W2, W3, bias, votes, nullptr, st);
   if (e != cudaSuccess) return e;
@@ -381,7 +386,7 @@ cudaError_t launch_route(const Dims& dm, const CacheView& cv, const void* hidden
   if (e != cudaSuccess) return e;
   if (votes_out && C > 0) {
     e = cudaMemcpy2DAsync(votes_out, sizeof(int32_t) * 4 * C, votes, sizeof(int32_t) * 4 * dm.max_chunks,
-                          sizeof(int32_t) * 4 * C, dm.batch, cudaMemcpyDeviceToDevice, st);
+                          sizeof(int32_t) * 4 * C, dm.n_tseq, cudaMemcpyDeviceToDevice, st);
   }
   return e;
 }
@@ -404,7 +409,7 @@ cudaError_t launch_flush_route(const Dims& dm, const CacheView& cv, const void* 
 
 cudaError_t launch_finalize_map(const Dims& dm, const CacheView& cv, int group, int n_chunks,
                                 const uint8_t* forced_map, cudaStream_t st) {
-  finalize_map_kernel<<<dm.batch, 256, 0, st>>>(dm, cv, group, n_chunks, forced_map);
+  finalize_map_kernel<<<dm.n_tseq, 256, 0, st>>>(dm, cv, group, n_chunks, forced_map);
   return cudaGetLastError();
 }
 

@@ -40,7 +40,7 @@ def test_version_and_error_strings(lib):
 
 
 def test_struct_sizes_match_header():
-    assert ctypes.sizeof(mq.MoqaeConfig) == 18 * 4
+    assert ctypes.sizeof(mq.MoqaeConfig) == 19 * 4
     assert ctypes.sizeof(mq.MoqaeCache) == 4 * 8 + 4 * 8 + 8 * 8
 
 

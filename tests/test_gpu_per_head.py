@@ -60,3 +60,71 @@ def test_per_head_routing_as_head_major_batch():
     want = O.decode_attn(synth.to_u16(q), dtype, ocache, chunk)
     ok, e_abs, e_rel = H.attn_tolerance_ok(out.cpu().numpy(), want)
     assert ok, (e_abs, e_rel)
+
+
+@pytest.mark.parametrize("chunk", [64, 16])
+def test_per_head_routing_token_major(chunk):
+    """cfg.per_head_routing: the tensors stay token-major ([batch][T][heads][128] for the router
+    input, K and V alike) and the library keeps one map per (sequence, kv head).  The oracle sees
+    the same data head by head (one single-head sequence per (b, h)): maps with the near-tie rule,
+    packed bytes exactly, attention within tolerance."""
+    B, Hkv, G, dtype = 2, 3, 2, 1
+    T = chunk * 9 + 5
+    C = T // chunk
+    K, V = H.make_kv(B, T, Hkv, dtype, 820, outlier_channels=(5, 64))
+    # every head's own 128 router features per token, chunk-structured per (sequence, head)
+    hid_hm = synth.hidden_states(B * Hkv, T, 128, chunk, dtype, 823, "cpu")            # [(b, h), T, 128]
+    hidden = hid_hm.view(B, Hkv, T, 128).permute(0, 2, 1, 3).contiguous()             # [B, T, H, 128]
+    W1, W2, W3, bias = synth.router_weights(128, 4, dtype, 821, "cpu", std=0.1)
+    q = synth.normal((B, Hkv * G, 128), dtype, 822, "cpu")
+    cfg = mq.make_config(n_layers=1, n_q_heads=Hkv * G, n_kv_heads=Hkv, chunk=chunk, dtype=dtype, d_in=128,
+                         max_tokens=T, batch=B, per_head_routing=True)
+    cache = mq.moqae_cache_bind(cfg, [C, C, C, C], zero_pools=True)
+    assert cache.map.shape == (1, B * Hkv, C)
+    votes_out = torch.full((B * Hkv, C, 4), -1, dtype=torch.int32, device="cuda")
+    mq.moqae_route(cfg, hidden.cuda(), T, W1.cuda(), W2.cuda(), W3.cuda(), bias.cuda(), 0, cache, votes_out)
+    mq.moqae_quantize_kv(cfg, K.cuda(), V.cuda(), T, 0, cache)
+    ws = torch.zeros(mq.moqae_decode_attn_workspace(cfg), dtype=torch.uint8, device="cuda")
+    out = torch.full((B, Hkv * G, 128), float("nan"), dtype=torch.float32, device="cuda")
+    mq.moqae_decode_attn(cfg, q.cuda(), 0, cache, out, ws)
+    torch.cuda.synchronize()
+    assert mq.moqae_poll_status(cache) == 0
+    gmap = cache.map[0].cpu().numpy()
+    gvotes = cache.votes[0].cpu().numpy()
+    assert (votes_out.cpu().numpy() == gvotes[:, :C]).all()
+    assert (gmap[:, 0] == 3).all()
+    assert any((gmap[b * Hkv] != gmap[b * Hkv + h]).any() for b in range(B) for h in range(1, Hkv))   # heads differ
+    w1, w2 = synth.to_u16(W1), synth.to_u16(W2)
+    n_fragile = 0
+    for b in range(B):
+        for h in range(Hkv):
+            s = b * Hkv + h
+            for c in range(1, C):
+                n_fragile += H.check_routed_chunk(synth.to_u16(hidden[b, c * chunk:(c + 1) * chunk, h]), dtype, w1, w2,
+                                                  W3.numpy(), bias.numpy(), gvotes[s, c], gmap[s, c])
+            # this head's slots against the oracle run on it as a one-head sequence with its own map
+            oc = O.quantize_kv(synth.to_u16(K[b:b + 1, :, h:h + 1]), synth.to_u16(V[b:b + 1, :, h:h + 1]), dtype, chunk,
+                               gmap[s:s + 1])
+            assert (cache.count[0, s].cpu().numpy() == oc["count"][0]).all()
+            assert (cache.slot[0, s, :C].cpu().numpy() == oc["slot"][0]).all()
+            for w in range(4):
+                n = int(oc["count"][0, w])
+                if n:
+                    assert (cache.pool(w)[0, b, h, :n].cpu().numpy() == oc["pools"][w][0, 0, :n]).all(), (b, h, w)
+            want = O.decode_attn(synth.to_u16(q[b:b + 1, h * G:(h + 1) * G]), dtype, oc, chunk)
+            ok, e_abs, e_rel = H.attn_tolerance_ok(out[b:b + 1, h * G:(h + 1) * G].cpu().numpy(), want)
+            assert ok, (b, h, e_abs, e_rel)
+    assert n_fragile < B * Hkv * C // 2
+
+
+def test_per_head_routing_argument_rules():
+    # the per-head router input is the head's own 128 channels
+    bad = mq.make_config(n_layers=1, n_q_heads=2, n_kv_heads=2, chunk=32, dtype=1, d_in=256, max_tokens=64, batch=1,
+                         per_head_routing=True)
+    with pytest.raises(mq.MoqaeError) as e:
+        mq.moqae_cache_bytes(bad, [1, 1, 1, 1])
+    assert e.value.code == mq.ERR_UNSUPPORTED
+    cfg = mq.make_config(n_layers=1, n_q_heads=2, n_kv_heads=2, chunk=32, dtype=1, d_in=128, max_tokens=64, batch=3,
+                         per_head_routing=True)
+    sizes = mq.moqae_cache_bytes(cfg, [1, 1, 1, 1])
+    assert sizes[4] == 3 * 2 * 2 and sizes[6] == 3 * 2 * 16            # map and count rows per (sequence, head)
