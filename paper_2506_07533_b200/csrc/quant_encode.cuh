@@ -88,9 +88,14 @@ template <int BITS> __device__ __forceinline__ int key_meta_index(int c) {
 }
 
 // ---- keys: lane owns channels 4*lane .. 4*lane+3 over the tile's 32 tokens --------------
-template <int BITS, bool BF16>
+// `out` is the start of the tile image (metadata at its documented offsets); `pay_at`, if given,
+// is where the key payload goes instead of out + 1024 (a warp that assembles only the key part
+// of a tile keeps metadata and payload side by side).
+// SHORT = false: all 32 rows are tokens (n_valid is ignored and the row tests fold away).
+template <int BITS, bool BF16, bool SHORT = false>
 __device__ __forceinline__ void encode_keys(const uint8_t* __restrict__ in, uint8_t* __restrict__ out, int lane,
-                                            int n_valid = kTileTokens) {
+                                            int n_valid_arg = kTileTokens, uint8_t* pay_at = nullptr) {
+  const int n_valid = SHORT ? n_valid_arg : kTileTokens;
   constexpr float qmax = static_cast<float>((1 << BITS) - 1);
   const uint2* rows = reinterpret_cast<const uint2*>(in) + lane;         // row t at rows[32 * t]
   uint32_t mn01, mn23, mx01, mx23;
@@ -120,7 +125,7 @@ __device__ __forceinline__ void encode_keys(const uint8_t* __restrict__ in, uint
     meta[128 + ((idx & ~6) | ((idx & 2) << 1) | ((idx & 4) >> 1))] = zb[k];
   }
   // payload: this lane's 4 codes of token t are 4*BITS contiguous bits of the (t, quarter) piece
-  uint8_t* pay = out + kMetaBytes;
+  uint8_t* pay = pay_at ? pay_at : out + kMetaBytes;
   const uint64_t negz01 = pack_f2(-zf[0], -zf[1]), negz23 = pack_f2(-zf[2], -zf[3]);
   const uint64_t inv01 = pack_f2(inv[0], inv[1]), inv23 = pack_f2(inv[2], inv[3]);
   const int q = lane >> 3, l7 = lane & 7;
@@ -144,35 +149,50 @@ __device__ __forceinline__ void encode_keys(const uint8_t* __restrict__ in, uint
 }
 
 // ---- values: groups are 32 channels of one token -----------------------------------------
-template <int BITS, bool BF16>
+template <int BITS, bool BF16, bool SHORT = false>
 __device__ __forceinline__ void encode_values(const uint8_t* __restrict__ in, uint8_t* __restrict__ out,
-                                              float4* __restrict__ prm, int lane, int n_valid = kTileTokens) {
+                                              float4* __restrict__ prm, int lane, int n_valid_arg = kTileTokens,
+                                              uint8_t* pay_at = nullptr) {
+  const int n_valid = SHORT ? n_valid_arg : kTileTokens;
   constexpr float qmax = static_cast<float>((1 << BITS) - 1);
   uint16_t* meta = reinterpret_cast<uint16_t*>(out);
   {
-    // statistics: lane = token; its row is read in 16-byte units, rotated inside each channel
-    // group so that neighbouring lanes start on different banks
+    // statistics: lane = token.  Its row is read in 16-byte units; within each half of the row
+    // (two channel groups = 8 units) lane t starts at unit t & 7, so the 32 lanes of one load
+    // spread over all eight 16-byte bank groups (4 lanes each: the minimum for 512 bytes).
     const int t = lane;
     const uint4* row = reinterpret_cast<const uint4*>(in + t * 256);
     const int blk = t >> 4, half = (t >> 3) & 1, t4 = (t >> 1) & 3, e = t & 1;
+    constexpr uint32_t kPosInf = BF16 ? 0x7F807F80u : 0x7C007C00u, kNegInf = BF16 ? 0xFF80FF80u : 0xFC00FC00u;
+    uint32_t mn4[4], mx4[4];
 #pragma unroll
-    for (int cg = 0; cg < 4; ++cg) {
-      uint32_t mn = 0, mx = 0;
+    for (int cp = 0; cp < 2; ++cp) {
+      uint32_t mnA = kPosInf, mxA = kNegInf, mnB = kPosInf, mxB = kNegInf;     // A: this lane's first group, B: its second
 #pragma unroll
-      for (int ii = 0; ii < 4; ++ii) {
-        const uint4 v = row[4 * cg + (ii ^ (t & 3))];
+      for (int k = 0; k < 8; ++k) {
+        const int u = k ^ (t & 7);
+        const uint4 v = row[8 * cp + u];
         const uint32_t a = min2<BF16>(min2<BF16>(v.x, v.y), min2<BF16>(v.z, v.w));
         const uint32_t b = max2<BF16>(max2<BF16>(v.x, v.y), max2<BF16>(v.z, v.w));
-        mn = ii == 0 ? a : min2<BF16>(mn, a);
-        mx = ii == 0 ? b : max2<BF16>(mx, b);
+        // units 0..3 belong to group 2cp, 4..7 to 2cp + 1; u >> 2 = (k >> 2) ^ ((t >> 2) & 1), so the
+        // first four loads of a lane fall into one group and the last four into the other
+        if (k < 4) { mnA = min2<BF16>(mnA, a); mxA = max2<BF16>(mxA, b); }
+        else { mnB = min2<BF16>(mnB, a); mxB = max2<BF16>(mxB, b); }
       }
+      const bool swap = (t >> 2) & 1;          // lanes with bit 2 set met group 2cp + 1 first
+      mn4[2 * cp] = swap ? mnB : mnA; mx4[2 * cp] = swap ? mxB : mxA;
+      mn4[2 * cp + 1] = swap ? mnA : mnB; mx4[2 * cp + 1] = swap ? mxA : mxB;
+    }
+#pragma unroll
+    for (int cg = 0; cg < 4; ++cg) {
+      const uint32_t mn = mn4[cg], mx = mx4[cg];
       float zf, inv;
       uint16_t sb, zb;
       group_params(fminf(lo_f<BF16>(mn), hi_f<BF16>(mn)), fmaxf(lo_f<BF16>(mx), hi_f<BF16>(mx)), qmax, sb, zb, zf, inv);
       if (t >= n_valid) {                      // padding token: scale 0, zero 0, every code 0
         sb = 0; zb = 0; zf = 0.0f; inv = 0.0f;
       }
-      prm[4 * t + cg] = make_float4(-zf, -zf, inv, inv);
+      prm[32 * cg + t] = make_float4(-zf, -zf, inv, inv);       // [group][token]: neighbouring lanes, neighbouring banks
       meta[256 + ((((blk * 2 + (cg >> 1)) * 4 + t4) * 4 + (cg & 1) * 2 + half) * 2) + e] = sb;
       meta[384 + ((((blk * 4 + cg) * 4 + t4) * 2 + half) * 2) + e] = zb;
     }
@@ -181,7 +201,7 @@ __device__ __forceinline__ void encode_values(const uint8_t* __restrict__ in, ui
   // codes: lane = channels 4*lane .. 4*lane+3 (group p = lane / 8); one word set per 4 tokens
   const int p = lane >> 3, g = lane & 7;
   const uint2* rows = reinterpret_cast<const uint2*>(in) + lane;
-  uint8_t* pay = out + kMetaBytes + kTileTokens * 16 * BITS;
+  uint8_t* pay = pay_at ? pay_at : out + kMetaBytes + kTileTokens * 16 * BITS;
 #pragma unroll
   for (int blk = 0; blk < 2; ++blk) {
 #pragma unroll
@@ -191,7 +211,7 @@ __device__ __forceinline__ void encode_values(const uint8_t* __restrict__ in, ui
       for (int bp = 0; bp < 4; ++bp) {
         const int t = 16 * blk + 8 * (bp & 1) + 2 * t4 + (bp >> 1);
         const uint2 w = rows[32 * t];
-        const ulonglong2 zi = *reinterpret_cast<const ulonglong2*>(prm + 4 * t + p);    // (-z, -z), (inv, inv)
+        const ulonglong2 zi = *reinterpret_cast<const ulonglong2*>(prm + 32 * p + t);   // (-z, -z), (inv, inv)
         encode2<BF16>(w.x, zi.x, zi.y, u[bp][0], u[bp][1]);
         encode2<BF16>(w.y, zi.x, zi.y, u[bp][2], u[bp][3]);
         if (t >= n_valid) {                    // padding token: code 0 whatever the row holds
@@ -230,8 +250,10 @@ __device__ __forceinline__ void encode_values(const uint8_t* __restrict__ in, ui
 }
 
 // 16-bit tile half (keys or values): rows copied in the input dtype, 16-byte units swizzled.
+template <bool SHORT = false>
 __device__ __forceinline__ void copy_raw_rows(const uint8_t* __restrict__ in, uint8_t* __restrict__ dst, int lane,
-                                              int n_valid = kTileTokens) {
+                                              int n_valid_arg = kTileTokens) {
+  const int n_valid = SHORT ? n_valid_arg : kTileTokens;
 #pragma unroll
   for (int i = 0; i < 16; ++i) {
     const int idx = i * 32 + lane;

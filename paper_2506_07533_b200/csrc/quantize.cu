@@ -55,6 +55,7 @@ quantize_pack_kernel(Dims dm, CacheView cv, const __grid_constant__ CUtensorMap 
   const int H = dm.n_kv_heads;
   const int tpc = tiles_per_chunk_of(dm.chunk);
   const int n_valid = tile_tokens_of(dm.chunk);      // rows of a tile that hold tokens (a short chunk: the rest is padding)
+  const bool full = n_valid == kTileTokens;
   const int C = T / dm.chunk;
   const long long stride = static_cast<long long>(gridDim.x) * kQWarps;
   const int group = layer / dm.rs_group;
@@ -135,16 +136,23 @@ quantize_pack_kernel(Dims dm, CacheView cv, const __grid_constant__ CUtensorMap 
     if (!mbar_wait_bounded(barK, parity)) { failed = 1; break; }
     if (valid) {
       if (w == 3) {
-        copy_raw_rows(bufK, tile, lane, n_valid);
+        if (full) copy_raw_rows(bufK, tile, lane);
+        else copy_raw_rows<true>(bufK, tile, lane, n_valid);
       } else {
         if (store_pending) {                  // the previous tile's bulk store must have read `out`
           if (lane == 0) bulk_store_wait_read();
           __syncwarp();
           store_pending = false;
         }
-        if (w == 0) encode_keys<2, BF16>(bufK, out, lane, n_valid);
-        else if (w == 1) encode_keys<4, BF16>(bufK, out, lane, n_valid);
-        else encode_keys<8, BF16>(bufK, out, lane, n_valid);
+        if (full) {
+          if (w == 0) encode_keys<2, BF16>(bufK, out, lane);
+          else if (w == 1) encode_keys<4, BF16>(bufK, out, lane);
+          else encode_keys<8, BF16>(bufK, out, lane);
+        } else {                              // a chunk of 8 or 16 tokens: rows past it are padding
+          if (w == 0) encode_keys<2, BF16, true>(bufK, out, lane, n_valid);
+          else if (w == 1) encode_keys<4, BF16, true>(bufK, out, lane, n_valid);
+          else encode_keys<8, BF16, true>(bufK, out, lane, n_valid);
+        }
       }
     }
     __syncwarp();                             // every lane is done reading bufK
@@ -154,11 +162,16 @@ quantize_pack_kernel(Dims dm, CacheView cv, const __grid_constant__ CUtensorMap 
     if (!mbar_wait_bounded(barV, parity)) { failed = 2; break; }
     if (valid) {
       if (w == 3) {
-        copy_raw_rows(bufV, tile + 8192, lane, n_valid);
+        if (full) copy_raw_rows(bufV, tile + 8192, lane);
+        else copy_raw_rows<true>(bufV, tile + 8192, lane, n_valid);
+      } else if (full) {
+        if (w == 0) encode_values<2, BF16>(bufV, out, prm, lane);
+        else if (w == 1) encode_values<4, BF16>(bufV, out, prm, lane);
+        else encode_values<8, BF16>(bufV, out, prm, lane);
       } else {
-        if (w == 0) encode_values<2, BF16>(bufV, out, prm, lane, n_valid);
-        else if (w == 1) encode_values<4, BF16>(bufV, out, prm, lane, n_valid);
-        else encode_values<8, BF16>(bufV, out, prm, lane, n_valid);
+        if (w == 0) encode_values<2, BF16, true>(bufV, out, prm, lane, n_valid);
+        else if (w == 1) encode_values<4, BF16, true>(bufV, out, prm, lane, n_valid);
+        else encode_values<8, BF16, true>(bufV, out, prm, lane, n_valid);
       }
     }
     __syncwarp();
