@@ -89,6 +89,7 @@ extern "C" {
 #define MOQAE_ERR_WORKSPACE_TOO_SMALL (-5)
 #define MOQAE_ERR_CUDA (-6)
 #define MOQAE_ERR_TIMEOUT (-7)
+#define MOQAE_ERR_CORRUPT_TABLE (-8)
 
 #define MOQAE_DTYPE_FP16 0
 #define MOQAE_DTYPE_BF16 1
@@ -342,6 +343,27 @@ int moqae_prefill_attn(const moqae_config* cfg, const void* q, int32_t T, int32_
 int64_t moqae_decode_attn_static_max_bytes(void);
 int moqae_decode_attn_static(const moqae_config* cfg, const void* q, int32_t layer,
                              const moqae_cache* cache, float* out, float scale, void* stream);
+
+/*
+ * Debugging aid: check the chunk index tables of one routing-sharing group against the rules
+ * the kernels rely on (the slot rule of the storage format above: chunks of one width occupy
+ * slots 0, 1, 2, .. of that width's pool in chunk order).  For every table row and its first
+ * n_chunks chunks: map[c] is an expert index 0..3; slot[c] equals the number of earlier chunks
+ * of the row with the same width; slot[c] < capacity[width]; count[w] equals the number of chunks
+ * of width w.  The kernels never follow a slot beyond its pool (they report MOQAE_ERR_POOL_FULL
+ * or clamp), but a table that breaks these rules means chunks overwrite each other or are skipped.
+ *   moqae_validate_tables_host: map / slot / count are HOST arrays of one group laid out as the
+ *   device tables ([rows][max_chunks], count [rows][4]); pure host arithmetic.
+ *   moqae_validate_tables: copies the group's tables from the device (waits for `stream`) and
+ *   runs the same check; T is the context the tables describe (n_chunks = T / chunk).
+ * Returns MOQAE_OK or MOQAE_ERR_CORRUPT_TABLE; *bad_row / *bad_chunk (host, may be NULL) receive
+ * the first offending position.
+ */
+int moqae_validate_tables_host(const uint8_t* map, const int32_t* slot, const int32_t* count,
+                               int32_t rows, int32_t max_chunks, int32_t n_chunks,
+                               const int64_t capacity[4], int32_t* bad_row, int32_t* bad_chunk);
+int moqae_validate_tables(const moqae_config* cfg, const moqae_cache* cache, int32_t T,
+                          int32_t layer_group, void* stream, int32_t* bad_row, int32_t* bad_chunk);
 
 /*
  * Synchronous read of the cache's device status word: *out_status (host) receives MOQAE_OK

@@ -21,12 +21,14 @@ DT_FP16, DT_BF16 = 0, 1
 OK = 0
 ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_MISALIGNED, ERR_POOL_FULL = -1, -2, -3, -4
 ERR_WORKSPACE_TOO_SMALL, ERR_CUDA, ERR_TIMEOUT = -5, -6, -7
+ERR_CORRUPT_TABLE = -8
 
 EXPORTS = ["moqae_version", "moqae_last_cuda_error", "moqae_error_string", "moqae_cache_bytes",
            "moqae_cache_bind", "moqae_route", "moqae_quantize_kv", "moqae_append_kv",
            "moqae_decode_attn_workspace", "moqae_decode_attn", "moqae_poll_status",
            "moqae_decode_attn_static", "moqae_decode_attn_static_max_bytes", "moqae_flush_tail", "moqae_prefill_attn",
-           "moqae_prefill_attn_workspace", "moqae_decode_attn_ex", "moqae_project_quantize_kv"]
+           "moqae_prefill_attn_workspace", "moqae_decode_attn_ex", "moqae_project_quantize_kv",
+           "moqae_validate_tables", "moqae_validate_tables_host"]
 
 
 class MoqaeConfig(C.Structure):
@@ -98,6 +100,10 @@ def lib() -> C.CDLL:
         L.moqae_decode_attn_ex.argtypes = [C.POINTER(MoqaeConfig), C.c_void_p, C.c_int32, C.POINTER(MoqaeCache),
                                            C.c_void_p, C.c_float, C.c_void_p, C.c_int64, C.c_int32, C.c_void_p]
         L.moqae_poll_status.argtypes = [C.POINTER(MoqaeCache), C.c_void_p, C.POINTER(C.c_int32)]
+        L.moqae_validate_tables.argtypes = [C.POINTER(MoqaeConfig), C.POINTER(MoqaeCache), C.c_int32, C.c_int32,
+                                            C.c_void_p, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
+        L.moqae_validate_tables_host.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
+                                                 C.POINTER(C.c_int64), C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
         L.moqae_decode_attn_static.argtypes = [C.POINTER(MoqaeConfig), C.c_void_p, C.c_int32,
                                                C.POINTER(MoqaeCache), C.c_void_p, C.c_float, C.c_void_p]
         L.moqae_decode_attn_static_max_bytes.argtypes = []
@@ -296,6 +302,30 @@ def moqae_decode_attn_static(cfg, q, layer, cache: Cache, out, scale=0.0):
     device memory, the split partials live in a fixed array inside the library."""
     _check(lib().moqae_decode_attn_static(C.byref(cfg), _ptr(q), int(layer), C.byref(cache.view), _ptr(out),
                                           C.c_float(scale), _stream()), "moqae_decode_attn_static")
+
+
+def moqae_validate_tables(cfg, cache: Cache, T, layer_group=0):
+    """(code, bad_row, bad_chunk): OK, or ERR_CORRUPT_TABLE with the first offending position."""
+    r, c = C.c_int32(-1), C.c_int32(-1)
+    rc = lib().moqae_validate_tables(C.byref(cfg), C.byref(cache.view), int(T), int(layer_group), _stream(),
+                                     C.byref(r), C.byref(c))
+    if rc not in (OK, ERR_CORRUPT_TABLE):
+        raise MoqaeError(rc, "moqae_validate_tables")
+    return rc, int(r.value), int(c.value)
+
+
+def moqae_validate_tables_host(map_u8, slot_i32, count_i32, n_chunks, capacity):
+    """The same check on host numpy arrays map / slot [rows, max_chunks] and count [rows, 4]."""
+    import numpy as np
+    m = np.ascontiguousarray(map_u8, dtype=np.uint8)
+    s = np.ascontiguousarray(slot_i32, dtype=np.int32)
+    k = np.ascontiguousarray(count_i32, dtype=np.int32)
+    cap = (C.c_int64 * 4)(*[int(x) for x in capacity])
+    r, c = C.c_int32(-1), C.c_int32(-1)
+    rc = lib().moqae_validate_tables_host(m.ctypes.data_as(C.c_void_p), s.ctypes.data_as(C.c_void_p),
+                                          k.ctypes.data_as(C.c_void_p), m.shape[0], m.shape[1], int(n_chunks), cap,
+                                          C.byref(r), C.byref(c))
+    return rc, int(r.value), int(c.value)
 
 
 def moqae_poll_status(cache: Cache) -> int:

@@ -1,5 +1,6 @@
 // C ABI of the library: argument validation and dispatch to the kernel launchers.
 #include <atomic>
+#include <vector>
 
 #include "common.cuh"
 
@@ -114,6 +115,7 @@ const char* moqae_error_string(int code) {
     case MOQAE_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
     case MOQAE_ERR_CUDA: return "CUDA runtime error (see moqae_last_cuda_error)";
     case MOQAE_ERR_TIMEOUT: return "bounded device wait expired";
+    case MOQAE_ERR_CORRUPT_TABLE: return "chunk index table breaks the slot rules";
     default: return "unknown error";
   }
 }
@@ -329,6 +331,54 @@ int moqae_prefill_attn(const moqae_config* cfg, const void* q, int32_t T, int32_
   if (!(scale > 0.0f)) scale = 0.08838834764831845f;   // 1/sqrt(128)
   cudaError_t e = moqae::launch_prefill_attn(dims_of(cfg), cv, q, T, layer, scale, out, workspace, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? MOQAE_OK : cuda_fail(e);
+}
+
+int moqae_validate_tables_host(const uint8_t* map, const int32_t* slot, const int32_t* count, int32_t rows,
+                               int32_t max_chunks, int32_t n_chunks, const int64_t capacity[4], int32_t* bad_row,
+                               int32_t* bad_chunk) {
+  if (!map || !slot || !count || !capacity || rows < 0 || n_chunks < 0 || n_chunks > max_chunks) return MOQAE_ERR_INVALID_ARG;
+  auto fail = [&](int r, int c) {
+    if (bad_row) *bad_row = r;
+    if (bad_chunk) *bad_chunk = c;
+    return MOQAE_ERR_CORRUPT_TABLE;
+  };
+  for (int r = 0; r < rows; ++r) {
+    int64_t seen[4] = {0, 0, 0, 0};
+    for (int c = 0; c < n_chunks; ++c) {
+      const int w = map[static_cast<int64_t>(r) * max_chunks + c];
+      if (w > 3) return fail(r, c);
+      const int32_t s = slot[static_cast<int64_t>(r) * max_chunks + c];
+      if (s != seen[w] || s >= capacity[w]) return fail(r, c);
+      seen[w]++;
+    }
+    for (int w = 0; w < 4; ++w)
+      if (count[4 * r + w] != seen[w]) return fail(r, -1);
+  }
+  return MOQAE_OK;
+}
+
+int moqae_validate_tables(const moqae_config* cfg, const moqae_cache* cache, int32_t T, int32_t layer_group,
+                          void* stream, int32_t* bad_row, int32_t* bad_chunk) {
+  int rc = check_config(cfg);
+  if (rc != MOQAE_OK) return rc;
+  moqae::CacheView cv;
+  rc = check_cache(cache, &cv);
+  if (rc != MOQAE_OK) return rc;
+  if (T < 0 || T > cfg->max_tokens || layer_group < 0 || layer_group >= n_groups(cfg)) return MOQAE_ERR_INVALID_ARG;
+  const moqae::Dims dm = dims_of(cfg);
+  const int64_t rows = dm.n_tseq, mc = dm.max_chunks;
+  std::vector<uint8_t> map(static_cast<size_t>(rows * mc));
+  std::vector<int32_t> slot(static_cast<size_t>(rows * mc)), count(static_cast<size_t>(rows * 4));
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  cudaError_t e = cudaMemcpyAsync(map.data(), cv.map + layer_group * rows * mc, map.size(), cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(slot.data(), cv.slot + layer_group * rows * mc, slot.size() * 4, cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(count.data(), cv.count + layer_group * rows * 4, count.size() * 4, cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) return cuda_fail(e);
+  return moqae_validate_tables_host(map.data(), slot.data(), count.data(), static_cast<int32_t>(rows), static_cast<int32_t>(mc),
+                                    T / cfg->chunk, cache->capacity, bad_row, bad_chunk);
 }
 
 int moqae_poll_status(const moqae_cache* cache, void* stream, int32_t* out_status) {

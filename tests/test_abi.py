@@ -79,3 +79,27 @@ def test_host_side_argument_errors(lib):
     bufs[2] = 4097
     cap = (ctypes.c_int64 * 4)(1, 1, 1, 1)
     assert lib.moqae_cache_bind(ctypes.byref(ok), cap, bufs, ctypes.byref(cache)) == mq.ERR_MISALIGNED
+
+
+def test_table_validator_on_host_arrays(lib):
+    """The index-table checker (host arithmetic, no GPU): tables made by the oracle's slot rule pass;
+    a wrong slot, a slot beyond its pool, an unknown width and a wrong count are each reported at
+    their position."""
+    import numpy as np
+    from oracle import moqae_oracle as O
+    rs = np.random.RandomState(0)
+    bmap = rs.randint(0, 4, size=(3, 40)).astype(np.uint8)
+    slot, count = O.assign_slots(bmap)
+    cap = [int(count[:, w].max()) for w in range(4)]
+    assert mq.moqae_validate_tables_host(bmap, slot, count, 40, cap)[0] == mq.OK
+    assert mq.moqae_validate_tables_host(bmap, slot, np.zeros_like(count), 0, cap)[0] == mq.OK      # an empty context
+    bad = slot.copy(); bad[1, 17] += 1
+    assert mq.moqae_validate_tables_host(bmap, bad, count, 40, cap) == (mq.ERR_CORRUPT_TABLE, 1, 17)
+    assert mq.moqae_validate_tables_host(bmap, bad, count, 17, cap)[0] == mq.ERR_CORRUPT_TABLE     # count row no longer fits
+    small = list(cap); small[int(bmap[2, 39])] = int(slot[2, 39])                                  # last chunk's slot == capacity
+    rc, r, c = mq.moqae_validate_tables_host(bmap, slot, count, 40, small)
+    assert rc == mq.ERR_CORRUPT_TABLE and c >= 0
+    m2 = bmap.copy(); m2[0, 3] = 7
+    assert mq.moqae_validate_tables_host(m2, slot, count, 40, cap) == (mq.ERR_CORRUPT_TABLE, 0, 3)
+    k2 = count.copy(); k2[2, 1] += 1
+    assert mq.moqae_validate_tables_host(bmap, slot, k2, 40, cap) == (mq.ERR_CORRUPT_TABLE, 2, -1)

@@ -156,3 +156,17 @@ def test_three_expert_set_through_a_masked_logit():
     n_frag, n_chunks, m = check_route(2, chunk * 12 + 9, D, chunk, dtype, True, True, seed=90,
                                       weights=(W1_4, W2_4, W3_4, b_4), abs_margin=1e-3)
     assert not (m == 2).any() and len(np.unique(m)) > 1 and n_frag < n_chunks // 2
+
+
+def test_table_validator_reports_a_corrupted_slot_table():
+    # tables written by the router pass the validator; one overwritten slot entry is found
+    B, T, D, chunk = 2, 64 * 9 + 5, 64, 64
+    cfg = mq.make_config(n_layers=1, n_q_heads=2, n_kv_heads=2, chunk=chunk, dtype=1, d_in=D, max_tokens=T, batch=B)
+    cache = mq.moqae_cache_bind(cfg, [9, 9, 9, 9])
+    hid = synth.hidden_states(B, T, D, chunk, 1, 77, "cuda")
+    W1, W2, W3, b0 = synth.router_weights(D, 4, 1, 78, "cuda", std=0.2)
+    mq.moqae_route(cfg, hid, T, W1, W2, W3, b0, 0, cache)
+    assert mq.moqae_validate_tables(cfg, cache, T)[0] == mq.OK
+    cache.slot[0, 1, 4] += 3
+    assert mq.moqae_validate_tables(cfg, cache, T) == (mq.ERR_CORRUPT_TABLE, 1, 4)
+    assert mq.moqae_validate_tables(cfg, cache, 4 * chunk)[0] == mq.ERR_CORRUPT_TABLE      # the counts describe 9 chunks
