@@ -22,10 +22,9 @@
 // MOQAE_ERR_TIMEOUT, every role stops and the tensor memory is still freed.
 #include <cstring>
 
-#include <cuda.h>
 #include <cuda_bf16.h>
 
-#include "common.cuh"
+#include "ptx.cuh"
 
 namespace moqae {
 
@@ -33,20 +32,8 @@ namespace {
 
 constexpr int kQTile = 128;                    // query rows per CTA
 constexpr int kKvBlock = 128;                  // tokens per block (four storage tiles)
-constexpr long long kWaitCycles = 1ll << 31;    // about a second: no wait of a healthy launch comes near
-constexpr uint32_t kSuspendNs = 20000;         // how long one try_wait may keep the warp parked
+constexpr long long kPrefillWaitCycles = 1ll << 31;    // about a second: no wait of a healthy launch comes near
 
-__device__ __forceinline__ uint32_t smem_addr(const void* p) {
-  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-// One try_wait with a suspend-time hint: the warp is parked by the hardware until the phase
-// completes or the hint runs out, so a waiting role issues almost nothing.
-__device__ __forceinline__ bool mbar_try_wait_p(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\nselp.u32 %0, 1, 0, p;\n}\n"
-               : "=r"(ok) : "r"(bar), "r"(parity), "r"(kSuspendNs) : "memory");
-  return ok != 0;
-}
 // ---- tcgen05 wrappers -------------------------------------------------------------------
 // Shared-memory matrix descriptor, no swizzle: start address, leading-dimension byte offset
 // (between the two 8-element halves of a K step, or between groups of 8 K rows for an
@@ -353,9 +340,6 @@ constexpr int kQTileBytes = kQTile * 128 * 2;
 enum { BAR_KFULL = 0, BAR_VFULL = kStages, BAR_KFREE = 2 * kStages, BAR_VFREE = 3 * kStages,
        BAR_SFULL = 4 * kStages, BAR_PFULL = 4 * kStages + 2, BAR_OFULL = 4 * kStages + 4, BAR_COUNT = 4 * kStages + 6 };
 
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(bar) : "memory");
-}
 // 32 consecutive 32-bit columns of this thread's tensor-memory lane
 __device__ __forceinline__ void tmem_st32u(uint32_t taddr, const uint32_t (&v)[32]) {
   asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
@@ -462,14 +446,6 @@ __global__ void __launch_bounds__(64) prefill_dequant_kernel(Dims dm, CacheView 
   dequant_subtile<BF16, true>(ks, pos0, 0, warp != 0, dst, lane);
 }
 
-// tiled TMA load of the box whose corner is (x = channel, y = row) into a 128-byte swizzled tile
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
-  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];\n"
-               ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
-}
 // Descriptors of the 128-byte swizzled layouts TMA writes (bits 61..63 = 2).  K-major (K^: one
 // row of 64 channels = 128 bytes, 1 KiB between groups of 8 token rows; the leading offset is not
 // used) and MN-major (V^: 64 channels contiguous, 128 bytes between the 8 tokens of a group,
@@ -485,7 +461,7 @@ prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T
                     float* __restrict__ out, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                     int t_pad) {
   extern __shared__ __align__(128) uint8_t smem_raw[];
-  uint8_t* smem = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);   // swizzled tiles want 1 KiB alignment
+  uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);   // swizzled tiles want 1 KiB alignment
   uint8_t* sQ = smem;                               // two query tiles
   uint8_t* sK = sQ + 2 * kQTileBytes;               // kStages blocks
   uint8_t* sV = sK + kStages * kStageBytes;         // kStages blocks
@@ -494,7 +470,7 @@ prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   float* exch = reinterpret_cast<float*>(bar_mem + BAR_COUNT + 2);      // [256 rows][2 halves]
   volatile int* pair_flag = reinterpret_cast<volatile int*>(exch + 512);  // [2 block parities][8 pairs][2 halves]
-  const uint32_t bar0 = smem_addr(bar_mem);
+  const uint32_t bar0 = smem_u32(bar_mem);
   auto bar = [&](int i) { return bar0 + 8u * i; };
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -507,7 +483,7 @@ prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T
   const int nb0 = min(2 * pair + 1, nb_all), nb1 = min(2 * pair + 2, nb_all);
 
   if (warp == kIssueWarp) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_addr(tmem_slot)), "r"(kTmemCols2) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols2) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
   }
   if (tid == 0) {
@@ -537,11 +513,11 @@ prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T
   // bounded wait that also gives up when another role has given up
   auto wait = [&](int which, int completion) -> bool {
     const uint32_t a = bar(which), parity = static_cast<uint32_t>(completion) & 1u;
-    if (mbar_try_wait_p(a, parity)) return true;
+    if (mbar_try_wait(a, parity)) return true;
     const long long t0 = clock64();
     while (!*abort_flag) {
-      if (mbar_try_wait_p(a, parity)) return true;
-      if (clock64() - t0 > kWaitCycles) *abort_flag = 1;
+      if (mbar_try_wait(a, parity)) return true;
+      if (clock64() - t0 > kPrefillWaitCycles) *abort_flag = 1;
     }
     return false;
   };
@@ -792,7 +768,7 @@ prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T
         const int st = kb % kStages;
         if (kb >= kStages && !wait((is_v ? BAR_VFREE : BAR_KFREE) + st, kb / kStages - 1)) break;
         const uint32_t full = bar((is_v ? BAR_VFULL : BAR_KFULL) + st);
-        const uint32_t dst = smem_addr((is_v ? sV : sK) + st * kStageBytes);
+        const uint32_t dst = smem_u32((is_v ? sV : sK) + st * kStageBytes);
         mbar_expect_tx(full, kStageBytes);
         tma_load_2d(dst, map, 0, row0 + kb * kKvBlock, full);                    // channels 0..63
         tma_load_2d(dst + kStageBytes / 2, map, 64, row0 + kb * kKvBlock, full);  // channels 64..127
@@ -818,9 +794,9 @@ prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T
     // ================= MMA issue (one thread) =================
     // descriptors of stage 0, K step 0; a stage adds kStageBytes / 16 to the low word, a K step
     // (two 2 KiB slabs of 8 channels or 8 tokens) 256
-    const uint64_t qd = make_desc(smem_addr(sQ), 2048, 128);
-    const uint64_t kd = PRE ? make_desc_sw128(smem_addr(sK), 16, 1024) : make_desc(smem_addr(sK), 2048, 128);
-    const uint64_t vd = PRE ? make_desc_sw128(smem_addr(sV), kStageBytes / 2, 1024) : make_desc(smem_addr(sV), 2048, 128);
+    const uint64_t qd = make_desc(smem_u32(sQ), 2048, 128);
+    const uint64_t kd = PRE ? make_desc_sw128(smem_u32(sK), 16, 1024) : make_desc(smem_u32(sK), 2048, 128);
+    const uint64_t vd = PRE ? make_desc_sw128(smem_u32(sV), kStageBytes / 2, 1024) : make_desc(smem_u32(sV), 2048, 128);
     const uint32_t qd_lo = static_cast<uint32_t>(qd), qd_hi = static_cast<uint32_t>(qd >> 32);
     const uint32_t kd_lo = static_cast<uint32_t>(kd), kd_hi = static_cast<uint32_t>(kd >> 32);
     const uint32_t vd_lo = static_cast<uint32_t>(vd), vd_hi = static_cast<uint32_t>(vd >> 32);
@@ -882,21 +858,9 @@ prefill_attn_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ Q, int T
 
 }  // namespace
 
-// cuTensorMapEncodeTiled through the runtime's driver entry-point lookup (no link against libcuda)
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
 // [rows][128] fp16 rows, boxes of 64 channels x 128 rows, 128-byte swizzle
 static bool make_block_map(CUtensorMap* m, const void* base, long long rows) {
-  static EncodeTiledFn enc = [] {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
-        qres != cudaDriverEntryPointSuccess)
-      p = nullptr;
-    return reinterpret_cast<EncodeTiledFn>(p);
-  }();
+  EncodeTiledFn enc = encode_tiled_fn();
   if (!enc) return false;
   const cuuint64_t gdim[2] = {kHeadDim, static_cast<cuuint64_t>(rows)};
   const cuuint64_t gstride[1] = {kHeadDim * 2};

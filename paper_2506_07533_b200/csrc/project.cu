@@ -52,9 +52,6 @@ constexpr long long kProjWait = 1ll << 31;      // about a second of SM cycles
 
 enum { PB_FULL = 0, PB_EMPTY = kPStages, PB_ACC_FULL = 2 * kPStages, PB_ACC_EMPTY = 2 * kPStages + 2, PB_COUNT = 2 * kPStages + 4 };
 
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(bar) : "memory");
-}
 // Shared-memory matrix descriptor of a K-major operand tile in the 128-byte swizzled layout TMA
 // writes: rows of 128 bytes (64 elements), 1 KiB between groups of 8 rows; start address, leading
 // and stride byte offsets in units of 16 bytes, descriptor version 1 (bit 46), layout type 2
