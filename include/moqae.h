@@ -295,6 +295,21 @@ int moqae_decode_attn_ex(const moqae_config* cfg, const void* q, int32_t layer,
                          int64_t workspace_bytes, int32_t flags, void* stream);
 
 /*
+ * One generation step of a layer without touching the cache: moqae_decode_attn_ex that also
+ * attends to the CURRENT token's own key / value rows k_new, v_new [batch][n_kv_heads][128]
+ * (input dtype), taken as the 16-bit row that would follow the tail (Section 3.2: tokens that do
+ * not fill a chunk stay 16-bit).  The result equals moqae_append_kv followed by
+ * moqae_decode_attn, but nothing is written to the cache, so the call reads nothing a previous
+ * decode call writes and a whole step (layer after layer) can be chained with
+ * MOQAE_DECODE_OVERLAP_PREVIOUS; the rows are appended afterwards with moqae_append_kv, at any
+ * time before the layer's next step.  k_new = v_new = NULL gives moqae_decode_attn_ex.
+ */
+int moqae_decode_attn_step(const moqae_config* cfg, const void* q, const void* k_new,
+                           const void* v_new, int32_t layer, const moqae_cache* cache, float* out,
+                           float scale, void* workspace, int64_t workspace_bytes, int32_t flags,
+                           void* stream);
+
+/*
  * Causal attention of the prompt over its own quantised cache (Section 3.1: a block quantises
  * its chunks, then carries out its attention; Limitations section: keys are dequantised to
  * 16-bit floats before the product with the query).  For every position t < T and query head h

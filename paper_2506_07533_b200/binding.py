@@ -28,7 +28,7 @@ EXPORTS = ["moqae_version", "moqae_last_cuda_error", "moqae_error_string", "moqa
            "moqae_decode_attn_workspace", "moqae_decode_attn", "moqae_poll_status",
            "moqae_decode_attn_static", "moqae_decode_attn_static_max_bytes", "moqae_flush_tail", "moqae_prefill_attn",
            "moqae_prefill_attn_workspace", "moqae_decode_attn_ex", "moqae_project_quantize_kv",
-           "moqae_validate_tables", "moqae_validate_tables_host"]
+           "moqae_validate_tables", "moqae_validate_tables_host", "moqae_decode_attn_step"]
 
 
 class MoqaeConfig(C.Structure):
@@ -99,6 +99,9 @@ def lib() -> C.CDLL:
                                         C.c_void_p, C.c_float, C.c_void_p, C.c_int64, C.c_void_p]
         L.moqae_decode_attn_ex.argtypes = [C.POINTER(MoqaeConfig), C.c_void_p, C.c_int32, C.POINTER(MoqaeCache),
                                            C.c_void_p, C.c_float, C.c_void_p, C.c_int64, C.c_int32, C.c_void_p]
+        L.moqae_decode_attn_step.argtypes = [C.POINTER(MoqaeConfig), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
+                                             C.POINTER(MoqaeCache), C.c_void_p, C.c_float, C.c_void_p, C.c_int64,
+                                             C.c_int32, C.c_void_p]
         L.moqae_poll_status.argtypes = [C.POINTER(MoqaeCache), C.c_void_p, C.POINTER(C.c_int32)]
         L.moqae_validate_tables.argtypes = [C.POINTER(MoqaeConfig), C.POINTER(MoqaeCache), C.c_int32, C.c_int32,
                                             C.c_void_p, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
@@ -291,6 +294,15 @@ def moqae_decode_attn_ex(cfg, q, layer, cache: Cache, out, workspace, flags=0, s
     _check(lib().moqae_decode_attn_ex(C.byref(cfg), _ptr(q), int(layer), C.byref(cache.view), _ptr(out),
                                       C.c_float(scale), _ptr(workspace), int(workspace.numel() * workspace.element_size()),
                                       int(flags), _stream()), "moqae_decode_attn_ex")
+
+
+def moqae_decode_attn_step(cfg, q, k_new, v_new, layer, cache: Cache, out, workspace, flags=0, scale=0.0):
+    """Decode attention that also attends to the current token's own rows k_new / v_new (not yet in the
+    cache); append them afterwards with moqae_append_kv."""
+    _check(lib().moqae_decode_attn_step(C.byref(cfg), _ptr(q), _ptr(k_new), _ptr(v_new), int(layer), C.byref(cache.view),
+                                        _ptr(out), C.c_float(scale), _ptr(workspace),
+                                        int(workspace.numel() * workspace.element_size()), int(flags), _stream()),
+           "moqae_decode_attn_step")
 
 
 def moqae_decode_attn_static_max_bytes() -> int:

@@ -289,7 +289,15 @@ int moqae_decode_attn(const moqae_config* cfg, const void* q, int32_t layer, con
 int moqae_decode_attn_ex(const moqae_config* cfg, const void* q, int32_t layer, const moqae_cache* cache,
                          float* out, float scale, void* workspace, int64_t workspace_bytes, int32_t flags,
                          void* stream) {
+  return moqae_decode_attn_step(cfg, q, nullptr, nullptr, layer, cache, out, scale, workspace, workspace_bytes, flags, stream);
+}
+
+int moqae_decode_attn_step(const moqae_config* cfg, const void* q, const void* k_new, const void* v_new, int32_t layer,
+                           const moqae_cache* cache, float* out, float scale, void* workspace, int64_t workspace_bytes,
+                           int32_t flags, void* stream) {
   if (flags & ~MOQAE_DECODE_OVERLAP_PREVIOUS) return MOQAE_ERR_INVALID_ARG;
+  if ((k_new == nullptr) != (v_new == nullptr)) return MOQAE_ERR_INVALID_ARG;
+  if (!aligned16(k_new) || !aligned16(v_new)) return MOQAE_ERR_MISALIGNED;
   int rc = check_config(cfg);
   if (rc != MOQAE_OK) return rc;
   moqae::CacheView cv;
@@ -303,7 +311,8 @@ int moqae_decode_attn_ex(const moqae_config* cfg, const void* q, int32_t layer, 
   if (workspace_bytes < need) return MOQAE_ERR_WORKSPACE_TOO_SMALL;
   if (!(scale > 0.0f)) scale = 0.08838834764831845f;   // 1/sqrt(128)
   cudaError_t e = moqae::launch_decode(dm, cv, q, layer, out, scale, static_cast<float*>(workspace), s,
-                                       (flags & MOQAE_DECODE_OVERLAP_PREVIOUS) != 0, static_cast<cudaStream_t>(stream));
+                                       (flags & MOQAE_DECODE_OVERLAP_PREVIOUS) != 0, k_new, v_new,
+                                       static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? MOQAE_OK : cuda_fail(e);
 }
 

@@ -106,8 +106,9 @@ long long decode_workspace_bytes(const Dims& dm, int n_splits);
 void decode_counter_region(const moqae_config* cfg, long long* offset, long long* bytes);
 cudaError_t launch_decode_mma(const Dims& dm, const CacheView& cv, const void* q, int layer, float scale,
                               float* ws_o, float* ws_ml, int* arrived, float* out, int n_splits, bool overlap_previous,
-                              cudaStream_t st);
+                              const void* k_new, const void* v_new, cudaStream_t st);
 cudaError_t launch_decode(const Dims& dm, const CacheView& cv, const void* q, int layer, float* out,
-                          float scale, float* workspace, int n_splits, bool overlap_previous, cudaStream_t st);
+                          float scale, float* workspace, int n_splits, bool overlap_previous, const void* k_new,
+                          const void* v_new, cudaStream_t st);
 
 }  // namespace moqae

@@ -42,14 +42,15 @@ void decode_counter_region(const moqae_config* cfg, long long* offset, long long
 }
 
 cudaError_t launch_decode(const Dims& dm, const CacheView& cv, const void* q, int layer, float* out,
-                          float scale, float* workspace, int n_splits, bool overlap_previous, cudaStream_t st) {
+                          float scale, float* workspace, int n_splits, bool overlap_previous, const void* k_new,
+                          const void* v_new, cudaStream_t st) {
   const long long rows = static_cast<long long>(dm.batch) * dm.n_q_heads * n_splits;
   float* ws_o = workspace;
   float* ws_ml = workspace + rows * kHeadDim;
   int* arrived = reinterpret_cast<int*>(ws_ml + rows * 2);
   // the counters are zero on entry (the caller zeroes a new workspace once) and the kernel
   // leaves them zero: the last arrival of every (sequence, kv head) wraps its counter around
-  return launch_decode_mma(dm, cv, q, layer, scale, ws_o, ws_ml, arrived, out, n_splits, overlap_previous, st);
+  return launch_decode_mma(dm, cv, q, layer, scale, ws_o, ws_ml, arrived, out, n_splits, overlap_previous, k_new, v_new, st);
 }
 
 }  // namespace moqae

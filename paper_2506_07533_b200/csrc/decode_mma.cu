@@ -565,7 +565,8 @@ template <bool BF16, bool G4>
 __global__ void __launch_bounds__(kThreads, 2)
 decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int layer, float scale,
                   float* __restrict__ ws_o, float* __restrict__ ws_ml, int* __restrict__ arrived,
-                  float* __restrict__ out, int n_splits) {
+                  float* __restrict__ out, int n_splits, const uint16_t* __restrict__ k_new,
+                  const uint16_t* __restrict__ v_new) {
   extern __shared__ __align__(128) uint8_t smem[];
   uint8_t* rings = smem;                                              // kWarps * kRingBytes
   uint16_t* q_in = reinterpret_cast<uint16_t*>(smem + kWarps * kRingBytes);        // [8][128] input dtype
@@ -734,7 +735,11 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
   }
   // ---- 16-bit tail (last split, warp 0): rows are staged by hand, swizzled, zero padded
   if (split == n_splits - 1 && warp == 0 && pp.ok) {
-    const int len = cv.tail_len[layer * dm.batch + b];
+    // k_new / v_new (optional): the current token's own rows, attended to as the row after the tail
+    // without being in the cache yet
+    const int tail_rows = cv.tail_len[layer * dm.batch + b];
+    const int len = tail_rows + (k_new ? 1 : 0);
+    const long long nbase = (static_cast<long long>(b) * dm.n_kv_heads + h) * kHeadDim;
     const long long tbase = ((static_cast<long long>(layer) * dm.batch + b) * dm.n_kv_heads + h) * dm.tail_capacity * kHeadDim;
     uint8_t* stg = rings;    // warp 0's ring; all its bulk copies have completed
     phase_scale<16>(st, true);
@@ -745,9 +750,12 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
         const int row = i >> 4, U = i & 15;
         const int up = (U & 8) | ((U ^ row) & 7);
         uint4 kv = make_uint4(0u, 0u, 0u, 0u), vv = kv;
-        if (row < nv) {
+        if (t0 + row < tail_rows) {
           kv = *reinterpret_cast<const uint4*>(cv.tail_k + tbase + static_cast<long long>(t0 + row) * kHeadDim + 8 * U);
           vv = *reinterpret_cast<const uint4*>(cv.tail_v + tbase + static_cast<long long>(t0 + row) * kHeadDim + 8 * U);
+        } else if (row < nv) {
+          kv = *reinterpret_cast<const uint4*>(k_new + nbase + 8 * U);
+          vv = *reinterpret_cast<const uint4*>(v_new + nbase + 8 * U);
         }
         *reinterpret_cast<uint4*>(stg + row * 256 + up * 16) = kv;
         *reinterpret_cast<uint4*>(stg + 4096 + row * 256 + up * 16) = vv;
@@ -838,7 +846,7 @@ int decode_mma_ctas_per_sm() { return 2; }
 
 cudaError_t launch_decode_mma(const Dims& dm, const CacheView& cv, const void* q, int layer, float scale,
                               float* ws_o, float* ws_ml, int* arrived, float* out, int n_splits, bool overlap_previous,
-                              cudaStream_t st) {
+                              const void* k_new, const void* v_new, cudaStream_t st) {
   const size_t smem = static_cast<size_t>(kWarps) * kRingBytes + 2 * kQBytes + kWarps * 6 * 8;
   const bool g4 = dm.n_q_heads / dm.n_kv_heads <= 4;
   auto launch = [&](auto kernel) -> cudaError_t {
@@ -858,7 +866,7 @@ cudaError_t launch_decode_mma(const Dims& dm, const CacheView& cv, const void* q
     lc.attrs = attr;
     lc.numAttrs = overlap_previous ? 1 : 0;
     return cudaLaunchKernelEx(&lc, kernel, dm, cv, static_cast<const uint16_t*>(q), layer, scale, ws_o, ws_ml, arrived, out,
-                              n_splits);
+                              n_splits, static_cast<const uint16_t*>(k_new), static_cast<const uint16_t*>(v_new));
   };
   cudaError_t e;
   if (dm.dtype == MOQAE_DTYPE_BF16) e = g4 ? launch(decode_mma_kernel<true, true>) : launch(decode_mma_kernel<true, false>);

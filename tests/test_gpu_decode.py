@@ -193,6 +193,57 @@ def test_append_then_decode_matches_oracle_with_longer_tail():
     assert mq.moqae_poll_status(cache) == 0
 
 
+def test_generation_steps_attend_to_the_new_token_before_it_is_appended():
+    # moqae_decode_attn_step: the current token's K/V rows take part in the attention without being in the
+    # cache; the layers of a step are chained (each launch may overlap the previous one), the appends follow
+    # the step.  After every step the outputs equal the oracle on "cache + tail + the new token".
+    B, Hq, Hkv, chunk, dtype, L = 2, 4, 2, 64, 1, 3
+    T = 64 * 3 + 7
+    cfg = mq.make_config(n_layers=L, n_q_heads=Hq, n_kv_heads=Hkv, chunk=chunk, dtype=dtype, d_in=64,
+                         max_tokens=T + chunk, batch=B)
+    cache = mq.moqae_cache_bind(cfg, [3, 3, 3, 3], zero_pools=True)
+    KV, maps = [], []
+    for l in range(L):
+        K, V = H.make_kv(B, T + 6, Hkv, dtype, 950 + l)
+        bmap = np.random.RandomState(950 + l).randint(0, 4, size=(B, T // chunk)).astype(np.uint8)
+        mq.moqae_quantize_kv(cfg, K[:, :T].contiguous().cuda(), V[:, :T].contiguous().cuda(), T, l, cache,
+                             forced_map=torch.from_numpy(bmap).cuda())
+        KV.append((K, V))
+        maps.append(bmap)
+    torch.cuda.synchronize()
+    ws = torch.zeros(mq.moqae_decode_attn_workspace(cfg), dtype=torch.uint8, device="cuda")
+    out = torch.full((L, B, Hq, 128), float("nan"), dtype=torch.float32, device="cuda")
+    for step in range(6):
+        qs = [synth.normal((B, Hq, 128), dtype, 970 + 10 * step + l, "cpu") for l in range(L)]
+        new = [(KV[l][0][:, T + step].contiguous().cuda(), KV[l][1][:, T + step].contiguous().cuda()) for l in range(L)]
+        qd = [x.cuda() for x in qs]
+        torch.cuda.synchronize()
+        for l in range(L):
+            mq.moqae_decode_attn_step(cfg, qd[l], new[l][0], new[l][1], l, cache, out[l], ws,
+                                      flags=mq.DECODE_OVERLAP_PREVIOUS if l > 0 else 0)
+        for l in range(L):
+            mq.moqae_append_kv(cfg, new[l][0], new[l][1], l, cache)
+        torch.cuda.synchronize()
+        n = T + step + 1
+        for l in range(L):
+            K, V = KV[l]
+            ocache = O.quantize_kv(synth.to_u16(K[:, :n]), synth.to_u16(V[:, :n]), dtype, chunk, maps[l])
+            assert ocache["tail_len"] == 7 + step + 1
+            ok, e_abs, e_rel = H.attn_tolerance_ok(out[l].cpu().numpy(), O.decode_attn(synth.to_u16(qs[l]), dtype, ocache, chunk))
+            assert ok, (step, l, e_abs, e_rel)
+        assert (cache.tail_len.cpu().numpy() == 7 + step + 1).all()
+    assert mq.moqae_poll_status(cache) == 0
+    # an empty cache plus the new token: the output is that token's value row
+    cfg1 = mq.make_config(n_layers=1, n_q_heads=2, n_kv_heads=1, chunk=32, dtype=0, d_in=64, max_tokens=32, batch=1)
+    c1 = mq.moqae_cache_bind(cfg1, [1, 1, 1, 1])
+    k1, v1 = synth.normal((1, 1, 128), 0, 1, "cuda"), synth.normal((1, 1, 128), 0, 2, "cuda")
+    o1 = torch.full((1, 2, 128), float("nan"), dtype=torch.float32, device="cuda")
+    w1 = torch.zeros(mq.moqae_decode_attn_workspace(cfg1), dtype=torch.uint8, device="cuda")
+    mq.moqae_decode_attn_step(cfg1, synth.normal((1, 2, 128), 0, 3, "cuda"), k1, v1, 0, c1, o1, w1)
+    torch.cuda.synchronize()
+    assert torch.allclose(o1[0, 0], v1[0, 0].float(), atol=2e-3) and torch.allclose(o1[0, 1], v1[0, 0].float(), atol=2e-3)
+
+
 def test_decode_is_deterministic_and_leaves_neighbours_alone():
     # same call twice -> identical bits; bytes around `out` are never touched
     B, T, Hq, Hkv, chunk, dtype = 2, 64 * 5 + 9, 8, 2, 64, 1
