@@ -192,7 +192,10 @@ __device__ __forceinline__ void encode_values(const uint8_t* __restrict__ in, ui
       if (t >= n_valid) {                      // padding token: scale 0, zero 0, every code 0
         sb = 0; zb = 0; zf = 0.0f; inv = 0.0f;
       }
-      prm[32 * cg + t] = make_float4(-zf, -zf, inv, inv);       // [group][token]: neighbouring lanes, neighbouring banks
+      // [token][group], the four groups of a token rotated by t / 2: the 32 lanes of this store spread evenly
+      // over the eight 16-byte bank groups, and the four entries of one token that the encode pass reads in
+      // one load sit in one 64-byte row
+      prm[4 * t + ((cg + (t >> 1)) & 3)] = make_float4(-zf, -zf, inv, inv);
       meta[256 + ((((blk * 2 + (cg >> 1)) * 4 + t4) * 4 + (cg & 1) * 2 + half) * 2) + e] = sb;
       meta[384 + ((((blk * 4 + cg) * 4 + t4) * 2 + half) * 2) + e] = zb;
     }
@@ -202,7 +205,9 @@ __device__ __forceinline__ void encode_values(const uint8_t* __restrict__ in, ui
   const int p = lane >> 3, g = lane & 7;
   const uint2* rows = reinterpret_cast<const uint2*>(in) + lane;
   uint8_t* pay = pay_at ? pay_at : out + kMetaBytes + kTileTokens * 16 * BITS;
-#pragma unroll
+  // not unrolled over the two halves: the kernel's warps sit in different phases of different widths, and
+  // keeping their code small enough for the instruction cache is worth more than the longer basic block
+#pragma unroll 1
   for (int blk = 0; blk < 2; ++blk) {
 #pragma unroll
     for (int t4 = 0; t4 < 4; ++t4) {
@@ -211,7 +216,7 @@ __device__ __forceinline__ void encode_values(const uint8_t* __restrict__ in, ui
       for (int bp = 0; bp < 4; ++bp) {
         const int t = 16 * blk + 8 * (bp & 1) + 2 * t4 + (bp >> 1);
         const uint2 w = rows[32 * t];
-        const ulonglong2 zi = *reinterpret_cast<const ulonglong2*>(prm + 32 * p + t);   // (-z, -z), (inv, inv)
+        const ulonglong2 zi = *reinterpret_cast<const ulonglong2*>(prm + 4 * t + ((p + (t >> 1)) & 3));   // (-z, -z), (inv, inv)
         encode2<BF16>(w.x, zi.x, zi.y, u[bp][0], u[bp][1]);
         encode2<BF16>(w.y, zi.x, zi.y, u[bp][2], u[bp][3]);
         if (t >= n_valid) {                    // padding token: code 0 whatever the row holds

@@ -33,7 +33,9 @@ struct TileRef {
   int w, slot;         // routed width and slot of the tile's chunk
 };
 
-template <bool BF16>
+// FULL: every tile holds 32 tokens (chunk >= 32).  Chunks of 8 or 16 tokens get their own instantiation, so that
+// the padding-row variants of the encoders do not take instruction-cache space in the ordinary kernel.
+template <bool BF16, bool FULL>
 __global__ void __launch_bounds__(kQWarps * 32, 2)
 quantize_pack_kernel(Dims dm, CacheView cv, const __grid_constant__ CUtensorMap mapK,
                      const __grid_constant__ CUtensorMap mapV, int T, int layer, long long n_tiles, int flush) {
@@ -55,7 +57,7 @@ quantize_pack_kernel(Dims dm, CacheView cv, const __grid_constant__ CUtensorMap 
   const int H = dm.n_kv_heads;
   const int tpc = tiles_per_chunk_of(dm.chunk);
   const int n_valid = tile_tokens_of(dm.chunk);      // rows of a tile that hold tokens (a short chunk: the rest is padding)
-  const bool full = n_valid == kTileTokens;
+  constexpr bool full = FULL;
   const int C = T / dm.chunk;
   const long long stride = static_cast<long long>(gridDim.x) * kQWarps;
   const int group = layer / dm.rs_group;
@@ -63,17 +65,42 @@ quantize_pack_kernel(Dims dm, CacheView cv, const __grid_constant__ CUtensorMap 
   const int32_t* slot_g = cv.slot + static_cast<long long>(group) * dm.n_tseq * dm.max_chunks;
 
   const int32_t* count_g = cv.count + static_cast<long long>(group) * dm.batch * 4;
-  auto tile_ref = [&](long long id) {
-    // id = ((b * C + c) * tpc + j) * H + h : heads fastest, so neighbouring warps read
-    // neighbouring 256-byte segments of the same token rows
-    TileRef r;
-    r.h = static_cast<int>(id % H);
+  // Tile id = ((b * Cd + c) * tpc + j) * H + h (heads fastest, so neighbouring warps read neighbouring
+  // 256-byte segments of the same token rows); Cd = chunks per sequence (1 for a flush: one chunk per
+  // sequence).  The id is taken apart by division once per warp; after that the four digits advance by
+  // the digits of the grid stride with carries, which costs a dozen instructions per tile instead of
+  // three 64-bit divisions.
+  struct TilePos { int h, j, c, b; };
+  const int Cd = flush ? 1 : C;
+  auto split_id = [&](long long id) {
+    TilePos p;
+    p.h = static_cast<int>(id % H);
     long long x = id / H;
-    r.j = static_cast<int>(x % tpc);
+    p.j = static_cast<int>(x % tpc);
     x /= tpc;
+    p.c = static_cast<int>(x % Cd);
+    p.b = static_cast<int>(x / Cd);
+    return p;
+  };
+  auto advance = [&](TilePos& p, const TilePos& d) {
+    p.h += d.h;
+    int carry = p.h >= H ? 1 : 0;
+    p.h -= carry * H;
+    p.j += d.j + carry;
+    carry = p.j >= tpc ? 1 : 0;
+    p.j -= carry * tpc;
+    p.c += d.c + carry;
+    carry = p.c >= Cd ? 1 : 0;
+    p.c -= carry * Cd;
+    p.b += d.b + carry;
+  };
+  auto tile_ref = [&](const TilePos& p) {
+    TileRef r;
+    r.h = p.h;
+    r.j = p.j;
     if (!flush) {
-      const int c = static_cast<int>(x % C);
-      r.b = static_cast<int>(x / C);
+      const int c = p.c;
+      r.b = p.b;
       r.x = r.h * kHeadDim;
       r.y = r.b * T + c * dm.chunk + r.j * kTileTokens;
       const long long tbl = static_cast<long long>(table_row(dm, r.b, r.h)) * dm.max_chunks + c;
@@ -82,7 +109,7 @@ quantize_pack_kernel(Dims dm, CacheView cv, const __grid_constant__ CUtensorMap 
     } else {
       // flush of a full tail: the source is the tail itself ([layer][b][h][row][128]); the target is
       // the sequence's newest chunk, marked with bit 7 in the map while its rows are being packed
-      r.b = static_cast<int>(x);
+      r.b = p.b;
       r.x = 0;
       r.y = ((layer * dm.batch + r.b) * H + r.h) * dm.tail_capacity + r.j * kTileTokens;
       const int c = count_g[4 * r.b] + count_g[4 * r.b + 1] + count_g[4 * r.b + 2] + count_g[4 * r.b + 3] - 1;
@@ -105,7 +132,9 @@ quantize_pack_kernel(Dims dm, CacheView cv, const __grid_constant__ CUtensorMap 
 
   long long id = static_cast<long long>(blockIdx.x) * kQWarps + warp;
   if (id >= n_tiles) return;
-  TileRef cur = tile_ref(id);
+  TilePos pos = split_id(id);
+  const TilePos step = split_id(stride);
+  TileRef cur = tile_ref(pos);
   fetch(&mapK, cur, bufK, barK);
   fetch(&mapV, cur, bufV, barV);
   uint32_t parity = 0;
@@ -115,7 +144,10 @@ quantize_pack_kernel(Dims dm, CacheView cv, const __grid_constant__ CUtensorMap 
   for (; id < n_tiles; id += stride) {
     const long long next = id + stride;
     TileRef nxt = cur;
-    if (next < n_tiles) nxt = tile_ref(next);
+    if (next < n_tiles) {
+      advance(pos, step);
+      nxt = tile_ref(pos);
+    }
     const int w = cur.w, slot = cur.slot;
     long long cap = 0;
 #pragma unroll
@@ -136,7 +168,7 @@ quantize_pack_kernel(Dims dm, CacheView cv, const __grid_constant__ CUtensorMap 
     if (!mbar_wait_bounded(barK, parity)) { failed = 1; break; }
     if (valid) {
       if (w == 3) {
-        if (full) copy_raw_rows(bufK, tile, lane);
+        if constexpr (full) copy_raw_rows(bufK, tile, lane);
         else copy_raw_rows<true>(bufK, tile, lane, n_valid);
       } else {
         if (store_pending) {                  // the previous tile's bulk store must have read `out`
@@ -144,7 +176,7 @@ quantize_pack_kernel(Dims dm, CacheView cv, const __grid_constant__ CUtensorMap 
           __syncwarp();
           store_pending = false;
         }
-        if (full) {
+        if constexpr (full) {
           if (w == 0) encode_keys<2, BF16>(bufK, out, lane);
           else if (w == 1) encode_keys<4, BF16>(bufK, out, lane);
           else encode_keys<8, BF16>(bufK, out, lane);
@@ -162,9 +194,9 @@ quantize_pack_kernel(Dims dm, CacheView cv, const __grid_constant__ CUtensorMap 
     if (!mbar_wait_bounded(barV, parity)) { failed = 2; break; }
     if (valid) {
       if (w == 3) {
-        if (full) copy_raw_rows(bufV, tile + 8192, lane);
+        if constexpr (full) copy_raw_rows(bufV, tile + 8192, lane);
         else copy_raw_rows<true>(bufV, tile + 8192, lane, n_valid);
-      } else if (full) {
+      } else if constexpr (full) {
         if (w == 0) encode_values<2, BF16>(bufV, out, prm, lane);
         else if (w == 1) encode_values<4, BF16>(bufV, out, prm, lane);
         else encode_values<8, BF16>(bufV, out, prm, lane);
@@ -274,6 +306,28 @@ static bool make_tile_map(CUtensorMap* m, const void* base, long long rows, long
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+template <bool BF16, bool FULL>
+static cudaError_t launch_quantize_pack_t(const Dims& dm, const CacheView& cv, const CUtensorMap& mapK, const CUtensorMap& mapV,
+                                          int T, int layer, long long n_tiles, int flush, unsigned grid, size_t smem,
+                                          cudaStream_t st) {
+  const cudaError_t e = cudaFuncSetAttribute(quantize_pack_kernel<BF16, FULL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             static_cast<int>(smem));
+  if (e != cudaSuccess) return e;
+  quantize_pack_kernel<BF16, FULL><<<grid, kQWarps * 32, smem, st>>>(dm, cv, mapK, mapV, T, layer, n_tiles, flush);
+  return cudaGetLastError();
+}
+
+// one instantiation per (input dtype, whole tiles / chunks shorter than a tile)
+static cudaError_t launch_quantize_pack(const Dims& dm, const CacheView& cv, const CUtensorMap& mapK, const CUtensorMap& mapV,
+                                        int T, int layer, long long n_tiles, int flush, unsigned grid, size_t smem,
+                                        cudaStream_t st) {
+  const bool bf16 = dm.dtype == MOQAE_DTYPE_BF16, full = tile_tokens_of(dm.chunk) == kTileTokens;
+  if (bf16) return full ? launch_quantize_pack_t<true, true>(dm, cv, mapK, mapV, T, layer, n_tiles, flush, grid, smem, st)
+                        : launch_quantize_pack_t<true, false>(dm, cv, mapK, mapV, T, layer, n_tiles, flush, grid, smem, st);
+  return full ? launch_quantize_pack_t<false, true>(dm, cv, mapK, mapV, T, layer, n_tiles, flush, grid, smem, st)
+              : launch_quantize_pack_t<false, false>(dm, cv, mapK, mapV, T, layer, n_tiles, flush, grid, smem, st);
+}
+
 cudaError_t launch_quantize(const Dims& dm, const CacheView& cv, const void* K, const void* V, int T,
                             int layer, cudaStream_t st) {
   const int C = T / dm.chunk;
@@ -286,17 +340,7 @@ cudaError_t launch_quantize(const Dims& dm, const CacheView& cv, const void* K, 
     const long long want = (n_tiles + kQWarps - 1) / kQWarps;
     const long long cap = 2ll * sm_count();                    // two resident CTAs per SM, grid-stride
     const unsigned grid = static_cast<unsigned>(want < cap ? want : cap);
-    cudaError_t e;
-    if (dm.dtype == MOQAE_DTYPE_BF16) {
-      e = cudaFuncSetAttribute(quantize_pack_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-      if (e != cudaSuccess) return e;
-      quantize_pack_kernel<true><<<grid, kQWarps * 32, smem, st>>>(dm, cv, mapK, mapV, T, layer, n_tiles, 0);
-    } else {
-      e = cudaFuncSetAttribute(quantize_pack_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-      if (e != cudaSuccess) return e;
-      quantize_pack_kernel<false><<<grid, kQWarps * 32, smem, st>>>(dm, cv, mapK, mapV, T, layer, n_tiles, 0);
-    }
-    e = cudaGetLastError();
+    const cudaError_t e = launch_quantize_pack(dm, cv, mapK, mapV, T, layer, n_tiles, 0, grid, smem, st);
     if (e != cudaSuccess) return e;
   }
   dim3 g(8, dm.batch);
@@ -315,17 +359,7 @@ cudaError_t launch_flush_quantize(const Dims& dm, const CacheView& cv, int layer
   const long long want = (n_tiles + kQWarps - 1) / kQWarps;
   const long long cap = 2ll * sm_count();
   const unsigned grid = static_cast<unsigned>(want < cap ? want : cap);
-  cudaError_t e;
-  if (dm.dtype == MOQAE_DTYPE_BF16) {
-    e = cudaFuncSetAttribute(quantize_pack_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-    if (e != cudaSuccess) return e;
-    quantize_pack_kernel<true><<<grid, kQWarps * 32, smem, st>>>(dm, cv, mapK, mapV, 0, layer, n_tiles, 1);
-  } else {
-    e = cudaFuncSetAttribute(quantize_pack_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-    if (e != cudaSuccess) return e;
-    quantize_pack_kernel<false><<<grid, kQWarps * 32, smem, st>>>(dm, cv, mapK, mapV, 0, layer, n_tiles, 1);
-  }
-  return cudaGetLastError();
+  return launch_quantize_pack(dm, cv, mapK, mapV, 0, layer, n_tiles, 1, grid, smem, st);
 }
 
 // After every layer of the group has packed its rows: clear the marker and empty the tails.
