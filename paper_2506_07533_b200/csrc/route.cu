@@ -117,22 +117,28 @@ route_score_vote_kernel(Dims dm, int32_t* __restrict__ votes /* [batch][max_chun
     // b is the table row: a sequence, or with per-head routing (sequence, kv head) = (b / H, b % H)
     row = (dm.per_head ? b / dm.n_kv_heads : b) * T + c * dm.chunk + sub * 16;
   };
-  auto issue = [&](long long u) {       // lane 0: stage u of this warp's stream
-    const long long blk = blk0 + (u / n_stages) * blk_stride;
-    const int st = static_cast<int>(u % n_stages);
-    int b, c, row;
-    block_coords(blk, b, c, row);
-    const int slot = static_cast<int>(u % kStages);
-    const int box0 = st * kBoxesPerStage;
+  // Lane 0 issues the stages of this warp's stream in order; the cursor (block, stage, ring slot and the
+  // block's coordinates) moves along with it, so the divisions of block_coords run once per block and
+  // not once per stage.
+  long long ib_i = 0;
+  int st_i = 0, slot_i = 0, b_i = 0, c_i = 0, row_i = 0;
+  if (lane == 0 && my_blocks > 0) block_coords(blk0, b_i, c_i, row_i);
+  auto issue_next = [&]() {             // lane 0
+    const int box0 = st_i * kBoxesPerStage;
     const int nb = min(kBoxesPerStage, n_boxes - box0);
-    const uint32_t bar = smem_u32(bars + slot);
+    const uint32_t bar = smem_u32(bars + slot_i);
     mbar_expect_tx(bar, nb * kBoxBytes);
-    const int head = dm.per_head ? b % dm.n_kv_heads : 0;     // middle coordinate: which 128-wide row of the token
+    const int head = dm.per_head ? b_i % dm.n_kv_heads : 0;   // middle coordinate: which 128-wide row of the token
     for (int i = 0; i < nb; ++i)
-      tma_load_3d(smem_u32(ring + slot * kStageBytes + i * kBoxBytes), &map_hidden, (box0 + i) * kBoxCols, head, row, bar);
+      tma_load_3d(smem_u32(ring + slot_i * kStageBytes + i * kBoxBytes), &map_hidden, (box0 + i) * kBoxCols, head, row_i, bar);
+    slot_i = slot_i + 1 == kStages ? 0 : slot_i + 1;
+    if (++st_i == n_stages) {
+      st_i = 0;
+      if (++ib_i < my_blocks) block_coords(blk0 + ib_i * blk_stride, b_i, c_i, row_i);
+    }
   };
   if (lane == 0)
-    for (long long u = 0; u < kStages && u < total_units; ++u) issue(u);
+    for (long long u = 0; u < kStages && u < total_units; ++u) issue_next();
 
   // ldmatrix row address of this lane inside a box: matrices (rows 0-7 | 8-15) x (k 0-7 | 8-15)
   const int lm_row = (lane & 7) + ((lane >> 3) & 1) * 8;
@@ -167,7 +173,7 @@ route_score_vote_kernel(Dims dm, int32_t* __restrict__ votes /* [batch][max_chun
         }
       }
       __syncwarp();
-      if (lane == 0 && u + kStages < total_units) issue(u + kStages);
+      if (lane == 0 && u + kStages < total_units) issue_next();
     }
     if (!ok) break;
 #pragma unroll
