@@ -5,7 +5,9 @@ to the host and recomputed by the oracle one by one:
   * router: sampled chunks (vote histograms away from near-ties, winner),
   * quantise+pack: every tile of sampled (sequence, kv head, chunk) slots, byte for byte,
   * decode attention: sampled (sequence, kv head) pairs over the whole context, all four
-    query heads of the group, against the oracle run on the GPU's own packed cache and map.
+    query heads of the group, against the oracle run on the GPU's own packed cache and map,
+  * prefill attention (32k prompt) and the fused projection + quantise (one layer of the 128k
+    workload): sampled rows / slots, each in its own test below.
 """
 import numpy as np
 import pytest
@@ -165,3 +167,67 @@ def test_prefill_attention_sampled_rows_at_the_32k_prompt():
                     got = out[0, t, hq].cpu().numpy().astype(np.float64)
                     err = np.abs(got - want)
                     assert err.max() <= abs_tol and err.max() <= 1e-2 * max(np.abs(want).max(), 1e-30), (h, g, t, err.max())
+
+
+def test_fused_producer_sampled_slots_at_the_layer_size():
+    """moqae_project_quantize_kv at the size the benchmark times it (one layer of the 128k workload:
+    4 x 131072 (+ tail) tokens, d_in 4096, 8 kv heads, seeded mixed map).  Sampled (sequence, chunk, kv
+    head) slots: the rows the kernel rounded are within one unit in the last place (plus the float32
+    accumulation bound) of the oracle's float64 projection of the same hidden rows, and the slot's
+    packed bytes are what the oracle's quantiser makes of the kernel's own rows."""
+    wl = W.WORKLOADS["cfg4"]
+    B, Hkv, chunk, D, dtype = wl.batch, wl.n_kv_heads, wl.chunk, wl.d_in, wl.dtype
+    T = wl.context + 37
+    C = T // chunk
+    dev = "cuda"
+    cfg = mq.make_config(n_layers=1, n_q_heads=wl.n_q_heads, n_kv_heads=Hkv, chunk=chunk, dtype=dtype, d_in=D,
+                         max_tokens=T, batch=B, rs_group=1, rf_first_chunk=1, tail_capacity=chunk)
+    hidden = synth.hidden_states(B, T, D, chunk, dtype, 6161, dev)
+    Wk = synth.normal((Hkv * 128, D), dtype, 6162, dev, std=1.0 / np.sqrt(D))
+    Wv = synth.normal((Hkv * 128, D), dtype, 6163, dev, std=1.0 / np.sqrt(D))
+    Wk[5] *= 10.0                                          # an outlier key channel
+    cache = mq.moqae_cache_bind(cfg, [C, C, C, C])
+    gmap = synth.multinomial_map(B, C, wl.mix, 79)
+    tdt = synth.torch_dtype(dtype)
+    k_r = torch.zeros((B, T, Hkv, 128), dtype=tdt, device=dev)
+    v_r = torch.zeros((B, T, Hkv, 128), dtype=tdt, device=dev)
+    mq.moqae_project_quantize_kv(cfg, hidden, Wk, Wv, T, 0, cache, forced_map=torch.from_numpy(gmap).to(dev),
+                                 k_rounded=k_r, v_rounded=v_r)
+    torch.cuda.synchronize()
+    assert mq.moqae_poll_status(cache) == 0
+    assert (cache.map[0, :, :C].cpu().numpy() == gmap).all()
+    slot, count = O.assign_slots(gmap)
+    assert (cache.slot[0, :, :C].cpu().numpy() == slot).all() and (cache.count[0].cpu().numpy() == count).all()
+    wk, wv = synth.to_u16(Wk), synth.to_u16(Wv)
+
+    def ulp_of(x64):
+        sig, emin = (11, -14) if dtype == 0 else (8, -126)
+        _, e = np.frexp(x64)
+        return np.ldexp(1.0, np.maximum(e, emin + 1) - sig)
+
+    def check_rows(b, t0, t1, h):
+        rows = synth.to_u16(hidden[b, t0:t1])[None]                       # [1, n, D]
+        _, _, K64, V64 = O.project_kv(rows, wk[h * 128:(h + 1) * 128], wv[h * 128:(h + 1) * 128], dtype, 1)
+        absh = np.abs(O.to_f64(rows[0], dtype))
+        for got_t, x64, wm in ((k_r, K64, wk), (v_r, V64, wv)):
+            g = O.to_f64(synth.to_u16(got_t[b, t0:t1, h]), dtype)
+            acc = D * 2.0 ** -24 * (absh @ np.abs(O.to_f64(wm[h * 128:(h + 1) * 128], dtype)).T)
+            assert (np.abs(g - x64[0, :, 0]) <= ulp_of(x64[0, :, 0]) * 1.001 + acc).all(), (b, t0, h)
+
+    rs = np.random.RandomState(8)
+    for w in range(4):                                     # four slots of every width
+        where = np.argwhere(gmap == w)
+        for b, c in where[rs.choice(len(where), 4, replace=False)]:
+            h = rs.randint(Hkv)
+            check_rows(b, c * chunk, (c + 1) * chunk, h)
+            Kc = synth.to_u16(k_r[b, c * chunk:(c + 1) * chunk, h])[None, :, None]
+            Vc = synth.to_u16(v_r[b, c * chunk:(c + 1) * chunk, h])[None, :, None]
+            ref = O.quantize_kv(Kc, Vc, dtype, chunk, gmap[b:b + 1, c:c + 1])
+            got = cache.pool(w)[0, b, h, int(slot[b, c])].cpu().numpy()
+            assert (got == ref["pools"][w][0, 0, 0]).all(), (b, h, c, w)
+    # the trailing tokens stay 16-bit: the tail holds the kernel's rounded rows
+    r = T % chunk
+    assert (cache.tail_len[0].cpu().numpy() == r).all()
+    check_rows(2, C * chunk, T, 6)
+    assert (cache.tail("k")[0, 2, 6, :r].cpu().numpy().view(np.uint16) == synth.to_u16(k_r[2, C * chunk:, 6])).all()
+    assert (cache.tail("v")[0, 2, 6, :r].cpu().numpy().view(np.uint16) == synth.to_u16(v_r[2, C * chunk:, 6])).all()
