@@ -401,6 +401,7 @@ def run_ours(args):
     ms_route = sum(e[0].elapsed_time(e[1]) for e in events) / args.steps
     ms_quant = sum(e[1].elapsed_time(e[2]) for e in events) / args.steps
     ms_dec = sum(e[2].elapsed_time(e[3]) for e in events) / args.steps
+    dec_steps_ms = sorted(e[2].elapsed_time(e[3]) for e in events)          # this rank's decode phase, step by step
 
     # end to end, right after the timed steps (same power state): the decode calls with the
     # queries coming from and the outputs going to pinned host memory, then the whole step with
@@ -448,6 +449,8 @@ def run_ours(args):
                                            if job.overlap else "serialised")},
             "phase_ms": {"route": round(ms_route, 4), "quantize_pack": round(ms_quant, 4),
                          "decode_attn": round(ms_dec, 4)},
+            "decode_ms_per_step": {"mean": round(ms_dec, 4), "median": round(dec_steps_ms[len(dec_steps_ms) // 2], 4),
+                                   "min": round(dec_steps_ms[0], 4), "max": round(dec_steps_ms[-1], 4)},
             "context_tokens_per_s": round(world * wl.batch * job.T * wl.decode_steps / (ms_dec * 1e-3), 1),
             "quantize_route_gbs": round(world * (b_route + b_quant) / ((ms_route + ms_quant) * 1e6), 1),
             "bytes_per_step": {"route": b_route, "quantize_pack": b_quant, "decode_attn": b_dec},
