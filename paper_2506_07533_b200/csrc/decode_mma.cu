@@ -139,6 +139,23 @@ __device__ __forceinline__ void rescale(State& st, float c0, float c1) {
 constexpr float kSlack = 3.0f;
 template <int BITS> __host__ __device__ constexpr int pmax_log2() { return BITS == 2 ? 1 : BITS == 4 ? 3 : BITS == 8 ? 7 : 6; }
 
+// The same for a query group of at most 4, where a lane's even column (2 t4) is query t4 and its odd column is
+// not used: xm0 = this lane's largest score of that query.
+__device__ __forceinline__ void move_reference_even(State& st, float xm0) {
+  if (__any_sync(0xffffffffu, xm0 > st.m[0] + kSlack)) {
+#pragma unroll
+    for (int o = 4; o <= 16; o <<= 1) xm0 = fmaxf(xm0, __shfl_xor_sync(0xffffffffu, xm0, o));
+    const float n0 = fmaxf(st.m[0], xm0);
+    const float c0 = (st.m[0] == -INFINITY) ? 0.0f : ex2f(st.m[0] - n0);
+#pragma unroll
+    for (int mt = 0; mt < 8; ++mt) {
+      st.acc[mt][0] *= c0; st.acc[mt][2] *= c0;
+    }
+    st.oz[0] *= c0; st.oz[2] *= c0;
+    st.m[0] = n0;
+  }
+}
+
 // xm0 / xm1: this lane's largest scores of queries 2t4 / 2t4+1 in the unit about to be weighted
 __device__ __forceinline__ void move_reference(State& st, float xm0, float xm1) {
   const bool over = (xm0 > st.m[0] + kSlack) || (xm1 > st.m[1] + kSlack);
@@ -180,9 +197,11 @@ __device__ __forceinline__ void softmax_update(State& st, float x[NV][4]) {
 // Lane (g, t4) = (lane / 4, lane % 4).  qb[r], r = 0..15: fp16 pair (q'[c_lo(r)], q'[c_hi(r)])
 // of query g (zero for g >= G) for the channels 32*t4 + .. that key register r carries;
 // qc[r] = qb[r] times the power of two that undoes the register's bit position.
-// G4 (query group of at most 4): B columns 4..7 carry the low parts of the folded queries
-// 0..3, so one MMA chain yields both halves of the exact product and the score of query c
-// is column c plus column c + 4; columns 4..7 then simply mirror 0..3 in everything after.
+// G4 (query group of at most 4): B column 2q carries the high part and column 2q + 1 the low part of
+// folded query q, so one MMA chain yields both halves of the exact product and lane (g, t4) finds
+// the two halves of query t4 side by side in its own accumulator registers.  Everything after the
+// scores then works on the lane's even column only (one query per lane, half the weights to
+// compute); the odd columns of P are zero and the odd accumulator columns are never read.
 // NT = 2 (neighbouring 2-bit tiles, fetched by one copy): one reference-maximum check, one set of
 // zero-point MMAs and one round of bias shuffles serve both tiles.
 template <int BITS, int NT, bool G4>
@@ -200,7 +219,7 @@ __device__ __forceinline__ void process_qunit(const uint8_t* __restrict__ unit, 
 #pragma unroll
   for (int tl = 0; tl < NT; ++tl) {
     const uint4* sp = reinterpret_cast<const uint4*>(unit + tl * TB) + t4;
-    const bool lo_lane = G4 && g >= 4;
+    const bool lo_lane = G4 && (g & 1);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const uint4 s4 = sp[4 * i];
@@ -209,7 +228,7 @@ __device__ __forceinline__ void process_qunit(const uint8_t* __restrict__ unit, 
       for (int j = 0; j < 4; ++j) {
         uint32_t hi = hmul2_u32(qc[4 * i + j], sv[j]);
         if (G4) {
-          // lanes of columns 4..7 replace hi by lo = fma(q', s, -hi)
+          // lanes of the odd columns replace hi by lo = fma(q', s, -hi)
           if (lo_lane) hi = hfma2_sub_u32(qc[4 * i + j], sv[j], hi);
         } else {
           ql[G4 ? 0 : tl][(4 * i + j) % (G4 ? 1 : 16)] = hfma2_sub_u32(qc[4 * i + j], sv[j], hi);
@@ -295,11 +314,11 @@ __device__ __forceinline__ void process_qunit(const uint8_t* __restrict__ unit, 
   }
   float bias[NT][2];
   {
-    const float bq = (bd[0] + bd[3]) * lc.cbg;            // query g, tile t4 & 1
+    const float bq = (bd[0] + bd[3]) * lc.cbg;            // query of row g, tile t4 & 1
 #pragma unroll
     for (int tl = 0; tl < NT; ++tl) {
       bias[tl][0] = __shfl_sync(0xffffffffu, bq, 8 * t4 + (NT == 2 ? tl : 0));
-      bias[tl][1] = __shfl_sync(0xffffffffu, bq, 8 * t4 + 4 + (NT == 2 ? tl : 0));
+      bias[tl][1] = G4 ? 0.0f : __shfl_sync(0xffffffffu, bq, 8 * t4 + 4 + (NT == 2 ? tl : 0));
     }
   }
   float v[NB][4];
@@ -309,9 +328,16 @@ __device__ __forceinline__ void process_qunit(const uint8_t* __restrict__ unit, 
     for (int i = 0; i < 4; ++i) {
       float x = sc[b2][0][i];
       if (CH == 2) x += sc[b2][CH - 1][i];
-      if (G4) x += __shfl_xor_sync(0xffffffffu, x, 2);       // column c + column c ^ 4
       v[b2][i] = x;
     }
+  if (G4) {
+    // high part (even column) + low part (odd column) of the lane's query, rows g and g + 8
+#pragma unroll
+    for (int b2 = 0; b2 < NB; ++b2) {
+      v[b2][0] += v[b2][1];
+      v[b2][2] += v[b2][3];
+    }
+  }
   if (n_valid < kTileTokens) {
     // tiles of a chunk shorter than 32 tokens: positions n_valid (8 or 16) .. 31 are padding and get
     // weight zero (row g of block 0 is token g, row g + 8 token g + 8, block 1 tokens 16..31)
@@ -325,7 +351,27 @@ __device__ __forceinline__ void process_qunit(const uint8_t* __restrict__ unit, 
 
   // softmax: the factor cs > 0 and the per-tile bias commute with the maximum, so the reference
   // check runs on the raw sums and every weight costs one FMA and one ex2
-  {
+  if (G4) {
+    float xm0 = -INFINITY;
+#pragma unroll
+    for (int tl = 0; tl < NT; ++tl) {
+      const float r0 = fmaxf(fmaxf(v[2 * tl][0], v[2 * tl][2]), fmaxf(v[2 * tl + 1][0], v[2 * tl + 1][2]));
+      xm0 = fmaxf(xm0, fmaf(r0, lc.cs[0], bias[tl][0]));
+    }
+    move_reference_even(st, xm0);
+    constexpr float kPmaxLog2 = static_cast<float>(pmax_log2<BITS>());
+    const float o0 = (kPmaxLog2 - kSlack) - st.m[0];
+#pragma unroll
+    for (int tl = 0; tl < NT; ++tl) {
+      const float ob0 = bias[tl][0] + o0;
+#pragma unroll
+      for (int blk = 0; blk < 2; ++blk) {
+        float* x = v[2 * tl + blk];
+        x[0] = ex2f(fmaf(x[0], lc.cs[0], ob0)); x[1] = 0.0f;
+        x[2] = ex2f(fmaf(x[2], lc.cs[0], ob0)); x[3] = 0.0f;
+      }
+    }
+  } else {
     float xm0 = -INFINITY, xm1 = -INFINITY;
 #pragma unroll
     for (int tl = 0; tl < NT; ++tl) {
@@ -430,7 +476,7 @@ __device__ __forceinline__ void load_q_phase(uint32_t (&qb)[16], uint32_t (&qc)[
 // ---- 16 raw rows (pool tile half or tail block) from shared memory ---------------------
 // ks/vs: 16 rows x 256 B, 16-byte units swizzled by (row & 7).  qr[r]: q pairs of the raw
 // channel set (units 2t4, 2t4+1, 8+2t4, 9+2t4) in the INPUT dtype.
-template <bool BF16>
+template <bool BF16, bool G4>
 __device__ __forceinline__ void process_raw16(const uint8_t* __restrict__ ks, const uint8_t* __restrict__ vs,
                                               int n_valid, State& st, const uint32_t (&qr)[16], float c_score, int lane) {
   const int g = lane >> 2, t4 = lane & 3;
@@ -446,10 +492,18 @@ __device__ __forceinline__ void process_raw16(const uint8_t* __restrict__ ks, co
   }
   float x[1][4];
   x[0][0] = (g < n_valid) ? (s0[0] + s1[0]) * c_score : -INFINITY;
-  x[0][1] = (g < n_valid) ? (s0[1] + s1[1]) * c_score : -INFINITY;
   x[0][2] = (g + 8 < n_valid) ? (s0[2] + s1[2]) * c_score : -INFINITY;
-  x[0][3] = (g + 8 < n_valid) ? (s0[3] + s1[3]) * c_score : -INFINITY;
-  softmax_update<1>(st, x);
+  if (G4) {
+    // a query group of at most 4: the lane's even column is its query, the odd one (the same query again) is not used
+    move_reference_even(st, fmaxf(x[0][0], x[0][2]));
+    const float o0 = (static_cast<float>(pmax_log2<16>()) - kSlack) - st.m[0];
+    x[0][0] = ex2f(x[0][0] + o0); x[0][1] = 0.0f;
+    x[0][2] = ex2f(x[0][2] + o0); x[0][3] = 0.0f;
+  } else {
+    x[0][1] = (g < n_valid) ? (s0[1] + s1[1]) * c_score : -INFINITY;
+    x[0][3] = (g + 8 < n_valid) ? (s0[3] + s1[3]) * c_score : -INFINITY;
+    softmax_update<1>(st, x);
+  }
   uint32_t p0, p1, q0 = 0u, q1 = 0u;
   if (BF16) {   // p~ = hi + lo, both bf16, so the weights keep ~16 bits
     const uint32_t h01 = pack_bf162(x[0][0], x[0][1]), h23 = pack_bf162(x[0][2], x[0][3]);
@@ -587,7 +641,7 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
   int q_exp[8];
 #pragma unroll
   for (int qi = 0; qi < 8; ++qi) {
-    const int qs = G4 ? (qi & 3) : qi;                        // G4: rows 4..7 mirror rows 0..3
+    const int qs = G4 ? (qi >> 1) : qi;                       // G4: rows 2q and 2q + 1 both hold query q
     float mx = 0.0f;
     if (qs < G) {
       const uint2 raw4 = *reinterpret_cast<const uint2*>(q + (static_cast<long long>(b) * dm.n_q_heads + h * G + qs) * kHeadDim + 4 * lane);
@@ -605,7 +659,7 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
   for (int i = threadIdx.x; i < 8 * kHeadDim; i += kThreads) {
     const int qi = i / kHeadDim, c = i % kHeadDim;
     uint16_t raw = 0;
-    const int qs = G4 ? (qi & 3) : qi;
+    const int qs = G4 ? (qi >> 1) : qi;
     if (qs < G) raw = q[(static_cast<long long>(b) * dm.n_q_heads + h * G + qs) * kHeadDim + c];
     q_in[i] = raw;
     int e = 0;
@@ -728,7 +782,7 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
           },
           [&](const uint8_t* stg, int u) {
             const int nv = min(16, n_valid - 16 * (u & 1));   // a short chunk's tile: rows past n_valid are padding
-            if (nv > 0) process_raw16<BF16>(stg, stg + 4096, nv, st, qr, c_bias, lane);
+            if (nv > 0) process_raw16<BF16, G4>(stg, stg + 4096, nv, st, qr, c_bias, lane);
           }, my_ring);
       phase_scale<16>(st, false);
     }
@@ -761,7 +815,7 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
         *reinterpret_cast<uint4*>(stg + 4096 + row * 256 + up * 16) = vv;
       }
       __syncwarp();
-      process_raw16<BF16>(stg, stg + 4096, nv, st, qr, c_bias, lane);
+      process_raw16<BF16, G4>(stg, stg + 4096, nv, st, qr, c_bias, lane);
     }
     phase_scale<16>(st, false);
   }
@@ -779,12 +833,12 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
     const int ch = 32 * cg + 4 * g + 2 * (mt & 1);
     float* o0 = red_o + (warp * 8 + 2 * t4) * kHeadDim;
     float* o1 = o0 + kHeadDim;
-    o0[ch] = st.acc[mt][0] + z0; o1[ch] = st.acc[mt][1] + z1;
-    o0[ch + 1] = st.acc[mt][2] + z0; o1[ch + 1] = st.acc[mt][3] + z1;
+    o0[ch] = st.acc[mt][0] + z0; o0[ch + 1] = st.acc[mt][2] + z0;
+    if (!G4) { o1[ch] = st.acc[mt][1] + z1; o1[ch + 1] = st.acc[mt][3] + z1; }     // G4: odd columns are not used
   }
   if (g == 4) {                          // this lane's oz row holds the sums
     red_ml[(warp * 8 + 2 * t4) * 2] = st.m[0]; red_ml[(warp * 8 + 2 * t4) * 2 + 1] = st.oz[0];
-    red_ml[(warp * 8 + 2 * t4 + 1) * 2] = st.m[1]; red_ml[(warp * 8 + 2 * t4 + 1) * 2 + 1] = st.oz[1];
+    if (!G4) { red_ml[(warp * 8 + 2 * t4 + 1) * 2] = st.m[1]; red_ml[(warp * 8 + 2 * t4 + 1) * 2 + 1] = st.oz[1]; }
   }
   __syncthreads();
   // Everything up to here only read the caller's inputs and worked in registers and shared memory.
@@ -794,16 +848,17 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
   if (timed_out && lane == 0) set_status(cv.status, MOQAE_ERR_TIMEOUT, blockIdx.x, warp);
   for (int i = threadIdx.x; i < G * kHeadDim; i += kThreads) {
     const int qi = i / kHeadDim, c = i % kHeadDim;
+    const int col = G4 ? 2 * qi : qi;      // fragment column (row of the reduction buffers) that holds query qi
     float m = -INFINITY;
 #pragma unroll
-    for (int wv = 0; wv < kWarps; ++wv) m = fmaxf(m, red_ml[(wv * 8 + qi) * 2]);
+    for (int wv = 0; wv < kWarps; ++wv) m = fmaxf(m, red_ml[(wv * 8 + col) * 2]);
     float l = 0.0f, o = 0.0f;
 #pragma unroll
     for (int wv = 0; wv < kWarps; ++wv) {
-      const float mw = red_ml[(wv * 8 + qi) * 2];
+      const float mw = red_ml[(wv * 8 + col) * 2];
       const float f = (mw == -INFINITY) ? 0.0f : ex2f(mw - m);
-      l += red_ml[(wv * 8 + qi) * 2 + 1] * f;
-      o += red_o[(wv * 8 + qi) * kHeadDim + c] * f;
+      l += red_ml[(wv * 8 + col) * 2 + 1] * f;
+      o += red_o[(wv * 8 + col) * kHeadDim + c] * f;
     }
     const long long row = (static_cast<long long>(b) * dm.n_q_heads + h * G + qi) * n_splits + split;
     ws_o[row * kHeadDim + c] = o;
