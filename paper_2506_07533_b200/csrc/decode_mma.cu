@@ -572,22 +572,32 @@ struct Pipe {
 
 // Stream `n_units` units of `unit_bytes` (each made of `pieces` bulk copies) through the ring.
 // UNIT_BYTES / STAGES are compile-time; src(u, piece) gives each piece's global address.
+// expect_tx + one bulk copy, executed by the whole warp without a branch: only the lane with `on` set acts
+__device__ __forceinline__ void issue_copy(bool on, uint32_t bar, uint32_t dst, const void* src, uint32_t bytes, bool expect,
+                                           uint32_t expect_bytes) {
+  asm volatile("{\n.reg .pred p, q;\nsetp.ne.b32 p, %4, 0;\nsetp.ne.b32 q, %5, 0;\n"
+               "@q mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %6;\n"
+               "@p cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%1], [%2], %3, [%0];\n}\n"
+               ::"r"(bar), "r"(dst), "l"(src), "r"(bytes), "r"(on ? 1 : 0), "r"((on && expect) ? 1 : 0), "r"(expect_bytes) : "memory");
+}
+
 template <int STAGES, int STAGE_BYTES, int PIECES, typename SrcFn, typename ConsumeFn>
 __device__ __forceinline__ void stream_units(Pipe& pp, int n_units, int lane, SrcFn src, ConsumeFn consume,
                                              const uint8_t* ring_generic, uint32_t last_unit_bytes = STAGE_BYTES) {
   if (n_units <= 0 || !pp.ok) return;
-  auto issue = [&](int u) {              // lane 0; the last unit of the stream may be shorter
+  // issued by the whole warp, predicated on lane 0 and on the unit's existence (no divergent branch)
+  auto issue = [&](int u, bool on) {     // the last unit of the stream may be shorter
     const uint32_t bytes = (u == n_units - 1) ? last_unit_bytes : STAGE_BYTES;
     const uint32_t piece_bytes = bytes / PIECES;
     const int s = u % STAGES;
     const uint32_t bar = pp.bars + 8 * s;
-    mbar_expect_tx(bar, bytes);
 #pragma unroll
-    for (int p = 0; p < PIECES; ++p) bulk_load(pp.ring + s * STAGE_BYTES + p * piece_bytes, src(u, p), piece_bytes, bar);
+    for (int p = 0; p < PIECES; ++p)
+      issue_copy(on, bar, pp.ring + s * STAGE_BYTES + p * piece_bytes, src(on ? u : 0, p), piece_bytes, p == 0, bytes);
   };
-  if (lane == 0) {
+  {
     const int pre = n_units < STAGES ? n_units : STAGES;
-    for (int u = 0; u < pre; ++u) issue(u);
+    for (int u = 0; u < pre; ++u) issue(u, lane == 0);
   }
   for (int u = 0; u < n_units; ++u) {
     const int s = u % STAGES;
@@ -602,7 +612,7 @@ __device__ __forceinline__ void stream_units(Pipe& pp, int n_units, int lane, Sr
     pp.parity ^= (1u << s);
     consume(ring_generic + s * STAGE_BYTES, u);
     __syncwarp();
-    if (lane == 0 && u + STAGES < n_units) issue(u + STAGES);
+    issue(u + STAGES, lane == 0 && u + STAGES < n_units);
   }
 }
 
