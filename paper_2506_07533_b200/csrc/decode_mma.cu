@@ -149,9 +149,9 @@ __device__ __forceinline__ void move_reference_even(State& st, float xm0) {
     const float c0 = (st.m[0] == -INFINITY) ? 0.0f : ex2f(st.m[0] - n0);
 #pragma unroll
     for (int mt = 0; mt < 8; ++mt) {
-      st.acc[mt][0] *= c0; st.acc[mt][2] *= c0;
+      st.acc[mt][0] *= c0; st.acc[mt][1] *= c0; st.acc[mt][2] *= c0; st.acc[mt][3] *= c0;
     }
-    st.oz[0] *= c0; st.oz[2] *= c0;
+    st.oz[0] *= c0; st.oz[1] *= c0; st.oz[2] *= c0; st.oz[3] *= c0;
     st.m[0] = n0;
   }
 }
@@ -201,7 +201,8 @@ __device__ __forceinline__ void softmax_update(State& st, float x[NV][4]) {
 // folded query q, so one MMA chain yields both halves of the exact product and lane (g, t4) finds
 // the two halves of query t4 side by side in its own accumulator registers.  Everything after the
 // scores then works on the lane's even column only (one query per lane, half the weights to
-// compute); the odd columns of P are zero and the odd accumulator columns are never read.
+// compute); for quantised tiles the odd columns of P are zero, 16-bit bf16 tiles put the low parts of their
+// weights there, and a query's result is its even plus its odd accumulator column.
 // NT = 2 (neighbouring 2-bit tiles, fetched by one copy): one reference-maximum check, one set of
 // zero-point MMAs and one round of bias shuffles serve both tiles.
 template <int BITS, int NT, bool G4>
@@ -505,7 +506,13 @@ __device__ __forceinline__ void process_raw16(const uint8_t* __restrict__ ks, co
     softmax_update<1>(st, x);
   }
   uint32_t p0, p1, q0 = 0u, q1 = 0u;
-  if (BF16) {   // p~ = hi + lo, both bf16, so the weights keep ~16 bits
+  constexpr bool kLowInOddColumn = BF16 && G4;   // the odd column of a lane's query carries the low part: one product instead of two
+  if (kLowInOddColumn) {
+    const uint32_t h0 = pack_bf162(x[0][0], 0.0f), h2 = pack_bf162(x[0][2], 0.0f);
+    const float r0 = x[0][0] - __uint_as_float(h0 << 16), r2 = x[0][2] - __uint_as_float(h2 << 16);
+    p0 = movmatrix_trans(pack_bf162(__uint_as_float(h0 << 16), r0));
+    p1 = movmatrix_trans(pack_bf162(__uint_as_float(h2 << 16), r2));
+  } else if (BF16) {   // p~ = hi + lo, both bf16, so the weights keep ~16 bits
     const uint32_t h01 = pack_bf162(x[0][0], x[0][1]), h23 = pack_bf162(x[0][2], x[0][3]);
     const float r0 = x[0][0] - __uint_as_float(h01 << 16), r1 = x[0][1] - __uint_as_float(h01 & 0xffff0000u);
     const float r2 = x[0][2] - __uint_as_float(h23 << 16), r3 = x[0][3] - __uint_as_float(h23 & 0xffff0000u);
@@ -518,7 +525,7 @@ __device__ __forceinline__ void process_raw16(const uint8_t* __restrict__ ks, co
   {  // running sums: a row of ones in oz row 4
     const uint32_t ones = (g == 4) ? (BF16 ? 0x3F803F80u : 0x3C003C00u) : 0u;
     mma16816<BF16>(st.oz, ones, 0u, ones, 0u, p0, p1);
-    if (BF16) mma16816<BF16>(st.oz, ones, 0u, ones, 0u, q0, q1);
+    if (BF16 && !kLowInOddColumn) mma16816<BF16>(st.oz, ones, 0u, ones, 0u, q0, q1);
   }
 #pragma unroll
   for (int cg = 0; cg < 4; ++cg) {
@@ -538,7 +545,7 @@ __device__ __forceinline__ void process_raw16(const uint8_t* __restrict__ ks, co
       const uint32_t a0 = __byte_perm(w0, w1, 0x5410), a1 = __byte_perm(w0, w1, 0x7632);
       const uint32_t a2 = __byte_perm(w2, w3, 0x5410), a3 = __byte_perm(w2, w3, 0x7632);
       mma16816<BF16>(st.acc[2 * cg + hf], a0, a1, a2, a3, p0, p1);
-      if (BF16) mma16816<BF16>(st.acc[2 * cg + hf], a0, a1, a2, a3, q0, q1);
+      if (BF16 && !kLowInOddColumn) mma16816<BF16>(st.acc[2 * cg + hf], a0, a1, a2, a3, q0, q1);
     }
   }
 }
@@ -843,11 +850,15 @@ decode_mma_kernel(Dims dm, CacheView cv, const uint16_t* __restrict__ q, int lay
     const int ch = 32 * cg + 4 * g + 2 * (mt & 1);
     float* o0 = red_o + (warp * 8 + 2 * t4) * kHeadDim;
     float* o1 = o0 + kHeadDim;
-    o0[ch] = st.acc[mt][0] + z0; o0[ch + 1] = st.acc[mt][2] + z0;
-    if (!G4) { o1[ch] = st.acc[mt][1] + z1; o1[ch + 1] = st.acc[mt][3] + z1; }     // G4: odd columns are not used
+    if (G4) {   // the odd column holds what 16-bit tiles added through the low parts of their weights (zero otherwise)
+      o0[ch] = (st.acc[mt][0] + z0) + (st.acc[mt][1] + z1); o0[ch + 1] = (st.acc[mt][2] + z0) + (st.acc[mt][3] + z1);
+    } else {
+      o0[ch] = st.acc[mt][0] + z0; o0[ch + 1] = st.acc[mt][2] + z0;
+      o1[ch] = st.acc[mt][1] + z1; o1[ch + 1] = st.acc[mt][3] + z1;
+    }
   }
   if (g == 4) {                          // this lane's oz row holds the sums
-    red_ml[(warp * 8 + 2 * t4) * 2] = st.m[0]; red_ml[(warp * 8 + 2 * t4) * 2 + 1] = st.oz[0];
+    red_ml[(warp * 8 + 2 * t4) * 2] = st.m[0]; red_ml[(warp * 8 + 2 * t4) * 2 + 1] = G4 ? st.oz[0] + st.oz[1] : st.oz[0];
     if (!G4) { red_ml[(warp * 8 + 2 * t4 + 1) * 2] = st.m[1]; red_ml[(warp * 8 + 2 * t4 + 1) * 2 + 1] = st.oz[1]; }
   }
   __syncthreads();
