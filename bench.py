@@ -33,9 +33,9 @@ L2_BYTES = 126 * 1024 * 1024
 
 # dram__bytes_read.sum + dram__bytes_write.sum of ONE decode_mma_kernel launch (one cfg4 layer at full
 # context, realised mix 57.7/31.4/6.4/4.5), from the ncu capture summarised in
-# profiles/decode_mma_kernel_cfg4.txt: 617.83 MB + 5.76 MB against 619.0 MB of algorithmic bytes.
+# profiles/decode_mma_kernel_cfg4.txt: 617.81 MB + 5.65 MB against 619.0 MB of algorithmic bytes.
 # Reported only for the workload and launch shape it was taken on.
-NCU_DECODE_TRAFFIC = {"cfg4": 623593728}
+NCU_DECODE_TRAFFIC = {"cfg4": 623457536}
 
 
 def read_peaks():
